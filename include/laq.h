@@ -1,0 +1,198 @@
+/*
+ * laq.h -- C ABI of the B200 (sm_100a) LAQ library.
+ *
+ * LAQ = Lazily Aggregated Quantized gradients (Sun, Chen, Giannakis, Yang, NeurIPS 2019).
+ * The library runs Algorithm 2 of the paper for M workers simulated on ONE GPU.  One iteration is
+ *   1. every worker's local gradient g_m = grad f_m(theta^k)                       (Algorithm 2, worker step)
+ *   2. the b-bit innovation quantizer: R_m = ||g_m - Q_m(theta_hat^{k-1})||_inf,
+ *      tau = 1/(2^b-1), codes q = floor((g_m - Q_prev + R_m)/(2 tau R_m) + 1/2)     (Sec. 2.1, Eq. (5))
+ *      and the innovation dQ_m = 2 tau R_m q - R_m 1                               (Sec. 2.1, Eq. (6))
+ *   3. the squared norms ||dQ_m||^2 and ||eps_m||^2, eps_m = g_m - (Q_prev + dQ_m)  (Sec. 2.1, Sec. 2.2)
+ *   4. the skip rule (7a) with the staleness clock (7b)                            (Sec. 2.2, Eq. (7a), (7b))
+ *   5. grad^k = grad^{k-1} + sum_{uploading m} dQ_m ; theta^{k+1} = theta^k - alpha grad^k   (Eq. (4))
+ * All five steps run in CUDA kernels; there is no CPU fallback.
+ *
+ * Conventions
+ *   - Every pointer is marked HOST or DEVICE.  The caller owns every buffer, including the device
+ *     workspace and the CUDA stream; the library owns only the laq_ctx it returns.
+ *   - All device work is enqueued on the stream given to laq_init.
+ *   - No function throws, aborts or traps the device.  Every fallible function returns a laq_status;
+ *     laq_last_error() gives a text for the most recent failure on that context.
+ *   - Conditions detected on the device (a non-finite gradient or radius) freeze the state at the
+ *     iteration where they occurred and are reported by the next call that synchronises
+ *     (laq_step with a trace, laq_get_state, laq_sync) as LAQ_ENONFINITE.
+ *   - Floating point: theta, gradients and quantizer state are fp32; each quantizer operation is one
+ *     IEEE round-to-nearest operation in the order  d = g - Q_prev ; R = max|d| ; s = (2 tau) R ;
+ *     t = (d + R)/s + 1/2 ; q = clamp(floor t) ; dQ = s q - R ; Q_new = Q_prev + dQ ; eps = g - Q_new,
+ *     with no fused multiply-add; squared norms are fp64 sums of exact fp32 products; the skip rule
+ *     is evaluated in fp64.
+ *   - Code stream of worker m (the paper's b p-bit part of the upload message): code i occupies bits
+ *     [(i b) mod 32, +b) of 32-bit word floor(i b / 32), least significant first.
+ *   - Readings where the paper is silent: initial Q_m = 0, ||eps_hat_m||^2 = 0, grad^0 = 0, the D stored
+ *     squared parameter differences start at 0, clocks start at t_bar + 1 (every worker uploads at
+ *     k = 1); R_m = 0 yields q = 0, dQ = 0; ||theta^{k+1}-theta^k||^2 is taken as ||alpha grad^k||^2.
+ */
+#ifndef LAQ_B200_H
+#define LAQ_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct laq_ctx laq_ctx;
+
+typedef enum {
+  LAQ_OK = 0,
+  LAQ_EINVAL = 1,      /* bad argument or unsupported configuration */
+  LAQ_EWORKSPACE = 2,  /* workspace pointer null, misaligned (256 B) or too small */
+  LAQ_ECUDA = 3,       /* a CUDA runtime call failed */
+  LAQ_ENONFINITE = 4,  /* a gradient or radius was inf/nan; state frozen at that iteration */
+  LAQ_ESTATE = 5       /* call not valid in the context's current state (e.g. shards missing) */
+} laq_status;
+
+/* Which f_m the workers hold (supplement, "Simulation details"; global loss f = (1/N) sum_m f_m,
+ * every sample loss carries (lambda/2)||theta||^2, so worker m adds (N_m/N) lambda theta). */
+typedef enum {
+  LAQ_MODEL_LOGREG_BIN = 0, /* z = x.theta, loss softplus(z) - y z, y in {0,1}; p = n_features (<= 256) */
+  LAQ_MODEL_SOFTMAX = 1,    /* softmax(theta x), theta [n_classes x n_features] row-major; p = C F */
+  LAQ_MODEL_MLP2 = 2,       /* ReLU network F-H-C; theta = W1[H x F], b1[H], W2[C x H], b2[C];
+                               the products X W1^T and dH^T X take bf16 operands, fp32 accumulation */
+  LAQ_MODEL_SYNTH = 3,      /* no data: g_m^k[i] generated in the kernels from (seed, m, i, k), see below */
+  LAQ_MODEL_EXTERNAL = 4    /* the caller supplies g (M x p) before every step with laq_set_gradients */
+} laq_model;
+
+/* LAQ_MODEL_SYNTH stream (fp32, every operation IEEE, no fused multiply-add):
+ *   fmix32(x): x ^= x>>16; x *= 0x85ebca6b; x ^= x>>13; x *= 0xc2b2ae35; x ^= x>>16
+ *   key_m = fmix32(seed_lo ^ fmix32(seed_hi + 0x9e3779b9 (m+1))),  h = fmix32((uint32) i ^ key_m)
+ *   with bytes b0..b3 of h (b0 lowest): zi = b0+b1+b2+b3-510, wi = b0-b1+b2-b3,
+ *   cz = fp32(synth_sigma / sqrt(21845)), eta_m = fp32(synth_eta0 (m+1)/M),
+ *   g_m^k[i] = zi cz + (k eta_m)(wi cz),  k = 1, 2, ...   (requires p < 2^32) */
+
+enum {
+  LAQ_FLAG_TRIGGER_OFF = 2u /* every worker uploads every iteration: Algorithm 1 (QGD) */
+};
+
+typedef struct {
+  int32_t model;            /* laq_model */
+  int32_t M;                /* number of workers, 1..1024 */
+  int64_t p;                /* dimension of theta (checked against the model shape) */
+  const int64_t* N;         /* HOST, length M: samples per worker {N_m}; ignored for SYNTH / EXTERNAL */
+  int32_t n_features;       /* F */
+  int32_t n_classes;        /* C (SOFTMAX: 2..16, MLP2) */
+  int32_t n_hidden;         /* H (MLP2) */
+  float alpha;              /* step size */
+  float lambda;             /* l2 regulariser */
+  int32_t b;                /* bits per coordinate: 1, 2, 4, 8 or 16 */
+  int32_t D;                /* number of stored parameter differences, 1..64; the paper requires D <= t_bar */
+  const float* xi;          /* HOST, length D: weights xi_1..xi_D of (7a), xi[0] pairs with the newest difference */
+  int32_t tbar;             /* staleness bound of (7b) */
+  int32_t clock_mode;       /* 0: Algorithm 2 as printed, skip allowed while t_m <= t_bar;
+                               1: strict, skip needs t_m + 2 <= t_bar (t_bar = 1 never skips) */
+  uint32_t flags;           /* LAQ_FLAG_* */
+  uint64_t seed;            /* SYNTH only */
+  float synth_sigma;        /* SYNTH only */
+  float synth_eta0;         /* SYNTH only */
+  int32_t trace_capacity;   /* per-iteration records kept on the device for laq_step's trace (0 = none) */
+} laq_config;
+
+/* Per-iteration report of laq_step.  All pointers HOST, each may be NULL; n = n_iters of that call.
+ * Row j describes the j-th iteration of the call. */
+typedef struct {
+  uint8_t* skip;     /* [n][M]  1 = worker skipped the upload, 0 = uploaded */
+  float* R;          /* [n][M]  radius R_m^k */
+  double* n_dq;      /* [n][M]  ||dQ_m^k||^2 */
+  double* n_eps;     /* [n][M]  ||eps_m^k||^2 */
+  double* rhs;       /* [n][M]  right-hand side of (7a) */
+  double* dtheta2;   /* [n]     ||theta^{k+1}-theta^k||^2 */
+  double* loss;      /* [n]     f(theta^k) (model workloads; 0 for SYNTH / EXTERNAL) */
+  int32_t* uploads;  /* [n]     |M^k| */
+} laq_trace;
+
+/* Explicit state for laq_get_state / laq_set_state.  All pointers HOST, each may be NULL (skipped).
+ * Together with the configuration and the shards, the fields marked (S) determine every later
+ * iteration; the others are read-only views of the last iteration. */
+typedef struct {
+  float* theta;       /* (S) [p]        theta^k */
+  float* agg;         /* (S) [p]        grad^{k-1}, the server's lazily aggregated gradient */
+  float* qprev;       /* (S) [M][p]     Q_m(theta_hat_m^{k-1}) */
+  double* n_eps_hat;  /* (S) [M]        ||eps_hat_m||^2, the error at worker m's last upload */
+  int32_t* clock;     /* (S) [M]        t_m */
+  double* ring;       /* (S) [D]        stored squared differences, newest first */
+  int64_t* counters;  /* (S) [3]        iterations done, uploads so far, bits so far (uploads x (32 + b p)) */
+  float* g;           /*     [M][p]     last local gradients (not for SYNTH) */
+  uint32_t* codes;    /*     [M][W]     last code streams, W = ceil(p b / 32) words per worker */
+  float* R;           /*     [M]        last radii */
+  double* n_dq;       /*     [M]        last ||dQ_m||^2 */
+  double* n_eps;      /*     [M]        last ||eps_m||^2 */
+  uint8_t* skip;      /*     [M]        last skip mask */
+} laq_state;
+
+/* Device memory the caller must provide for this configuration (bytes).  0 if the configuration is
+ * invalid.  Holds theta, grad, Q_prev, g, code streams, the resident shards and kernel scratch. */
+size_t laq_workspace_bytes(const laq_config* cfg /* HOST */);
+
+/* Create a context (Algorithm 2, "Initialize").  d_workspace: DEVICE, 256-byte aligned, at least
+ * laq_workspace_bytes(cfg) bytes, owned by the caller and kept alive until laq_destroy.
+ * theta0: HOST, length p, or NULL for zeros.  cuda_stream: a cudaStream_t (NULL = default stream).
+ * The configuration (including N and xi) is copied.  Returns LAQ_EINVAL / LAQ_EWORKSPACE / LAQ_ECUDA. */
+laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, size_t workspace_bytes,
+                    const float* theta0, void* cuda_stream);
+
+/* Make worker m's shard resident (Eq. (1): the N_m samples of f_m).  X: [N_m][n_features] fp32
+ * row-major, y: [N_m] int32 labels (0/1 for LOGREG_BIN, 0..C-1 otherwise); both HOST if
+ * on_device == 0, DEVICE otherwise.  The data is copied into the workspace.  N_m must equal cfg.N[m]. */
+laq_status laq_load_shards(laq_ctx* ctx, int32_t m, const float* X, const int32_t* y, int64_t N_m,
+                           int32_t on_device);
+
+/* LAQ_MODEL_EXTERNAL: provide the M x p local gradients of the next iteration (row m = g_m).
+ * HOST if on_device == 0, DEVICE otherwise; copied into the workspace. */
+laq_status laq_set_gradients(laq_ctx* ctx, const float* g, int32_t on_device);
+
+/* Run n_iters iterations of Algorithm 2 (for EXTERNAL: n_iters must be 1).  With trace == NULL the
+ * call only enqueues work on the stream and returns.  With a trace (n_iters <= trace_capacity) it
+ * synchronises once at the end, fills the HOST arrays and reports device-detected errors. */
+laq_status laq_step(laq_ctx* ctx, int32_t n_iters, const laq_trace* trace);
+
+/* Wait for the stream and report device-detected errors. */
+laq_status laq_sync(laq_ctx* ctx);
+
+/* Copy state to HOST buffers (synchronises).  Returns LAQ_ENONFINITE if the state is frozen. */
+laq_status laq_get_state(laq_ctx* ctx, const laq_state* out);
+
+/* One worker's rows after the last iteration (synchronises): qprev [p] = Q_m(theta_hat_m), g [p] = its
+ * last local gradient (not for SYNTH), and the upload message of Eq. (6): the radius R (one float) and the
+ * code stream codes [ceil(p b / 32)] words.  All HOST, each may be NULL. */
+laq_status laq_get_worker(laq_ctx* ctx, int32_t m, float* qprev, float* g, uint32_t* codes, float* R);
+
+/* Overwrite the (S) fields that are non-NULL (resume from a saved state; synchronises). */
+laq_status laq_set_state(laq_ctx* ctx, const laq_state* in);
+
+/* Number of kernels the library has launched on this context so far. */
+int64_t laq_kernel_launches(const laq_ctx* ctx);
+
+/* Launch-shape override for measurement sweeps: key "sweep_threads", "sweep_blocks_per_sm",
+ * "agg_threads", "agg_blocks_per_sm", "grad_blocks_per_worker".  Values outside the documented
+ * limits return LAQ_EINVAL and change nothing. */
+laq_status laq_tune(laq_ctx* ctx, const char* key, int32_t value);
+
+/* Per-kernel device timing for measurement.  While enabled, laq_step brackets every stage of an iteration
+ * with CUDA events on the context's stream (up to 512 iterations per call are recorded).
+ * laq_kernel_times synchronises and returns, summed since the last call to it, the milliseconds and the
+ * launch counts of the four stages: [0] local gradient, [1] radius, [2] quantize + norms + trigger,
+ * [3] lazy aggregate + theta step.  ms and launches: HOST arrays of 4. */
+laq_status laq_set_profiling(laq_ctx* ctx, int32_t enabled);
+laq_status laq_kernel_times(laq_ctx* ctx, double* ms, int64_t* launches);
+
+/* Text of the last failure on this context ("" if none).  Valid until the next call on ctx. */
+const char* laq_last_error(const laq_ctx* ctx);
+
+/* Free the context (not the workspace).  Waits for the stream first.  NULL is allowed. */
+void laq_destroy(laq_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LAQ_B200_H */

@@ -1,0 +1,611 @@
+// Host side of the C ABI declared in laq.h: configuration checks, carving of the caller's device
+// workspace, and the per-iteration launch plan of Algorithm 2.  No arithmetic of the method runs
+// on the host; every step of the iteration is a kernel (laq_sweeps.cu, laq_grad_*.cu).
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "laq_internal.cuh"
+
+using namespace laq;
+
+struct laq_ctx {
+  laq_config cfg;
+  std::vector<int64_t> N;
+  std::vector<float> xi;
+  Params P;
+  LaunchShape ls;
+  cudaStream_t st = nullptr;
+  int64_t launches = 0;
+  std::string err;
+  std::vector<char> shard_loaded;
+  bool ext_g_set = false;
+  int gbpw = 1, gbpw_cap = 1;
+  char* ws = nullptr;
+  size_t ws_bytes = 0;
+  std::vector<const float*> Xptr;
+  std::vector<const int32_t*> yptr;
+  MlpPlan mlp;
+  // optional per-stage timing
+  bool profiling = false;
+  std::vector<cudaEvent_t> ev;        // kProfIters x 5 events
+  int ev_used = 0;                    // iterations recorded and not yet read
+  double stage_ms[4] = {0, 0, 0, 0};
+  int64_t stage_launches[4] = {0, 0, 0, 0};
+};
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kMaxAggBlocks = kNumSMs * 32;
+constexpr int kGradBlocksCap = 64;
+constexpr int kProfIters = 512;
+
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+bool valid_b(int b) { return b == 1 || b == 2 || b == 4 || b == 8 || b == 16; }
+
+long long model_p(const laq_config& c) {
+  switch (c.model) {
+    case LAQ_MODEL_LOGREG_BIN: return c.n_features;
+    case LAQ_MODEL_SOFTMAX: return (long long)c.n_classes * c.n_features;
+    case LAQ_MODEL_MLP2:
+      return (long long)c.n_hidden * c.n_features + c.n_hidden + (long long)c.n_classes * c.n_hidden + c.n_classes;
+    default: return c.p;
+  }
+}
+
+const char* check_config(const laq_config* c) {
+  if (!c) return "config is null";
+  if (c->model < 0 || c->model > LAQ_MODEL_EXTERNAL) return "unknown model";
+  if (c->M < 1 || c->M > kMaxWorkers) return "M must be in 1..1024";
+  if (c->p < 1) return "p must be positive";
+  if (!valid_b(c->b)) return "b must be 1, 2, 4, 8 or 16";
+  if (c->D < 1 || c->D > kMaxD) return "D must be in 1..64";
+  if (!c->xi) return "xi is null";
+  if (!(c->alpha > 0.f) || !std::isfinite(c->alpha)) return "alpha must be positive and finite";
+  if (c->clock_mode != 0 && c->clock_mode != 1) return "clock_mode must be 0 or 1";
+  if (c->trace_capacity < 0) return "trace_capacity must be >= 0";
+  if (c->flags & ~(uint32_t)LAQ_FLAG_TRIGGER_OFF) return "unknown flag";
+  const bool data = c->model == LAQ_MODEL_LOGREG_BIN || c->model == LAQ_MODEL_SOFTMAX || c->model == LAQ_MODEL_MLP2;
+  if (data) {
+    if (!c->N) return "N is null";
+    for (int m = 0; m < c->M; ++m)
+      if (c->N[m] < 1 || c->N[m] > (1ll << 31) - 1) return "every N_m must be in 1..2^31-1";
+    if (c->n_features < 1) return "n_features must be positive";
+    if (model_p(*c) != c->p) return "p does not match the model shape";
+    if (!std::isfinite(c->lambda) || c->lambda < 0.f) return "lambda must be finite and >= 0";
+  }
+  if (c->model == LAQ_MODEL_LOGREG_BIN && c->n_features > 256) return "LOGREG_BIN supports n_features <= 256";
+  if (c->model == LAQ_MODEL_SOFTMAX) {
+    if (!softmax_classes_supported(c->n_classes)) return "SOFTMAX supports 2..16 classes";
+    if (c->n_features > 1024) return "SOFTMAX supports n_features <= 1024";
+  }
+  if (c->model == LAQ_MODEL_MLP2) {
+    const char* e = mlp_check_shape(c->n_features, c->n_hidden, c->n_classes);
+    if (e) return e;
+  }
+  if (c->model == LAQ_MODEL_SYNTH) {
+    if (c->p >= (1ll << 32)) return "SYNTH requires p < 2^32";
+    if (!std::isfinite(c->synth_sigma) || !std::isfinite(c->synth_eta0)) return "synth parameters must be finite";
+  }
+  return nullptr;
+}
+
+struct Plan {
+  size_t total = 0;
+  size_t sc, theta, agg, qp, g, codes, Rbits, norms, n_epshat, clock, skip, up_m, up_R, up_s, ring, xi, loss_m,
+      part_q, part_d, part_t, t_skip, t_R, t_ndq, t_neps, t_rhs, t_d2, t_loss, t_up, Xptr, yptr, Ndev, cnt_grad,
+      gpart, lpart, state_end, mlp;
+  std::vector<size_t> X, y;
+  long long ps, nv, cw;
+  int gbpw_cap;
+};
+
+int default_gbpw(const laq_config& c) {
+  int g = (2 * kNumSMs + c.M - 1) / c.M;
+  if (g > kGradBlocksCap) g = kGradBlocksCap;
+  return g < 1 ? 1 : g;
+}
+
+Plan make_plan(const laq_config& c) {
+  Plan pl;
+  const size_t M = (size_t)c.M;
+  pl.ps = (c.p + 15) / 16 * 16;
+  pl.nv = pl.ps / 4;
+  pl.cw = ((pl.ps * c.b + 31) / 32 + 3) / 4 * 4;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes);
+    return o;
+  };
+  const size_t cap = (size_t)c.trace_capacity;
+  const bool data = c.model == LAQ_MODEL_LOGREG_BIN || c.model == LAQ_MODEL_SOFTMAX || c.model == LAQ_MODEL_MLP2;
+  pl.sc = take(sizeof(DevScalars));
+  pl.theta = take(pl.ps * 4);
+  pl.agg = take(pl.ps * 4);
+  pl.qp = take(M * pl.ps * 4);
+  pl.g = (c.model == LAQ_MODEL_SYNTH) ? off : take(M * pl.ps * 4);
+  pl.codes = take(M * pl.cw * 4);
+  pl.Rbits = take(2 * M * 4);
+  pl.norms = take(3 * M * 8);
+  pl.n_epshat = take(M * 8);
+  pl.clock = take(M * 4);
+  pl.skip = take(M);
+  pl.up_m = take(M * 4);
+  pl.up_R = take(M * 4);
+  pl.up_s = take(M * 4);
+  pl.ring = take((size_t)c.D * 8);
+  pl.xi = take((size_t)c.D * 4);
+  pl.loss_m = take(M * 8);
+  pl.part_q = take(M * kMaxSweepBlocksPerWorker * 2 * 8);
+  pl.part_d = take((size_t)kMaxAggBlocks * 8);
+  pl.part_t = take((size_t)kMaxAggBlocks * 8);
+  pl.t_skip = take(cap * M);
+  pl.t_R = take(cap * M * 4);
+  pl.t_ndq = take(cap * M * 8);
+  pl.t_neps = take(cap * M * 8);
+  pl.t_rhs = take(cap * M * 8);
+  pl.t_d2 = take(cap * 8);
+  pl.t_loss = take(cap * 8);
+  pl.t_up = take(cap * 4);
+  pl.Xptr = take(M * 8);
+  pl.yptr = take(M * 8);
+  pl.Ndev = take(M * 8);
+  pl.cnt_grad = take(M * 4);
+  pl.state_end = off;  // everything up to here is zero-filled by laq_init
+  pl.gbpw_cap = 1;
+  pl.gpart = pl.lpart = pl.mlp = off;
+  if (data) {
+    pl.gbpw_cap = kGradBlocksCap;
+    if (c.model != LAQ_MODEL_MLP2) {
+      pl.gpart = take(M * (size_t)pl.gbpw_cap * pl.ps * 4);
+      pl.lpart = take(M * (size_t)pl.gbpw_cap * 8);
+    } else {
+      pl.mlp = take(mlp_scratch_bytes(c));
+    }
+    for (size_t m = 0; m < M; ++m) {
+      pl.X.push_back(take((size_t)c.N[m] * c.n_features * 4));
+      pl.y.push_back(take((size_t)c.N[m] * 4));
+    }
+  }
+  pl.total = off;
+  return pl;
+}
+
+laq_status fail(laq_ctx* ctx, laq_status s, const std::string& msg) {
+  if (ctx) ctx->err = msg;
+  return s;
+}
+
+laq_status cuda_fail(laq_ctx* ctx, cudaError_t e, const char* what) {
+  return fail(ctx, LAQ_ECUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+#define LAQ_CUDA(ctx, call)                                  \
+  do {                                                       \
+    cudaError_t e_ = (call);                                 \
+    if (e_ != cudaSuccess) return cuda_fail(ctx, e_, #call); \
+  } while (0)
+
+bool needs_shards(const laq_ctx* c) {
+  return c->cfg.model == LAQ_MODEL_LOGREG_BIN || c->cfg.model == LAQ_MODEL_SOFTMAX || c->cfg.model == LAQ_MODEL_MLP2;
+}
+
+// Reads the device error word after a synchronisation.
+laq_status check_device_error(laq_ctx* ctx) {
+  uint32_t err = 0;
+  LAQ_CUDA(ctx, cudaMemcpyAsync(&err, &ctx->P.sc->err, 4, cudaMemcpyDeviceToHost, ctx->st));
+  LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));
+  if (err & 1u)
+    return fail(ctx, LAQ_ENONFINITE, "a gradient or radius was not finite; the state is frozen at that iteration");
+  return LAQ_OK;
+}
+
+double host_sum_sq(const float* v, long long n) {
+  double s = 0.0;
+  for (long long i = 0; i < n; ++i) s += (double)v[i] * (double)v[i];
+  return s;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t laq_workspace_bytes(const laq_config* cfg) {
+  if (check_config(cfg)) return 0;
+  return make_plan(*cfg).total;
+}
+
+laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, size_t workspace_bytes,
+                    const float* theta0, void* cuda_stream) {
+  if (!out) return LAQ_EINVAL;
+  *out = nullptr;
+  laq_ctx* ctx = new (std::nothrow) laq_ctx();
+  if (!ctx) return LAQ_EINVAL;
+  *out = ctx;  // returned even on failure so that laq_last_error can be read; free with laq_destroy
+  std::memset(&ctx->P, 0, sizeof(Params));
+  std::memset(&ctx->cfg, 0, sizeof(laq_config));
+  if (const char* e = check_config(cfg)) return fail(ctx, LAQ_EINVAL, e);
+  ctx->cfg = *cfg;
+  ctx->xi.assign(cfg->xi, cfg->xi + cfg->D);
+  ctx->cfg.xi = ctx->xi.data();
+  ctx->N.assign(cfg->M, 0);
+  if (cfg->N && (cfg->model <= LAQ_MODEL_MLP2)) ctx->N.assign(cfg->N, cfg->N + cfg->M);
+  ctx->cfg.N = ctx->N.data();
+  ctx->st = (cudaStream_t)cuda_stream;
+  const Plan pl = make_plan(ctx->cfg);
+  if (!d_workspace) return fail(ctx, LAQ_EWORKSPACE, "workspace is null");
+  if ((uintptr_t)d_workspace % kAlign) return fail(ctx, LAQ_EWORKSPACE, "workspace must be 256-byte aligned");
+  if (workspace_bytes < pl.total) return fail(ctx, LAQ_EWORKSPACE, "workspace is smaller than laq_workspace_bytes(cfg)");
+  cudaPointerAttributes attr;
+  if (cudaPointerGetAttributes(&attr, d_workspace) != cudaSuccess ||
+      (attr.type != cudaMemoryTypeDevice && attr.type != cudaMemoryTypeManaged)) {
+    cudaGetLastError();
+    return fail(ctx, LAQ_EWORKSPACE, "workspace is not device memory");
+  }
+  char* ws = (char*)d_workspace;
+  ctx->ws = ws;
+  ctx->ws_bytes = workspace_bytes;
+  Params& P = ctx->P;
+  const laq_config& c = ctx->cfg;
+  P.M = c.M; P.b = c.b; P.D = c.D; P.tbar = c.tbar; P.clock_mode = c.clock_mode; P.model = c.model;
+  P.flags = c.flags;
+  P.F = c.n_features; P.C = c.n_classes; P.H = c.n_hidden;
+  P.p = c.p; P.ps = pl.ps; P.nv = pl.nv; P.cw = pl.cw;
+  P.alpha = c.alpha; P.lambda = c.lambda;
+  {
+    const double a = (double)c.alpha;
+    P.trig_c = (a * a) * ((double)c.M * (double)c.M);
+  }
+  P.sc = (DevScalars*)(ws + pl.sc);
+  P.theta = (float*)(ws + pl.theta);
+  P.agg = (float*)(ws + pl.agg);
+  P.qp = (float*)(ws + pl.qp);
+  P.g = (c.model == LAQ_MODEL_SYNTH) ? nullptr : (float*)(ws + pl.g);
+  P.codes = (uint32_t*)(ws + pl.codes);
+  P.Rbits = (uint32_t*)(ws + pl.Rbits);
+  P.norms = (double*)(ws + pl.norms);
+  P.n_epshat = (double*)(ws + pl.n_epshat);
+  P.clock = (int32_t*)(ws + pl.clock);
+  P.skip = (uint8_t*)(ws + pl.skip);
+  P.up_m = (int32_t*)(ws + pl.up_m);
+  P.up_R = (float*)(ws + pl.up_R);
+  P.up_s = (float*)(ws + pl.up_s);
+  P.ring = (double*)(ws + pl.ring);
+  P.xi = (float*)(ws + pl.xi);
+  P.loss_m = (double*)(ws + pl.loss_m);
+  P.part_q = (double*)(ws + pl.part_q);
+  P.part_d = (double*)(ws + pl.part_d);
+  P.part_t = (double*)(ws + pl.part_t);
+  P.trace_cap = c.trace_capacity;
+  P.t_skip = (uint8_t*)(ws + pl.t_skip);
+  P.t_R = (float*)(ws + pl.t_R);
+  P.t_ndq = (double*)(ws + pl.t_ndq);
+  P.t_neps = (double*)(ws + pl.t_neps);
+  P.t_rhs = (double*)(ws + pl.t_rhs);
+  P.t_d2 = (double*)(ws + pl.t_d2);
+  P.t_loss = (double*)(ws + pl.t_loss);
+  P.t_up = (int32_t*)(ws + pl.t_up);
+  P.seed_lo = (uint32_t)(c.seed & 0xffffffffull);
+  P.seed_hi = (uint32_t)(c.seed >> 32);
+  P.cz = (float)((double)c.synth_sigma / std::sqrt(21845.0));
+  P.eta0 = c.synth_eta0;
+  P.X = (const float* const*)(ws + pl.Xptr);
+  P.y = (const int32_t* const*)(ws + pl.yptr);
+  P.N = (const long long*)(ws + pl.Ndev);
+  P.cnt_grad = (uint32_t*)(ws + pl.cnt_grad);
+  P.gpart = (float*)(ws + pl.gpart);
+  P.lpart = (double*)(ws + pl.lpart);
+  P.Ntot = 0;
+  for (int m = 0; m < c.M; ++m) P.Ntot += ctx->N[m];
+  ctx->gbpw_cap = pl.gbpw_cap;
+  ctx->gbpw = default_gbpw(c);
+
+  LAQ_CUDA(ctx, cudaMemsetAsync(ws, 0, pl.state_end, ctx->st));
+  if (needs_shards(ctx)) {
+    ctx->shard_loaded.assign(c.M, 0);
+    ctx->Xptr.resize(c.M);
+    ctx->yptr.resize(c.M);
+    for (int m = 0; m < c.M; ++m) {
+      ctx->Xptr[m] = (const float*)(ws + pl.X[m]);
+      ctx->yptr[m] = (const int32_t*)(ws + pl.y[m]);
+    }
+    LAQ_CUDA(ctx, cudaMemcpyAsync(ws + pl.Xptr, ctx->Xptr.data(), 8 * (size_t)c.M, cudaMemcpyHostToDevice, ctx->st));
+    LAQ_CUDA(ctx, cudaMemcpyAsync(ws + pl.yptr, ctx->yptr.data(), 8 * (size_t)c.M, cudaMemcpyHostToDevice, ctx->st));
+    LAQ_CUDA(ctx, cudaMemcpyAsync(ws + pl.Ndev, ctx->N.data(), 8 * (size_t)c.M, cudaMemcpyHostToDevice, ctx->st));
+    if (c.model == LAQ_MODEL_MLP2) {
+      laq_status s = mlp_setup(ctx->mlp, P, ws + pl.mlp, ctx->st);
+      if (s != LAQ_OK) return fail(ctx, s, "network scratch set-up failed");
+    }
+  }
+  std::vector<int32_t> clocks(c.M, c.tbar + 1);  // every worker uploads at k = 1
+  LAQ_CUDA(ctx, cudaMemcpyAsync(P.clock, clocks.data(), 4 * (size_t)c.M, cudaMemcpyHostToDevice, ctx->st));
+  LAQ_CUDA(ctx, cudaMemcpyAsync(P.xi, ctx->xi.data(), 4 * (size_t)c.D, cudaMemcpyHostToDevice, ctx->st));
+  if (theta0) {
+    LAQ_CUDA(ctx, cudaMemcpyAsync(P.theta, theta0, 4 * (size_t)c.p, cudaMemcpyHostToDevice, ctx->st));
+    const double tsq = host_sum_sq(theta0, c.p);
+    LAQ_CUDA(ctx, cudaMemcpyAsync(&P.sc->theta_sq, &tsq, 8, cudaMemcpyHostToDevice, ctx->st));
+  }
+  LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));  // the host vectors above go out of scope
+  return LAQ_OK;
+}
+
+laq_status laq_load_shards(laq_ctx* ctx, int32_t m, const float* X, const int32_t* y, int64_t N_m,
+                           int32_t on_device) {
+  if (!ctx || !ctx->ws) return LAQ_EINVAL;
+  if (!needs_shards(ctx)) return fail(ctx, LAQ_ESTATE, "this model holds no data shards");
+  if (m < 0 || m >= ctx->cfg.M) return fail(ctx, LAQ_EINVAL, "worker index out of range");
+  if (!X || !y) return fail(ctx, LAQ_EINVAL, "X or y is null");
+  if (N_m != ctx->N[m]) return fail(ctx, LAQ_EINVAL, "N_m differs from the configured value");
+  const cudaMemcpyKind kind = on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+  LAQ_CUDA(ctx, cudaMemcpyAsync((void*)ctx->Xptr[m], X, (size_t)N_m * ctx->cfg.n_features * 4, kind, ctx->st));
+  LAQ_CUDA(ctx, cudaMemcpyAsync((void*)ctx->yptr[m], y, (size_t)N_m * 4, kind, ctx->st));
+  if (ctx->cfg.model == LAQ_MODEL_MLP2) {
+    ctx->launches += mlp_convert_shard(ctx->mlp, ctx->P, m, ctx->Xptr[m], N_m, ctx->st);
+  }
+  LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));  // the caller may reuse its buffers on return
+  ctx->shard_loaded[m] = 1;
+  return LAQ_OK;
+}
+
+laq_status laq_set_gradients(laq_ctx* ctx, const float* g, int32_t on_device) {
+  if (!ctx || !ctx->ws) return LAQ_EINVAL;
+  if (ctx->cfg.model != LAQ_MODEL_EXTERNAL) return fail(ctx, LAQ_ESTATE, "model is not LAQ_MODEL_EXTERNAL");
+  if (!g) return fail(ctx, LAQ_EINVAL, "g is null");
+  const cudaMemcpyKind kind = on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+  const Params& P = ctx->P;
+  LAQ_CUDA(ctx, cudaMemcpy2DAsync(P.g, (size_t)P.ps * 4, g, (size_t)P.p * 4, (size_t)P.p * 4, (size_t)P.M, kind,
+                                  ctx->st));
+  if (!on_device) LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));
+  ctx->ext_g_set = true;
+  return LAQ_OK;
+}
+
+laq_status laq_step(laq_ctx* ctx, int32_t n_iters, const laq_trace* trace) {
+  if (!ctx || !ctx->ws) return LAQ_EINVAL;
+  if (n_iters < 0) return fail(ctx, LAQ_EINVAL, "n_iters must be >= 0");
+  const laq_config& c = ctx->cfg;
+  const Params& P = ctx->P;
+  if (needs_shards(ctx))
+    for (int m = 0; m < c.M; ++m)
+      if (!ctx->shard_loaded[m]) return fail(ctx, LAQ_ESTATE, "laq_load_shards has not been called for every worker");
+  if (c.model == LAQ_MODEL_EXTERNAL) {
+    if (n_iters > 1) return fail(ctx, LAQ_EINVAL, "LAQ_MODEL_EXTERNAL steps one iteration per call");
+    if (n_iters == 1 && !ctx->ext_g_set) return fail(ctx, LAQ_ESTATE, "laq_set_gradients has not been called");
+  }
+  if (trace && n_iters > c.trace_capacity) return fail(ctx, LAQ_EINVAL, "n_iters exceeds trace_capacity");
+  LAQ_CUDA(ctx, cudaMemsetAsync(&P.sc->trace_pos, trace ? 0 : 0xff, 4, ctx->st));  // 0xffffffff = tracing off
+  for (int it = 0; it < n_iters; ++it) {
+    cudaEvent_t* ev = nullptr;
+    if (ctx->profiling && ctx->ev_used < kProfIters) {
+      ev = &ctx->ev[(size_t)ctx->ev_used * 5];
+      ctx->ev_used += 1;
+      cudaEventRecord(ev[0], ctx->st);
+    }
+    const int64_t l0 = ctx->launches;
+    switch (c.model) {
+      case LAQ_MODEL_LOGREG_BIN:
+        ctx->launches += launch_grad_logreg(P, ctx->ls, ctx->gbpw, ctx->st);
+        ctx->launches += launch_grad_finalize(P, ctx->gbpw, &P.sc->theta_sq, ctx->st);
+        break;
+      case LAQ_MODEL_SOFTMAX:
+        ctx->launches += launch_grad_softmax(P, ctx->ls, ctx->gbpw, ctx->st);
+        ctx->launches += launch_grad_finalize(P, ctx->gbpw, &P.sc->theta_sq, ctx->st);
+        break;
+      case LAQ_MODEL_MLP2:
+        ctx->launches += mlp_launch_gradients(ctx->mlp, P, ctx->st);
+        break;
+      default: break;
+    }
+    if (ev) {
+      cudaEventRecord(ev[1], ctx->st);
+      ctx->stage_launches[0] += ctx->launches - l0;
+    }
+    ctx->launches += launch_radius(P, ctx->ls, ctx->st);
+    if (ev) cudaEventRecord(ev[2], ctx->st);
+    ctx->launches += launch_quantize_trigger(P, ctx->ls, ctx->st);
+    if (ev) cudaEventRecord(ev[3], ctx->st);
+    ctx->launches += launch_aggregate(P, ctx->ls, ctx->st);
+    if (ev) {
+      cudaEventRecord(ev[4], ctx->st);
+      for (int s = 1; s < 4; ++s) ctx->stage_launches[s] += 1;
+    }
+  }
+  LAQ_CUDA(ctx, cudaGetLastError());
+  if (c.model == LAQ_MODEL_EXTERNAL && n_iters == 1) ctx->ext_g_set = false;
+  if (!trace) return LAQ_OK;
+  const size_t n = (size_t)n_iters, M = (size_t)c.M;
+  auto pull = [&](void* dst, const void* src, size_t bytes) -> cudaError_t {
+    if (!dst || !bytes) return cudaSuccess;
+    return cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, ctx->st);
+  };
+  LAQ_CUDA(ctx, pull(trace->skip, P.t_skip, n * M));
+  LAQ_CUDA(ctx, pull(trace->R, P.t_R, n * M * 4));
+  LAQ_CUDA(ctx, pull(trace->n_dq, P.t_ndq, n * M * 8));
+  LAQ_CUDA(ctx, pull(trace->n_eps, P.t_neps, n * M * 8));
+  LAQ_CUDA(ctx, pull(trace->rhs, P.t_rhs, n * M * 8));
+  LAQ_CUDA(ctx, pull(trace->dtheta2, P.t_d2, n * 8));
+  LAQ_CUDA(ctx, pull(trace->loss, P.t_loss, n * 8));
+  LAQ_CUDA(ctx, pull(trace->uploads, P.t_up, n * 4));
+  return check_device_error(ctx);
+}
+
+laq_status laq_sync(laq_ctx* ctx) {
+  if (!ctx || !ctx->ws) return LAQ_EINVAL;
+  return check_device_error(ctx);
+}
+
+laq_status laq_get_state(laq_ctx* ctx, const laq_state* out) {
+  if (!ctx || !ctx->ws) return LAQ_EINVAL;
+  if (!out) return fail(ctx, LAQ_EINVAL, "state is null");
+  const Params& P = ctx->P;
+  const size_t M = (size_t)P.M, p = (size_t)P.p;
+  DevScalars sc;
+  LAQ_CUDA(ctx, cudaMemcpyAsync(&sc, P.sc, sizeof(sc), cudaMemcpyDeviceToHost, ctx->st));
+  LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));
+  auto pull = [&](void* dst, const void* src, size_t bytes) -> cudaError_t {
+    if (!dst || !bytes) return cudaSuccess;
+    return cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, ctx->st);
+  };
+  auto pull2d = [&](void* dst, size_t dpitch, const void* src, size_t spitch, size_t width, size_t rows) -> cudaError_t {
+    if (!dst) return cudaSuccess;
+    return cudaMemcpy2DAsync(dst, dpitch, src, spitch, width, rows, cudaMemcpyDeviceToHost, ctx->st);
+  };
+  LAQ_CUDA(ctx, pull(out->theta, P.theta, p * 4));
+  LAQ_CUDA(ctx, pull(out->agg, P.agg, p * 4));
+  LAQ_CUDA(ctx, pull2d(out->qprev, p * 4, P.qp, (size_t)P.ps * 4, p * 4, M));
+  if (out->g) {
+    if (!P.g) return fail(ctx, LAQ_EINVAL, "g is not stored for LAQ_MODEL_SYNTH");
+    LAQ_CUDA(ctx, pull2d(out->g, p * 4, P.g, (size_t)P.ps * 4, p * 4, M));
+  }
+  const size_t W = (p * (size_t)P.b + 31) / 32;
+  LAQ_CUDA(ctx, pull2d(out->codes, W * 4, P.codes, (size_t)P.cw * 4, W * 4, M));
+  LAQ_CUDA(ctx, pull(out->n_eps_hat, P.n_epshat, M * 8));
+  LAQ_CUDA(ctx, pull(out->clock, P.clock, M * 4));
+  LAQ_CUDA(ctx, pull(out->skip, P.skip, M));
+  std::vector<double> ring(P.D), norms(3 * M);
+  std::vector<uint32_t> Rb(2 * M);
+  LAQ_CUDA(ctx, pull(ring.data(), P.ring, (size_t)P.D * 8));
+  LAQ_CUDA(ctx, pull(norms.data(), P.norms, 3 * M * 8));
+  LAQ_CUDA(ctx, pull(Rb.data(), P.Rbits, 2 * M * 4));
+  LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));
+  if (out->ring)
+    for (int d = 0; d < P.D; ++d) out->ring[d] = ring[(sc.ring_head + d) % P.D];
+  for (size_t m = 0; m < M; ++m) {
+    if (out->n_dq) out->n_dq[m] = norms[3 * m];
+    if (out->n_eps) out->n_eps[m] = norms[3 * m + 1];
+    if (out->R) {
+      const uint32_t bits = sc.k ? Rb[((sc.k - 1) & 1ull) * M + m] : 0u;
+      std::memcpy(&out->R[m], &bits, 4);
+    }
+  }
+  if (out->counters) {
+    out->counters[0] = (int64_t)sc.k;
+    out->counters[1] = (int64_t)sc.uploads;
+    out->counters[2] = (int64_t)sc.bits;
+  }
+  if (sc.err & 1u)
+    return fail(ctx, LAQ_ENONFINITE, "a gradient or radius was not finite; the state is frozen at that iteration");
+  return LAQ_OK;
+}
+
+laq_status laq_get_worker(laq_ctx* ctx, int32_t m, float* qprev, float* g, uint32_t* codes, float* R) {
+  if (!ctx || !ctx->ws) return LAQ_EINVAL;
+  const Params& P = ctx->P;
+  if (m < 0 || m >= P.M) return fail(ctx, LAQ_EINVAL, "worker index out of range");
+  if (g && !P.g) return fail(ctx, LAQ_EINVAL, "g is not stored for LAQ_MODEL_SYNTH");
+  const size_t p = (size_t)P.p, W = (p * (size_t)P.b + 31) / 32;
+  DevScalars sc;
+  LAQ_CUDA(ctx, cudaMemcpyAsync(&sc, P.sc, sizeof(sc), cudaMemcpyDeviceToHost, ctx->st));
+  LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));
+  if (qprev) LAQ_CUDA(ctx, cudaMemcpyAsync(qprev, P.qp + (size_t)m * P.ps, p * 4, cudaMemcpyDeviceToHost, ctx->st));
+  if (g) LAQ_CUDA(ctx, cudaMemcpyAsync(g, P.g + (size_t)m * P.ps, p * 4, cudaMemcpyDeviceToHost, ctx->st));
+  if (codes) LAQ_CUDA(ctx, cudaMemcpyAsync(codes, P.codes + (size_t)m * P.cw, W * 4, cudaMemcpyDeviceToHost, ctx->st));
+  if (R) {
+    *R = 0.f;
+    if (sc.k)
+      LAQ_CUDA(ctx, cudaMemcpyAsync(R, P.Rbits + ((sc.k - 1) & 1ull) * P.M + m, 4, cudaMemcpyDeviceToHost, ctx->st));
+  }
+  LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));
+  return LAQ_OK;
+}
+
+laq_status laq_set_state(laq_ctx* ctx, const laq_state* in) {
+  if (!ctx || !ctx->ws) return LAQ_EINVAL;
+  if (!in) return fail(ctx, LAQ_EINVAL, "state is null");
+  const Params& P = ctx->P;
+  const size_t M = (size_t)P.M, p = (size_t)P.p;
+  DevScalars sc;
+  LAQ_CUDA(ctx, cudaMemcpyAsync(&sc, P.sc, sizeof(sc), cudaMemcpyDeviceToHost, ctx->st));
+  LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));
+  auto push = [&](void* dst, const void* src, size_t bytes) -> cudaError_t {
+    if (!src || !bytes) return cudaSuccess;
+    return cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, ctx->st);
+  };
+  LAQ_CUDA(ctx, push(P.theta, in->theta, p * 4));
+  if (in->theta) sc.theta_sq = host_sum_sq(in->theta, (long long)p);
+  LAQ_CUDA(ctx, push(P.agg, in->agg, p * 4));
+  if (in->qprev)
+    LAQ_CUDA(ctx, cudaMemcpy2DAsync(P.qp, (size_t)P.ps * 4, in->qprev, p * 4, p * 4, M, cudaMemcpyHostToDevice, ctx->st));
+  LAQ_CUDA(ctx, push(P.n_epshat, in->n_eps_hat, M * 8));
+  LAQ_CUDA(ctx, push(P.clock, in->clock, M * 4));
+  if (in->ring) {
+    LAQ_CUDA(ctx, push(P.ring, in->ring, (size_t)P.D * 8));
+    sc.ring_head = 0;
+  }
+  if (in->counters) {
+    if (in->counters[0] < 0 || in->counters[1] < 0 || in->counters[2] < 0) return fail(ctx, LAQ_EINVAL, "negative counter");
+    sc.k = (unsigned long long)in->counters[0];
+    sc.uploads = (unsigned long long)in->counters[1];
+    sc.bits = (unsigned long long)in->counters[2];
+  }
+  sc.err = 0;
+  sc.cnt_quant = sc.cnt_agg = 0;
+  LAQ_CUDA(ctx, cudaMemsetAsync(P.Rbits, 0, 2 * M * 4, ctx->st));
+  LAQ_CUDA(ctx, cudaMemcpyAsync(P.sc, &sc, sizeof(sc), cudaMemcpyHostToDevice, ctx->st));
+  LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));
+  return LAQ_OK;
+}
+
+int64_t laq_kernel_launches(const laq_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+laq_status laq_tune(laq_ctx* ctx, const char* key, int32_t value) {
+  if (!ctx || !ctx->ws || !key) return LAQ_EINVAL;
+  const std::string k(key);
+  auto pow2_threads = [](int v) { return v == 64 || v == 128 || v == 256 || v == 512; };
+  if (k == "sweep_threads" && pow2_threads(value)) ctx->ls.sweep_threads = value;
+  else if (k == "sweep_blocks_per_sm" && value >= 1 && value <= 32) ctx->ls.sweep_blocks_per_sm = value;
+  else if (k == "agg_threads" && pow2_threads(value)) ctx->ls.agg_threads = value;
+  else if (k == "agg_blocks_per_sm" && value >= 1 && value <= 32) ctx->ls.agg_blocks_per_sm = value;
+  else if (k == "grad_blocks_per_worker" && value >= 1 && value <= ctx->gbpw_cap) ctx->gbpw = value;
+  else return fail(ctx, LAQ_EINVAL, "unknown tuning key or value outside its limits");
+  return LAQ_OK;
+}
+
+laq_status laq_set_profiling(laq_ctx* ctx, int32_t enabled) {
+  if (!ctx || !ctx->ws) return LAQ_EINVAL;
+  if (enabled && ctx->ev.empty()) {
+    ctx->ev.resize((size_t)kProfIters * 5);
+    for (auto& e : ctx->ev) LAQ_CUDA(ctx, cudaEventCreate(&e));
+  }
+  ctx->profiling = enabled != 0;
+  return LAQ_OK;
+}
+
+laq_status laq_kernel_times(laq_ctx* ctx, double* ms, int64_t* launches) {
+  if (!ctx || !ctx->ws) return LAQ_EINVAL;
+  LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));
+  for (int i = 0; i < ctx->ev_used; ++i) {
+    cudaEvent_t* ev = &ctx->ev[(size_t)i * 5];
+    for (int s = 0; s < 4; ++s) {
+      float t = 0.f;
+      LAQ_CUDA(ctx, cudaEventElapsedTime(&t, ev[s], ev[s + 1]));
+      ctx->stage_ms[s] += (double)t;
+    }
+  }
+  ctx->ev_used = 0;
+  for (int s = 0; s < 4; ++s) {
+    if (ms) ms[s] = ctx->stage_ms[s];
+    if (launches) launches[s] = ctx->stage_launches[s];
+    ctx->stage_ms[s] = 0.0;
+    ctx->stage_launches[s] = 0;
+  }
+  return LAQ_OK;
+}
+
+const char* laq_last_error(const laq_ctx* ctx) { return ctx ? ctx->err.c_str() : "context is null"; }
+
+void laq_destroy(laq_ctx* ctx) {
+  if (!ctx) return;
+  if (ctx->ws) cudaStreamSynchronize(ctx->st);
+  mlp_teardown(ctx->mlp);
+  for (auto& e : ctx->ev) cudaEventDestroy(e);
+  delete ctx;
+}
+
+}  // extern "C"

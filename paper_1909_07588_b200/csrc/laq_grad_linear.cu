@@ -1,0 +1,280 @@
+// Step 1 of the LAQ iteration for the two linear models of the paper's supplement
+// ("Simulation details"): worker m's gradient of f_m at theta^k over its resident shard,
+//   g_m = (1/N) sum_n grad CE(x_{m,n}; theta) + (N_m/N) lambda theta,
+// as a skinny contraction that reads every sample once: a block stages a tile of consecutive rows
+// (contiguous in memory) in shared memory, computes the residuals (sigma(z) - y, or softmax - onehot)
+// and accumulates residual^T x in registers across its tiles.  Block partials are combined in a
+// fixed order by grad_finalize_kernel, which also adds the regulariser share.
+#include "laq_internal.cuh"
+
+namespace laq {
+
+namespace {
+
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_sum_f(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Copy `count` consecutive floats global -> shared with 16-byte loads where alignment allows.
+__device__ __forceinline__ void stage_rows(const float* __restrict__ src, float* dst, int count) {
+  if ((reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
+    const int n4 = count >> 2;
+    const float4* s4 = reinterpret_cast<const float4*>(src);
+    float4* d4 = reinterpret_cast<float4*>(dst);
+    for (int i = threadIdx.x; i < n4; i += blockDim.x) d4[i] = __ldg(s4 + i);
+    for (int i = (n4 << 2) + threadIdx.x; i < count; i += blockDim.x) dst[i] = __ldg(src + i);
+  } else {
+    for (int i = threadIdx.x; i < count; i += blockDim.x) dst[i] = __ldg(src + i);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// binary logistic regression, F <= 256
+// ------------------------------------------------------------------------------------------------
+constexpr int kLrThreads = 256;
+constexpr int kLrMaxRows = 256;   // rows per tile: at most one per thread, fewer for wide rows
+
+__global__ void __launch_bounds__(kLrThreads) grad_logreg_kernel(const Params P, int gbpw, int rows) {
+  extern __shared__ __align__(16) float smem[];
+  const int F = P.F, m = blockIdx.y, t = threadIdx.x;
+  float* xs = smem;                          // [rows][F]
+  float* ths = xs + rows * F;                // [F]
+  float* rs = ths + ((F + 3) & ~3);          // [rows]
+  float* red = rs + kLrMaxRows;              // [kLrThreads]
+  __shared__ double shd[32];
+  const float* __restrict__ X = P.X[m];
+  const int32_t* __restrict__ y = P.y[m];
+  const long long n = P.N[m];
+  for (int f = t; f < F; f += blockDim.x) ths[f] = P.theta[f];
+  const int S = kLrThreads / F;              // row slices handled in parallel in the second phase
+  const bool active = t < S * F;
+  const int f_own = t % F, slice = t / F;
+  float acc = 0.f;
+  double loss = 0.0;
+  const long long ntiles = (n + rows - 1) / rows;
+  for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    const long long r0 = tile * rows;
+    const int nr = (int)((n - r0 < rows) ? (n - r0) : rows);
+    __syncthreads();
+    stage_rows(X + r0 * F, xs, nr * F);
+    __syncthreads();
+    if (t < nr) {
+      const float* xr = xs + t * F;
+      float z = 0.f;
+      for (int f = 0; f < F; ++f) z = fmaf(xr[f], ths[f], z);
+      const float yv = (float)y[r0 + t];
+      float sig, sp;
+      if (z >= 0.f) {
+        const float e = expf(-z);
+        sig = 1.0f / (1.0f + e);
+        sp = z + log1pf(e);
+      } else {
+        const float e = expf(z);
+        sig = e / (1.0f + e);
+        sp = log1pf(e);
+      }
+      rs[t] = sig - yv;
+      loss += (double)(sp - yv * z);
+    }
+    __syncthreads();
+    if (active)
+      for (int r = slice; r < nr; r += S) acc = fmaf(rs[r], xs[r * F + f_own], acc);  // address = (r-slice) F + t
+  }
+  __syncthreads();
+  red[t] = active ? acc : 0.f;
+  __syncthreads();
+  if (t < F) {
+    float s = 0.f;
+    for (int sl = 0; sl < S; ++sl) s += red[sl * F + t];
+    P.gpart[((long long)m * gbpw + blockIdx.x) * P.ps + t] = s;
+  }
+  loss = warp_sum_d(loss);
+  if ((t & 31) == 0) shd[t >> 5] = loss;
+  __syncthreads();
+  if (t == 0) {
+    double l = 0.0;
+    for (int i = 0; i < kLrThreads / 32; ++i) l += shd[i];
+    P.lpart[(long long)m * gbpw + blockIdx.x] = l;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// C-class softmax regression, F <= 1024
+// ------------------------------------------------------------------------------------------------
+constexpr int kSmThreads = 256;
+constexpr int kSmRows = 16;
+constexpr int kSmMaxJ = 4;  // features per thread: F <= kSmMaxJ * kSmThreads
+
+template <int C>
+__global__ void __launch_bounds__(kSmThreads) grad_softmax_kernel(const Params P, int gbpw) {
+  extern __shared__ __align__(16) float smem[];
+  const int F = P.F, m = blockIdx.y, t = threadIdx.x, lane = t & 31, w = t >> 5;
+  float* xs = smem;                 // [kSmRows][F]
+  float* res = xs + kSmRows * F;    // [kSmRows][C]
+  __shared__ double shd[32];
+  const float* __restrict__ X = P.X[m];
+  const int32_t* __restrict__ y = P.y[m];
+  const float* __restrict__ theta = P.theta;
+  const long long n = P.N[m];
+  float acc[kSmMaxJ][C];
+#pragma unroll
+  for (int j = 0; j < kSmMaxJ; ++j)
+#pragma unroll
+    for (int c = 0; c < C; ++c) acc[j][c] = 0.f;
+  double loss = 0.0;
+  const long long ntiles = (n + kSmRows - 1) / kSmRows;
+  for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    const long long r0 = tile * kSmRows;
+    const int nr = (int)((n - r0 < kSmRows) ? (n - r0) : kSmRows);
+    __syncthreads();
+    stage_rows(X + r0 * F, xs, nr * F);
+    __syncthreads();
+    // phase 1: a warp per row computes the C scores, the softmax and the residual
+    for (int r = w; r < nr; r += kSmThreads / 32) {
+      float z[C];
+#pragma unroll
+      for (int c = 0; c < C; ++c) z[c] = 0.f;
+      const float* xr = xs + r * F;
+      for (int f = lane; f < F; f += 32) {
+        const float x = xr[f];
+#pragma unroll
+        for (int c = 0; c < C; ++c) z[c] = fmaf(x, __ldg(theta + c * F + f), z[c]);
+      }
+#pragma unroll
+      for (int c = 0; c < C; ++c) z[c] = warp_sum_f(z[c]);
+      float zmax = z[0];
+#pragma unroll
+      for (int c = 1; c < C; ++c) zmax = fmaxf(zmax, z[c]);
+      float e[C], sum = 0.f;
+#pragma unroll
+      for (int c = 0; c < C; ++c) {
+        e[c] = expf(z[c] - zmax);
+        sum += e[c];
+      }
+      const int yv = y[r0 + r];
+      const float inv = 1.0f / sum;
+      float zy = 0.f;
+#pragma unroll
+      for (int c = 0; c < C; ++c) {
+        if (c == yv) zy = z[c];
+        if (lane == 0) res[r * C + c] = e[c] * inv - (c == yv ? 1.f : 0.f);
+      }
+      if (lane == 0) loss += (double)((zmax + logf(sum)) - zy);
+    }
+    __syncthreads();
+    // phase 2: thread t owns features t, t + 256, ...; residuals are broadcast from shared memory
+    for (int r = 0; r < nr; ++r) {
+      float rr[C];
+#pragma unroll
+      for (int c = 0; c < C; ++c) rr[c] = res[r * C + c];
+#pragma unroll
+      for (int j = 0; j < kSmMaxJ; ++j) {
+        const int f = t + j * kSmThreads;
+        if (f < F) {
+          const float x = xs[r * F + f];
+#pragma unroll
+          for (int c = 0; c < C; ++c) acc[j][c] = fmaf(rr[c], x, acc[j][c]);
+        }
+      }
+    }
+  }
+  float* gp = P.gpart + ((long long)m * gbpw + blockIdx.x) * P.ps;
+#pragma unroll
+  for (int j = 0; j < kSmMaxJ; ++j) {
+    const int f = t + j * kSmThreads;
+    if (f < F) {
+#pragma unroll
+      for (int c = 0; c < C; ++c) gp[c * F + f] = acc[j][c];
+    }
+  }
+  loss = warp_sum_d(loss);
+  __syncthreads();
+  if (lane == 0) shd[w] = loss;
+  __syncthreads();
+  if (t == 0) {
+    double l = 0.0;
+    for (int i = 0; i < kSmThreads / 32; ++i) l += shd[i];
+    P.lpart[(long long)m * gbpw + blockIdx.x] = l;
+  }
+}
+
+}  // namespace
+
+// Combine the block partials of worker blockIdx.y in block order, scale by 1/N and add the
+// worker's share (N_m/N) lambda theta of the regulariser; block 0 of each worker also writes the
+// worker's loss term.  theta_sq = ||theta^k||^2 comes from the previous theta step.
+__global__ void __launch_bounds__(256) grad_finalize_kernel(const Params P, int gbpw, const double* theta_sq) {
+  const int m = blockIdx.y;
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const double inv_N = 1.0 / (double)P.Ntot;
+  const double share = (double)P.N[m] / (double)P.Ntot;
+  if (i < P.p) {
+    const float* gp = P.gpart + (long long)m * gbpw * P.ps + i;
+    double s = 0.0;
+    for (int blk = 0; blk < gbpw; ++blk) s += (double)gp[(long long)blk * P.ps];
+    const double g = s * inv_N + share * (double)P.lambda * (double)P.theta[i];
+    P.g[(long long)m * P.ps + i] = (float)g;
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    double l = 0.0;
+    for (int blk = 0; blk < gbpw; ++blk) l += P.lpart[(long long)m * gbpw + blk];
+    P.loss_m[m] = l * inv_N + share * 0.5 * (double)P.lambda * (*theta_sq);
+  }
+}
+
+bool softmax_classes_supported(int C) { return C >= 2 && C <= 16; }
+
+// rows per tile: a multiple of 4 (so every tile starts 16-byte aligned), at most 160 KB of samples
+static int logreg_rows(int F) {
+  int r = (40960 / F) & ~3;
+  return r > kLrMaxRows ? kLrMaxRows : r;
+}
+static size_t logreg_smem(int F) {
+  return sizeof(float) * ((size_t)logreg_rows(F) * F + ((F + 3) & ~3) + kLrMaxRows + kLrThreads);
+}
+static size_t softmax_smem(int F, int C) { return sizeof(float) * ((size_t)kSmRows * F + (size_t)kSmRows * C); }
+
+int launch_grad_logreg(const Params& P, const LaunchShape&, int gbpw, cudaStream_t st) {
+  const size_t sm = logreg_smem(P.F);
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaFuncSetAttribute(grad_logreg_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    attr_done = true;
+  }
+  grad_logreg_kernel<<<dim3(gbpw, P.M), kLrThreads, sm, st>>>(P, gbpw, logreg_rows(P.F));
+  return 1;
+}
+
+template <int C>
+static void launch_sm(const Params& P, int gbpw, cudaStream_t st) {
+  const size_t sm = softmax_smem(P.F, C);
+  cudaFuncSetAttribute(grad_softmax_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  grad_softmax_kernel<C><<<dim3(gbpw, P.M), kSmThreads, sm, st>>>(P, gbpw);
+}
+
+int launch_grad_softmax(const Params& P, const LaunchShape&, int gbpw, cudaStream_t st) {
+  switch (P.C) {
+#define LAQ_SM_CASE(c) case c: launch_sm<c>(P, gbpw, st); break;
+    LAQ_SM_CASE(2) LAQ_SM_CASE(3) LAQ_SM_CASE(4) LAQ_SM_CASE(5) LAQ_SM_CASE(6) LAQ_SM_CASE(7) LAQ_SM_CASE(8)
+    LAQ_SM_CASE(9) LAQ_SM_CASE(10) LAQ_SM_CASE(11) LAQ_SM_CASE(12) LAQ_SM_CASE(13) LAQ_SM_CASE(14)
+    LAQ_SM_CASE(15) LAQ_SM_CASE(16)
+#undef LAQ_SM_CASE
+    default: return 0;
+  }
+  return 1;
+}
+
+int launch_grad_finalize(const Params& P, int gbpw, const double* theta_sq, cudaStream_t st) {
+  dim3 grid((unsigned)((P.p + 255) / 256), P.M);
+  grad_finalize_kernel<<<grid, 256, 0, st>>>(P, gbpw, theta_sq);
+  return 1;
+}
+
+}  // namespace laq

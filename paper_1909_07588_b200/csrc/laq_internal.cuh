@@ -1,0 +1,112 @@
+// Internal declarations shared by the library's translation units (not part of the public ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "laq.h"
+
+namespace laq {
+
+constexpr int kMaxWorkers = 1024;   // M limit: the trigger stage runs in one block
+constexpr int kMaxD = 64;           // D limit
+constexpr int kMaxSweepBlocksPerWorker = 256;
+constexpr int kNumSMs = 148;        // B200
+
+// Scalars that live on the device so that an iteration needs no host round trip.
+struct DevScalars {
+  uint32_t err;         // 0 = ok; bit 0 = non-finite gradient/radius (state frozen)
+  uint32_t ring_head;   // slot of the newest stored squared parameter difference
+  uint32_t trace_pos;   // next trace row
+  uint32_t n_up;        // |M^k| of the iteration in flight
+  uint32_t cnt_quant;   // "last block done" tickets
+  uint32_t cnt_agg;
+  uint32_t pad0, pad1;
+  unsigned long long k;        // iterations done
+  unsigned long long uploads;  // sum_k |M^k|
+  unsigned long long bits;     // uploads x (32 + b p)
+  double theta_sq;             // ||theta^k||^2 (for the regulariser term of the reported loss)
+};
+
+// Everything a kernel needs, passed by value.
+struct Params {
+  int M, b, D, tbar, clock_mode, model;
+  uint32_t flags;
+  int F, C, H;               // model shape
+  long long p, ps, nv, cw;   // coordinates, padded row stride (floats), ps/4, code words per row
+  float alpha, lambda;
+  double trig_c;             // alpha^2 M^2 (fp64)
+  // state
+  float* theta;
+  float* agg;
+  float* qp;        // [M][ps]
+  float* g;         // [M][ps]   (null for SYNTH)
+  uint32_t* codes;  // [M][cw]
+  uint32_t* Rbits;  // [2][M]   radius as float bits, double-buffered by iteration parity
+  double* norms;    // [M][3]   n_dq, n_eps, rhs of the last iteration
+  double* n_epshat; // [M]
+  int32_t* clock;   // [M]
+  uint8_t* skip;    // [M]
+  int32_t* up_m;    // [M] uploaders in ascending order
+  float* up_R;      // [M] their radii
+  float* up_s;      // [M] their grid steps 2 tau R
+  double* ring;     // [D] circular
+  float* xi;        // [D]
+  double* loss_m;   // [M]
+  DevScalars* sc;
+  // scratch for the fixed-order two-stage reductions
+  double* part_q;   // [M][kMaxSweepBlocksPerWorker][2]
+  double* part_d;   // [agg blocks]  partial ||alpha grad||^2
+  double* part_t;   // [agg blocks]  partial ||theta^{k+1}||^2
+  // trace (rows = iterations of the current laq_step call)
+  int trace_cap;
+  uint8_t* t_skip;
+  float* t_R;
+  double *t_ndq, *t_neps, *t_rhs, *t_d2, *t_loss;
+  int32_t* t_up;
+  // synthetic gradient stream
+  uint32_t seed_lo, seed_hi;
+  float cz, eta0;
+  // shards
+  long long Ntot;
+  const float* const* X;     // device array of M device pointers
+  const int32_t* const* y;   // device array of M device pointers
+  const long long* N;        // device [M]
+  // model scratch
+  float* gpart;              // gradient partials [M][gbpw][ps]
+  double* lpart;             // loss partials [M][gbpw]
+  uint32_t* cnt_grad;        // [M] tickets
+};
+
+struct LaunchShape {
+  int sweep_threads = 256;
+  int sweep_blocks_per_sm = 8;
+  int agg_threads = 256;
+  int agg_blocks_per_sm = 8;
+  int grad_blocks_per_worker = 0;  // 0 = automatic
+};
+
+// kernels' host-side launchers (each returns the number of kernels it launched)
+int launch_radius(const Params& P, const LaunchShape& ls, cudaStream_t st);
+int launch_quantize_trigger(const Params& P, const LaunchShape& ls, cudaStream_t st);
+int launch_aggregate(const Params& P, const LaunchShape& ls, cudaStream_t st);
+int launch_grad_logreg(const Params& P, const LaunchShape& ls, int gbpw, cudaStream_t st);
+int launch_grad_softmax(const Params& P, const LaunchShape& ls, int gbpw, cudaStream_t st);
+int launch_grad_finalize(const Params& P, int gbpw, const double* theta_sq, cudaStream_t st);
+bool softmax_classes_supported(int C);
+
+// one-hidden-layer ReLU network (laq_grad_mlp.cu)
+struct MlpPlan {
+  void* scratch = nullptr;
+  int ready = 0;
+};
+const char* mlp_check_shape(int F, int H, int C);   // null if supported, else the reason
+size_t mlp_scratch_bytes(const laq_config& c);
+laq_status mlp_setup(MlpPlan& mp, const Params& P, void* scratch, cudaStream_t st);
+int mlp_convert_shard(MlpPlan& mp, const Params& P, int m, const float* X, long long n, cudaStream_t st);
+int mlp_launch_gradients(MlpPlan& mp, const Params& P, cudaStream_t st);
+void mlp_teardown(MlpPlan& mp);
+int sweep_blocks_per_worker(const Params& P, const LaunchShape& ls);
+int aggregate_blocks(const Params& P, const LaunchShape& ls);
+
+}  // namespace laq

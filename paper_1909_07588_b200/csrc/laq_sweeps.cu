@@ -1,0 +1,533 @@
+// Steps 2-5 of the LAQ iteration as three streaming kernels over the per-worker vectors:
+//   radius_kernel     R_m = || g_m - Q_m(theta_hat^{k-1}) ||_inf                       (Sec. 2.1)
+//   quantize_kernel   codes of Eq. (5), ||dQ_m||^2 and ||eps_m||^2; its last block evaluates the
+//                     skip rule (7a)/(7b), advances the clocks and lists the uploaders    (Sec. 2.2)
+//   aggregate_kernel  for uploaders only: Q_m += dQ_m decoded from (R_m, codes) as the server
+//                     does after Eq. (6); grad += sum dQ_m; theta -= alpha grad; its last block
+//                     pushes ||alpha grad||^2 onto the ring of stored differences        (Eq. (4))
+// All three are bound by HBM bandwidth: a lane reads 16 B of a row per load, a warp 512 B
+// contiguous, with several independent loads in flight per thread.  Reductions are two-stage with
+// a fixed order (no floating-point atomics), so a run is reproducible bit for bit.
+//
+// Compiled with -fmad=false: every fp32 operation below is a single IEEE round-to-nearest
+// operation, in the order documented in laq.h.
+#include "laq_internal.cuh"
+
+namespace laq {
+
+namespace {
+
+__device__ __forceinline__ uint32_t fmix32(uint32_t x) {
+  x ^= x >> 16;
+  x *= 0x85ebca6bu;
+  x ^= x >> 13;
+  x *= 0xc2b2ae35u;
+  x ^= x >> 16;
+  return x;
+}
+
+// Exact int -> float for |v| < 2^23 without the conversion pipe.
+__device__ __forceinline__ float small_int_to_float(int v) {
+  return __int_as_float(0x4b400000 + v) - 12582912.0f;  // 1.5 * 2^23 + v, minus 1.5 * 2^23
+}
+
+struct Synth {
+  uint32_t key;
+  float cz, drift;
+  __device__ __forceinline__ void init(const Params& P, int m, unsigned long long k_iter) {
+    key = fmix32(P.seed_lo ^ fmix32(P.seed_hi + 0x9e3779b9u * (uint32_t)(m + 1)));
+    cz = P.cz;
+    float eta_m = (float)((double)P.eta0 * (double)(m + 1) / (double)P.M);
+    drift = __fmul_rn((float)k_iter, eta_m);
+  }
+  __device__ __forceinline__ float at(uint32_t i) const {
+    uint32_t h = fmix32(i ^ key);
+    const int ev = (int)__dp4a(h, 0x00010001u, 0u);          // b0 + b2
+    const int od = (int)__dp4a(h, 0x01000100u, 0u);          // b1 + b3
+    const int zi = ev + od - 510;
+    const int wi = ev - od;
+    float z = __fmul_rn(small_int_to_float(zi), cz);
+    float w = __fmul_rn(small_int_to_float(wi), cz);
+    return __fadd_rn(z, __fmul_rn(drift, w));
+  }
+  // coordinates 4v .. 4v+3, zero beyond p
+  __device__ __forceinline__ float4 at4(long long v, long long p) const {
+    long long i = 4 * v;
+    float4 r;
+    if (i + 3 < p) {
+      r.x = at((uint32_t)i);
+      r.y = at((uint32_t)i + 1);
+      r.z = at((uint32_t)i + 2);
+      r.w = at((uint32_t)i + 3);
+    } else {
+      r.x = (i < p) ? at((uint32_t)i) : 0.f;
+      r.y = (i + 1 < p) ? at((uint32_t)i + 1) : 0.f;
+      r.z = (i + 2 < p) ? at((uint32_t)i + 2) : 0.f;
+      r.w = (i + 3 < p) ? at((uint32_t)i + 3) : 0.f;
+    }
+    return r;
+  }
+};
+
+__device__ __forceinline__ uint32_t abs_bits(float x) { return __float_as_uint(x) & 0x7fffffffu; }
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Fixed-order block sum of one double per thread; result valid in thread 0.
+__device__ __forceinline__ double block_sum(double v, double* sh /* >= 32 doubles */) {
+  v = warp_sum(v);
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  __syncthreads();
+  if (lane == 0) sh[w] = v;
+  __syncthreads();
+  double t = 0.0;
+  if (threadIdx.x == 0)
+    for (int i = 0; i < nw; ++i) t += sh[i];
+  return t;
+}
+
+constexpr int kUnroll = 4;
+
+// ------------------------------------------------------------------------------------------------
+// radius
+// ------------------------------------------------------------------------------------------------
+template <bool SYNTH>
+__global__ void __launch_bounds__(512) radius_kernel(const Params P) {
+  if (*(volatile uint32_t*)&P.sc->err) return;
+  const int m = blockIdx.y;
+  const unsigned long long k = P.sc->k;
+  Synth sy;
+  if (SYNTH) sy.init(P, m, k + 1);
+  const float4* __restrict__ q4 = reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps);
+  const float4* __restrict__ g4 = SYNTH ? nullptr : reinterpret_cast<const float4*>(P.g + (long long)m * P.ps);
+  const long long nv = P.nv, stride = (long long)gridDim.x * blockDim.x;
+  uint32_t mx = 0;
+  for (long long v0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; v0 < nv; v0 += kUnroll * stride) {
+    float4 q[kUnroll], g[kUnroll];
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) {
+      const long long v = v0 + j * stride;
+      if (v < nv) {
+        q[j] = __ldg(q4 + v);
+        g[j] = SYNTH ? sy.at4(v, P.p) : __ldg(g4 + v);
+      } else {
+        q[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        g[j] = q[j];
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) {
+      // the ordering of |d| as unsigned bit patterns equals its ordering as floats, and puts
+      // inf and nan above every finite value, so a non-finite entry surfaces in R
+      mx = max(mx, abs_bits(__fsub_rn(g[j].x, q[j].x)));
+      mx = max(mx, abs_bits(__fsub_rn(g[j].y, q[j].y)));
+      mx = max(mx, abs_bits(__fsub_rn(g[j].z, q[j].z)));
+      mx = max(mx, abs_bits(__fsub_rn(g[j].w, q[j].w)));
+    }
+  }
+  mx = __reduce_max_sync(0xffffffffu, mx);
+  __shared__ uint32_t sh[32];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  if (lane == 0) sh[w] = mx;
+  __syncthreads();
+  if (w == 0) {
+    mx = (lane < ((blockDim.x + 31) >> 5)) ? sh[lane] : 0u;
+    mx = __reduce_max_sync(0xffffffffu, mx);
+    if (lane == 0) atomicMax(&P.Rbits[(k & 1ull) * P.M + m], mx);  // max is order independent
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// code packing: the 4 codes of coordinates 4v..4v+3 form one 4b-bit field at bit 4vb of the row
+// ------------------------------------------------------------------------------------------------
+template <int B>
+__device__ __forceinline__ void store_codes(uint32_t* row, long long v, uint32_t c0, uint32_t c1, uint32_t c2,
+                                            uint32_t c3, bool valid) {
+  if (B == 16) {
+    if (valid) reinterpret_cast<uint2*>(row)[v] = make_uint2(c0 | (c1 << 16), c2 | (c3 << 16));
+  } else if (B == 8) {
+    if (valid) row[v] = c0 | (c1 << 8) | (c2 << 16) | (c3 << 24);
+  } else if (B == 4) {
+    if (valid) reinterpret_cast<uint16_t*>(row)[v] = (uint16_t)(c0 | (c1 << 4) | (c2 << 8) | (c3 << 12));
+  } else if (B == 2) {
+    if (valid) reinterpret_cast<uint8_t*>(row)[v] = (uint8_t)(c0 | (c1 << 2) | (c2 << 4) | (c3 << 6));
+  } else {  // B == 1: two neighbouring lanes share a byte; v and the lane index have the same parity
+    uint32_t nib = valid ? (c0 | (c1 << 1) | (c2 << 2) | (c3 << 3)) : 0u;
+    uint32_t hi = __shfl_down_sync(0xffffffffu, nib, 1);
+    if (valid && !(v & 1)) reinterpret_cast<uint8_t*>(row)[v >> 1] = (uint8_t)(nib | (hi << 4));
+  }
+}
+
+template <int B>
+__device__ __forceinline__ void load_codes(const uint32_t* row, long long v, uint32_t c[4]) {
+  if (B == 16) {
+    uint2 w = __ldg(reinterpret_cast<const uint2*>(row) + v);
+    c[0] = w.x & 0xffffu; c[1] = w.x >> 16; c[2] = w.y & 0xffffu; c[3] = w.y >> 16;
+  } else if (B == 8) {
+    uint32_t w = __ldg(row + v);
+    c[0] = w & 255u; c[1] = (w >> 8) & 255u; c[2] = (w >> 16) & 255u; c[3] = w >> 24;
+  } else if (B == 4) {
+    uint32_t w = __ldg(reinterpret_cast<const uint16_t*>(row) + v);
+    c[0] = w & 15u; c[1] = (w >> 4) & 15u; c[2] = (w >> 8) & 15u; c[3] = (w >> 12) & 15u;
+  } else if (B == 2) {
+    uint32_t w = __ldg(reinterpret_cast<const uint8_t*>(row) + v);
+    c[0] = w & 3u; c[1] = (w >> 2) & 3u; c[2] = (w >> 4) & 3u; c[3] = (w >> 6) & 3u;
+  } else {
+    uint32_t w = __ldg(reinterpret_cast<const uint8_t*>(row) + (v >> 1)) >> (4 * (int)(v & 1));
+    c[0] = w & 1u; c[1] = (w >> 1) & 1u; c[2] = (w >> 2) & 1u; c[3] = (w >> 3) & 1u;
+  }
+}
+
+// One coordinate of Eq. (5)/(6).  Returns the code; updates the two fp64 sums.
+__device__ __forceinline__ uint32_t quantize_one(float g, float q, float R, float s, float levels, bool live,
+                                                 double& sdq, double& seps) {
+  if (!live) return 0u;
+  const float d = __fsub_rn(g, q);
+  const float t = __fadd_rn(__fdiv_rn(__fadd_rn(d, R), s), 0.5f);
+  const float f = fminf(fmaxf(floorf(t), 0.f), levels);
+  const float dq = __fsub_rn(__fmul_rn(s, f), R);
+  const float qn = __fadd_rn(q, dq);
+  const float e = __fsub_rn(g, qn);
+  sdq = fma((double)dq, (double)dq, sdq);   // the product of two fp32 values is exact in fp64
+  seps = fma((double)e, (double)e, seps);
+  return (uint32_t)f;
+}
+
+// Skip rule (7a)+(7b), clocks, uploader list, counters: run by the last block of quantize_kernel.
+__device__ void trigger_stage(const Params& P, int bpw) {
+  DevScalars* sc = P.sc;
+  const unsigned long long k = sc->k;
+  const int par = (int)(k & 1ull);
+  const bool tracing = P.trace_cap > 0 && sc->trace_pos < (uint32_t)P.trace_cap;
+  const long long trow = (long long)sc->trace_pos * P.M;
+  __shared__ int nonfinite;
+  if (threadIdx.x == 0) nonfinite = 0;
+  __syncthreads();
+  for (int m = threadIdx.x; m < P.M; m += blockDim.x)
+    if (P.Rbits[par * P.M + m] >= 0x7f800000u) atomicOr(&nonfinite, 1);
+  __syncthreads();
+  if (nonfinite) {  // freeze: nothing of this iteration is applied
+    if (threadIdx.x == 0) {
+      sc->n_up = 0;
+      atomicOr(&sc->err, 1u);
+    }
+    return;
+  }
+  for (int m = threadIdx.x; m < P.M; m += blockDim.x) {
+    double n_dq = 0.0, n_eps = 0.0;
+    const double* pq = P.part_q + (long long)m * kMaxSweepBlocksPerWorker * 2;
+    for (int i = 0; i < bpw; ++i) {  // fixed order
+      n_dq += __ldcg(pq + 2 * i);
+      n_eps += __ldcg(pq + 2 * i + 1);
+    }
+    double acc = 0.0;
+    for (int d = 0; d < P.D; ++d) {
+      const double term = (double)P.xi[d] * P.ring[(sc->ring_head + d) % P.D];
+      acc = acc + term;
+    }
+    const double rhs = acc / P.trig_c + 3.0 * (n_eps + P.n_epshat[m]);
+    const int t = P.clock[m];
+    const bool crit_a = n_dq <= rhs;
+    const bool crit_b = (P.clock_mode == 0) ? (t <= P.tbar) : (t + 2 <= P.tbar);
+    const bool skip = crit_a && crit_b && !(P.flags & LAQ_FLAG_TRIGGER_OFF);
+    if (skip) {
+      P.clock[m] = t + 1;
+    } else {
+      P.clock[m] = 0;
+      P.n_epshat[m] = n_eps;
+    }
+    P.skip[m] = skip ? 1 : 0;
+    P.norms[3 * m + 0] = n_dq;
+    P.norms[3 * m + 1] = n_eps;
+    P.norms[3 * m + 2] = rhs;
+    if (tracing) {
+      P.t_skip[trow + m] = skip ? 1 : 0;
+      P.t_R[trow + m] = __uint_as_float(P.Rbits[par * P.M + m]);
+      P.t_ndq[trow + m] = n_dq;
+      P.t_neps[trow + m] = n_eps;
+      P.t_rhs[trow + m] = rhs;
+    }
+    P.Rbits[(par ^ 1) * P.M + m] = 0u;  // clear the other parity for the next iteration's max
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const float levels = (float)((1u << P.b) - 1u);
+    const float two_tau = __fmul_rn(2.0f, __fdiv_rn(1.0f, levels));
+    int n = 0;
+    for (int m = 0; m < P.M; ++m) {
+      if (!P.skip[m]) {
+        const float R = __uint_as_float(P.Rbits[par * P.M + m]);
+        P.up_m[n] = m;
+        P.up_R[n] = R;
+        P.up_s[n] = __fmul_rn(two_tau, R);
+        ++n;
+      }
+    }
+    sc->n_up = n;
+    sc->uploads += (unsigned long long)n;
+    sc->bits += (unsigned long long)n * (32ull + (unsigned long long)P.b * (unsigned long long)P.p);
+    if (tracing) P.t_up[sc->trace_pos] = n;
+  }
+}
+
+template <bool SYNTH, int B>
+__global__ void __launch_bounds__(512) quantize_kernel(const Params P) {
+  __shared__ double sh[32];
+  __shared__ bool is_last;
+  const int m = blockIdx.y;
+  const bool frozen = *(volatile uint32_t*)&P.sc->err != 0;
+  const unsigned long long k = P.sc->k;
+  const uint32_t Rb = P.Rbits[(k & 1ull) * P.M + m];
+  const float R = __uint_as_float(Rb);
+  const bool finite = Rb < 0x7f800000u;
+  double sdq = 0.0, seps = 0.0;
+  if (!frozen && finite) {
+    Synth sy;
+    if (SYNTH) sy.init(P, m, k + 1);
+    const float levels = (float)((1u << B) - 1u);
+    const float s = __fmul_rn(__fmul_rn(2.0f, __fdiv_rn(1.0f, levels)), R);
+    const bool live = R > 0.f;  // R = 0: codes, dQ and eps are all zero
+    const float4* __restrict__ q4 = reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps);
+    const float4* __restrict__ g4 = SYNTH ? nullptr : reinterpret_cast<const float4*>(P.g + (long long)m * P.ps);
+    uint32_t* row = P.codes + (long long)m * P.cw;
+    const long long nv = P.nv, stride = (long long)gridDim.x * blockDim.x, p = P.p;
+    // all lanes of a warp run the same number of trips (the 1-bit packing shuffles between lanes)
+    const long long first = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long warp_first = first - (threadIdx.x & 31);
+    for (long long base = 0; warp_first + base < nv; base += kUnroll * stride) {
+      float4 q[kUnroll], g[kUnroll];
+      bool ok[kUnroll];
+#pragma unroll
+      for (int j = 0; j < kUnroll; ++j) {
+        const long long v = first + base + j * stride;
+        ok[j] = v < nv;
+        if (ok[j]) {
+          q[j] = __ldg(q4 + v);
+          g[j] = SYNTH ? sy.at4(v, p) : __ldg(g4 + v);
+        } else {
+          q[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+          g[j] = q[j];
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < kUnroll; ++j) {
+        const long long v = first + base + j * stride;
+        if (warp_first + base + j * stride >= nv) break;  // warp-uniform
+        const long long i = 4 * v;
+        const bool on = ok[j] && live;
+        const uint32_t c0 = quantize_one(g[j].x, q[j].x, R, s, levels, on && i < p, sdq, seps);
+        const uint32_t c1 = quantize_one(g[j].y, q[j].y, R, s, levels, on && i + 1 < p, sdq, seps);
+        const uint32_t c2 = quantize_one(g[j].z, q[j].z, R, s, levels, on && i + 2 < p, sdq, seps);
+        const uint32_t c3 = quantize_one(g[j].w, q[j].w, R, s, levels, on && i + 3 < p, sdq, seps);
+        store_codes<B>(row, v, c0, c1, c2, c3, ok[j]);
+      }
+    }
+  }
+  const double tdq = block_sum(sdq, sh);
+  const double teps = block_sum(seps, sh);
+  if (threadIdx.x == 0) {
+    double* pq = P.part_q + ((long long)m * kMaxSweepBlocksPerWorker + blockIdx.x) * 2;
+    __stcg(pq, tdq);
+    __stcg(pq + 1, teps);
+    __threadfence();
+    const uint32_t total = gridDim.x * gridDim.y;
+    const uint32_t ticket = atomicAdd(&P.sc->cnt_quant, 1u);
+    is_last = (ticket == total - 1);
+    if (is_last) P.sc->cnt_quant = 0;
+  }
+  __syncthreads();
+  if (is_last && !frozen) {
+    __threadfence();
+    trigger_stage(P, gridDim.x);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// lazy aggregate + theta step
+// ------------------------------------------------------------------------------------------------
+constexpr int kAggBatch = 4;  // uploaders whose loads are issued together
+
+template <int B>
+__global__ void __launch_bounds__(512) aggregate_kernel(const Params P) {
+  __shared__ int s_m[kMaxWorkers];
+  __shared__ float s_R[kMaxWorkers];
+  __shared__ float s_s[kMaxWorkers];
+  __shared__ double sh[32];
+  __shared__ bool is_last;
+  if (*(volatile uint32_t*)&P.sc->err) return;
+  const int n_up = (int)P.sc->n_up;
+  for (int u = threadIdx.x; u < n_up; u += blockDim.x) {
+    s_m[u] = P.up_m[u];
+    s_R[u] = P.up_R[u];
+    s_s[u] = P.up_s[u];
+  }
+  __syncthreads();
+  const long long nv = P.nv, p = P.p, stride = (long long)gridDim.x * blockDim.x;
+  float4* __restrict__ agg4 = reinterpret_cast<float4*>(P.agg);
+  float4* __restrict__ th4 = reinterpret_cast<float4*>(P.theta);
+  const float alpha = P.alpha;
+  double dsum = 0.0, tsum = 0.0;
+  for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < nv; v += stride) {
+    float4 a = agg4[v];
+    const long long i = 4 * v;
+    const bool tail = i + 3 >= p;
+    for (int u0 = 0; u0 < n_up; u0 += kAggBatch) {
+      float4 q[kAggBatch];
+      uint32_t c[kAggBatch][4];
+#pragma unroll
+      for (int j = 0; j < kAggBatch; ++j) {
+        if (u0 + j < n_up) {
+          const int m = s_m[u0 + j];
+          q[j] = *(reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps) + v);
+          load_codes<B>(P.codes + (long long)m * P.cw, v, c[j]);
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < kAggBatch; ++j) {
+        if (u0 + j < n_up) {
+          const int m = s_m[u0 + j];
+          const float R = s_R[u0 + j], s = s_s[u0 + j];
+          // the server's recovery of the innovation from the message: dQ = 2 tau R q - R
+          float d0 = __fsub_rn(__fmul_rn(s, (float)c[j][0]), R);
+          float d1 = __fsub_rn(__fmul_rn(s, (float)c[j][1]), R);
+          float d2 = __fsub_rn(__fmul_rn(s, (float)c[j][2]), R);
+          float d3 = __fsub_rn(__fmul_rn(s, (float)c[j][3]), R);
+          if (tail) {  // padding coordinates carry no innovation
+            if (i >= p) d0 = 0.f;
+            if (i + 1 >= p) d1 = 0.f;
+            if (i + 2 >= p) d2 = 0.f;
+            if (i + 3 >= p) d3 = 0.f;
+          }
+          q[j].x = __fadd_rn(q[j].x, d0);
+          q[j].y = __fadd_rn(q[j].y, d1);
+          q[j].z = __fadd_rn(q[j].z, d2);
+          q[j].w = __fadd_rn(q[j].w, d3);
+          *(reinterpret_cast<float4*>(P.qp + (long long)m * P.ps) + v) = q[j];
+          a.x = __fadd_rn(a.x, d0);  // uploads are applied in ascending worker order
+          a.y = __fadd_rn(a.y, d1);
+          a.z = __fadd_rn(a.z, d2);
+          a.w = __fadd_rn(a.w, d3);
+        }
+      }
+    }
+    agg4[v] = a;
+    float4 th = th4[v];
+    const float u0 = __fmul_rn(alpha, a.x), u1 = __fmul_rn(alpha, a.y), u2 = __fmul_rn(alpha, a.z),
+                u3 = __fmul_rn(alpha, a.w);
+    th.x = __fsub_rn(th.x, u0);
+    th.y = __fsub_rn(th.y, u1);
+    th.z = __fsub_rn(th.z, u2);
+    th.w = __fsub_rn(th.w, u3);
+    th4[v] = th;
+    dsum = fma((double)u0, (double)u0, dsum);
+    dsum = fma((double)u1, (double)u1, dsum);
+    dsum = fma((double)u2, (double)u2, dsum);
+    dsum = fma((double)u3, (double)u3, dsum);
+    tsum = fma((double)th.x, (double)th.x, tsum);
+    tsum = fma((double)th.y, (double)th.y, tsum);
+    tsum = fma((double)th.z, (double)th.z, tsum);
+    tsum = fma((double)th.w, (double)th.w, tsum);
+  }
+  const double bs = block_sum(dsum, sh);
+  const double bt = block_sum(tsum, sh);
+  if (threadIdx.x == 0) {
+    __stcg(P.part_d + blockIdx.x, bs);
+    __stcg(P.part_t + blockIdx.x, bt);
+    __threadfence();
+    const uint32_t ticket = atomicAdd(&P.sc->cnt_agg, 1u);
+    is_last = (ticket == gridDim.x - 1);
+    if (is_last) P.sc->cnt_agg = 0;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  // ||theta^{k+1} - theta^k||^2 = ||alpha grad^k||^2 : fixed-order sum of the block partials
+  double t = 0.0, t2 = 0.0;
+  for (int i = threadIdx.x; i < (int)gridDim.x; i += blockDim.x) {
+    t += __ldcg(P.part_d + i);
+    t2 += __ldcg(P.part_t + i);
+  }
+  const double d2 = block_sum(t, sh);
+  const double th2 = block_sum(t2, sh);
+  if (threadIdx.x == 0) {
+    DevScalars* sc = P.sc;
+    sc->theta_sq = th2;
+    const uint32_t head = (sc->ring_head + (uint32_t)P.D - 1u) % (uint32_t)P.D;
+    P.ring[head] = d2;
+    sc->ring_head = head;
+    if (P.trace_cap > 0 && sc->trace_pos < (uint32_t)P.trace_cap) {
+      P.t_d2[sc->trace_pos] = d2;
+      double loss = 0.0;
+      for (int m = 0; m < P.M; ++m) loss += P.loss_m[m];
+      P.t_loss[sc->trace_pos] = loss;
+      sc->trace_pos += 1;
+    }
+    sc->k += 1ull;
+  }
+}
+
+template <bool SYNTH>
+void launch_quant_b(const Params& P, dim3 grid, int threads, cudaStream_t st) {
+  switch (P.b) {
+    case 1: quantize_kernel<SYNTH, 1><<<grid, threads, 0, st>>>(P); break;
+    case 2: quantize_kernel<SYNTH, 2><<<grid, threads, 0, st>>>(P); break;
+    case 4: quantize_kernel<SYNTH, 4><<<grid, threads, 0, st>>>(P); break;
+    case 8: quantize_kernel<SYNTH, 8><<<grid, threads, 0, st>>>(P); break;
+    default: quantize_kernel<SYNTH, 16><<<grid, threads, 0, st>>>(P); break;
+  }
+}
+
+}  // namespace
+
+int sweep_blocks_per_worker(const Params& P, const LaunchShape& ls) {
+  // one resident wave: M x bpw blocks ~ SMs x blocks per SM, never more blocks than 16-byte groups
+  long long want = ((long long)kNumSMs * ls.sweep_blocks_per_sm + P.M - 1) / P.M;
+  long long need = (P.nv + ls.sweep_threads - 1) / ls.sweep_threads;
+  long long bpw = want < need ? want : need;
+  if (bpw < 1) bpw = 1;
+  if (bpw > kMaxSweepBlocksPerWorker) bpw = kMaxSweepBlocksPerWorker;
+  return (int)bpw;
+}
+
+int aggregate_blocks(const Params& P, const LaunchShape& ls) {
+  long long want = (long long)kNumSMs * ls.agg_blocks_per_sm;
+  long long need = (P.nv + ls.agg_threads - 1) / ls.agg_threads;
+  long long nb = want < need ? want : need;
+  return (int)(nb < 1 ? 1 : nb);
+}
+
+int launch_radius(const Params& P, const LaunchShape& ls, cudaStream_t st) {
+  dim3 grid(sweep_blocks_per_worker(P, ls), P.M);
+  if (P.model == LAQ_MODEL_SYNTH)
+    radius_kernel<true><<<grid, ls.sweep_threads, 0, st>>>(P);
+  else
+    radius_kernel<false><<<grid, ls.sweep_threads, 0, st>>>(P);
+  return 1;
+}
+
+int launch_quantize_trigger(const Params& P, const LaunchShape& ls, cudaStream_t st) {
+  dim3 grid(sweep_blocks_per_worker(P, ls), P.M);
+  if (P.model == LAQ_MODEL_SYNTH)
+    launch_quant_b<true>(P, grid, ls.sweep_threads, st);
+  else
+    launch_quant_b<false>(P, grid, ls.sweep_threads, st);
+  return 1;
+}
+
+int launch_aggregate(const Params& P, const LaunchShape& ls, cudaStream_t st) {
+  const int nb = aggregate_blocks(P, ls);
+  switch (P.b) {
+    case 1: aggregate_kernel<1><<<nb, ls.agg_threads, 0, st>>>(P); break;
+    case 2: aggregate_kernel<2><<<nb, ls.agg_threads, 0, st>>>(P); break;
+    case 4: aggregate_kernel<4><<<nb, ls.agg_threads, 0, st>>>(P); break;
+    case 8: aggregate_kernel<8><<<nb, ls.agg_threads, 0, st>>>(P); break;
+    default: aggregate_kernel<16><<<nb, ls.agg_threads, 0, st>>>(P); break;
+  }
+  return 1;
+}
+
+}  // namespace laq

@@ -1,0 +1,330 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same seeded inputs.
+
+Bars (written out here):
+  * codes, skip bits, clocks, counters, radii: bit-exact against the fp32 mirror on identical gradients;
+  * theta, grad, Q_prev: bit-exact against the fp32 mirror on identical gradients (same IEEE operation order);
+  * squared norms and the right-hand side of (7a): 1e-5 relative (fp64 sums in a different order: observed ~1e-15);
+  * model workloads (gradients computed by the GPU's own kernels): theta and loss within 1e-4 relative of the
+    fp64 oracle for as long as the skip decisions agree; the first disagreeing iteration is reported.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_1909_07588_b200 import laq, workloads
+
+pytestmark = pytest.mark.gpu
+
+NORM_RTOL = 1e-5
+TRAJ_RTOL = 1e-4
+
+
+def _mirror_for(w, precision=32, **over):
+    kw = dict(model=w.model, M=w.M, p=w.p, N=w.N, n_features=w.n_features, n_classes=w.n_classes,
+              n_hidden=w.n_hidden, alpha=w.alpha, lam=w.lam, b=w.b, D=w.D, xi=w.xi, tbar=w.tbar, seed=w.seed,
+              synth_sigma=w.synth_sigma, synth_eta0=w.synth_eta0, bf16_ops=w.bf16_ops, theta0=w.theta0)
+    kw.update(over)
+    model = kw.pop("model")
+    M, p = kw.pop("M"), kw.pop("p")
+    o = oracle.OracleLaq(precision, model, M, p, **kw)
+    if model in (oracle.MODEL_LOGREG_BIN, oracle.MODEL_SOFTMAX, oracle.MODEL_MLP2):
+        for m in range(w.M):
+            o.set_shard(m, w.X[m], w.y[m])
+    return o
+
+
+def _assert_state_bit_exact(gs, os_, p, b, check_codes=True, ctx=None):
+    """gs: laq.get_state(...) ; os_: oracle mirror state()."""
+    np.testing.assert_array_equal(gs["theta"], os_["theta"].astype(np.float32))
+    np.testing.assert_array_equal(gs["agg"], os_["agg"].astype(np.float32))
+    np.testing.assert_array_equal(gs["qprev"], os_["qp"].astype(np.float32))
+    np.testing.assert_array_equal(gs["clock"], os_["clock"])
+    assert gs["k"] == os_["k"] and gs["uploads"] == os_["uploads"] and gs["bits"] == os_["bits"]
+    np.testing.assert_allclose(gs["n_eps_hat"], os_["n_epshat"], rtol=NORM_RTOL, atol=0)
+    np.testing.assert_allclose(gs["ring"], os_["hist"], rtol=NORM_RTOL, atol=0)
+    if check_codes:
+        for m in range(gs["codes"].shape[0]):
+            np.testing.assert_array_equal(gs["codes"][m], oracle.pack_codes(os_["codes"][m], b))
+
+
+def _assert_trace_row(tr, j, st):
+    np.testing.assert_array_equal(tr["skip"][j], st["skip"].astype(np.uint8))
+    np.testing.assert_array_equal(tr["R"][j], st["R"].astype(np.float32))
+    np.testing.assert_allclose(tr["n_dq"][j], st["n_dq"], rtol=NORM_RTOL, atol=0)
+    np.testing.assert_allclose(tr["n_eps"][j], st["n_eps"], rtol=NORM_RTOL, atol=0)
+    np.testing.assert_allclose(tr["rhs"][j], st["rhs"], rtol=NORM_RTOL, atol=0)
+    assert tr["dtheta2"][j] == pytest.approx(st["dtheta2"], rel=NORM_RTOL)
+    assert tr["uploads"][j] == st["uploads"]
+
+
+# ------------------------------------------------------------------------------------------------
+# steps 2-5 on identical gradients (caller-supplied), every b, ragged sizes
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("b", [1, 2, 4, 8, 16])
+@pytest.mark.parametrize("p", [1, 3, 31, 33, 1000, 5003, 70001])
+def test_given_gradients_bit_exact(b, p):
+    M, D, tbar, alpha, iters = 5, 4, 6, 0.05, 25 if p < 10000 else 8
+    rng = np.random.default_rng(1000 * b + p)
+    c = rng.standard_normal((M, p))
+    Lm = rng.uniform(0.05, 2.0, M)
+    ctx = laq.Laq(model=laq.MODEL_EXTERNAL, M=M, p=p, alpha=alpha, b=b, D=D, xi=np.full(D, 0.2), tbar=tbar,
+                  trace_capacity=1)
+    mir = oracle.OracleLaq(32, oracle.MODEL_GIVEN, M, p, alpha=alpha, b=b, D=D, xi=np.full(D, 0.2), tbar=tbar)
+    theta = np.zeros(p, np.float32)
+    skipped = 0
+    for k in range(iters):
+        g = (Lm[:, None] * (theta.astype(np.float64)[None, :] - c)).astype(np.float32)
+        ctx.set_gradients(g)
+        tr = ctx.step(1, trace=True)
+        st = mir.step_given(g)
+        _assert_trace_row(tr, 0, st)
+        gs = ctx.get_state(codes=True, g=True)
+        np.testing.assert_array_equal(gs["g"], g)
+        _assert_state_bit_exact(gs, mir.state(), p, b)
+        np.testing.assert_array_equal(gs["skip"], st["skip"].astype(np.uint8))
+        theta = gs["theta"]
+        skipped += int(st["skip"].sum())
+    if b >= 4:
+        assert skipped > 0      # the lazy branch was exercised
+    ctx.close()
+
+
+def test_given_gradients_zero_innovation_and_trigger_off():
+    M, p, b = 3, 100, 4
+    g = np.random.default_rng(0).standard_normal((M, p)).astype(np.float32)
+    ctx = laq.Laq(model=laq.MODEL_EXTERNAL, M=M, p=p, alpha=0.1, b=b, D=2, xi=[0.4, 0.4], tbar=50,
+                  flags=laq.FLAG_TRIGGER_OFF, trace_capacity=1)
+    mir = oracle.OracleLaq(32, oracle.MODEL_GIVEN, M, p, alpha=0.1, b=b, D=2, xi=[0.4, 0.4], tbar=50,
+                           flags=oracle.FLAG_TRIGGER_OFF)
+    for k in range(6):
+        gk = g.copy()
+        if k >= 3:
+            gk[1] = ctx.get_state()["qprev"][1]        # worker 1: g equals its stored copy -> R = 0
+        ctx.set_gradients(gk)
+        tr = ctx.step(1, trace=True)
+        st = mir.step_given(gk)
+        _assert_trace_row(tr, 0, st)
+        assert not tr["skip"].any()                     # Algorithm 1: everybody uploads
+        _assert_state_bit_exact(ctx.get_state(codes=True), mir.state(), p, b)
+        if k >= 3:
+            assert tr["R"][0, 1] == 0.0 and tr["n_dq"][0, 1] == 0.0
+    assert ctx.get_state()["uploads"] == 6 * M
+    ctx.close()
+
+
+def test_strict_clock_tbar_one_never_skips():
+    M, p = 4, 64
+    rng = np.random.default_rng(3)
+    ctx = laq.Laq(model=laq.MODEL_EXTERNAL, M=M, p=p, alpha=0.3, b=4, D=1, xi=[0.8], tbar=1, clock_mode=1,
+                  trace_capacity=1)
+    g = rng.standard_normal((M, p)).astype(np.float32) * 1e-3
+    for k in range(20):
+        ctx.set_gradients(g + np.float32(1e-6) * k)
+        assert not ctx.step(1, trace=True)["skip"].any()
+    ctx.close()
+
+
+# ------------------------------------------------------------------------------------------------
+# the synthetic large-p stream, generated inside the kernels
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("b", [2, 4, 8])
+@pytest.mark.parametrize("M,p", [(8, 70001), (3, 1_000_003)])
+def test_synthetic_stream_bit_exact(b, M, p):
+    iters = 30 if p < 100000 else 6
+    w = workloads.c4(M=M, p=p, b=b, iters=iters)
+    ctx = laq.from_workload(w, trace_capacity=iters)
+    mir = _mirror_for(w)
+    tr = ctx.step(iters, trace=True)
+    for j in range(iters):
+        st = mir.step()
+        _assert_trace_row(tr, j, st)
+    _assert_state_bit_exact(ctx.get_state(codes=True), mir.state(), p, b)
+    assert tr["skip"][0].sum() == 0
+    if p < 100000:
+        assert tr["skip"].sum() > 0
+    ctx.close()
+
+
+def test_synthetic_full_size_sampled_workers():
+    """The benchmark's launch configuration (M = 64, p = 25.6 M, b = 8): worker messages of the first
+    iteration against the mirror for sampled workers, the aggregate invariant, and the clock rules."""
+    M, p, b = 64, 25_600_000, 8
+    w = workloads.c4(M=M, p=p, b=b)
+    ctx = laq.from_workload(w, trace_capacity=4)
+    tr = ctx.step(1, trace=True)
+    assert not tr["skip"].any() and tr["uploads"][0] == M          # every worker uploads at k = 1
+    zero = np.zeros(p, np.float32)
+    for m in (0, 17, 63):
+        g = oracle.synth_gradient(w.seed, m, M, p, 1, w.synth_sigma, w.synth_eta0)
+        r = oracle.quantize(g, zero, b, np.float32)
+        got = ctx.get_worker(m)
+        assert got["R"] == r["R"] == tr["R"][0, m]
+        np.testing.assert_array_equal(got["codes"], oracle.pack_codes(r["q"], b))
+        np.testing.assert_array_equal(got["qprev"], r["qnew"])
+        assert tr["n_dq"][0, m] == pytest.approx(r["n_dq"], rel=NORM_RTOL)
+        assert tr["n_eps"][0, m] == pytest.approx(r["n_eps"], rel=NORM_RTOL)
+        del g, r, got
+    # grad^1 = sum_m Q_m in ascending worker order (fp32 adds), theta^2 = -alpha grad^1 (theta^1 = 0)
+    acc = np.zeros(p, np.float32)
+    for m in range(M):
+        acc += ctx.get_worker(m, codes=False)["qprev"]
+    s = ctx.get_state(big=False)
+    np.testing.assert_array_equal(s["agg"], acc)
+    u = np.float32(w.alpha) * acc
+    np.testing.assert_array_equal(s["theta"], -u)
+    assert tr["dtheta2"][0] == pytest.approx(np.sum(u.astype(np.float64) ** 2), rel=NORM_RTOL)
+    assert s["bits"] == M * (32 + b * p)
+    # three more iterations: skips appear, clocks count them, the aggregate still equals the sum of copies
+    tr = ctx.step(3, trace=True)
+    assert tr["skip"].sum() > 0
+    s = ctx.get_state(big=False)
+    consecutive = np.zeros(M, int)
+    for j in range(3):
+        consecutive = np.where(tr["skip"][j] == 1, consecutive + 1, 0)
+    np.testing.assert_array_equal(s["clock"], consecutive)
+    acc64 = np.zeros(p)
+    for m in range(M):
+        acc64 += ctx.get_worker(m, codes=False)["qprev"]
+    assert np.max(np.abs(s["agg"] - acc64)) <= 1e-5 * np.max(np.abs(acc64))
+    ctx.close()
+
+
+# ------------------------------------------------------------------------------------------------
+# model workloads: gradients from the library's own kernels
+# ------------------------------------------------------------------------------------------------
+def _run_model_parity(w, iters, chunk=50):
+    """GPU trajectory vs fp64 oracle (trajectory bar) and vs the fp32 mirror fed with the GPU's own
+    gradients (bit-exact bar for steps 2-5).  Returns the first iteration whose skip mask differs from
+    the fp64 oracle's (or None)."""
+    ctx = laq.from_workload(w, trace_capacity=1)
+    o64 = _mirror_for(w, 64)
+    mir = oracle.OracleLaq(32, oracle.MODEL_GIVEN, w.M, w.p, alpha=w.alpha, b=w.b, D=w.D, xi=w.xi, tbar=w.tbar,
+                           theta0=w.theta0)
+    first_diff = None
+    for k in range(iters):
+        tr = ctx.step(1, trace=True)
+        gs = ctx.get_state(g=True, codes=True)
+        st32 = mir.step_given(gs["g"])
+        _assert_trace_row(tr, 0, st32)
+        _assert_state_bit_exact(gs, mir.state(), w.p, w.b)
+        if first_diff is None:
+            st64 = o64.step()
+            s64 = o64.state(big=False)
+            if not np.array_equal(st64["skip"].astype(np.uint8), tr["skip"][0]):
+                first_diff = k + 1
+            else:
+                # gradients agree with the fp64 model gradients, theta and loss follow the fp64 trajectory
+                g64 = o64.state()["g"]
+                assert np.linalg.norm(gs["g"] - g64) <= TRAJ_RTOL * np.linalg.norm(g64)
+                assert np.linalg.norm(gs["theta"] - s64["theta"]) <= TRAJ_RTOL * np.linalg.norm(s64["theta"])
+                assert tr["loss"][0] == pytest.approx(st64["loss"], rel=TRAJ_RTOL)
+    print("%s: %d iterations, first skip-mask disagreement with the fp64 oracle: %s" % (w.name, iters, first_diff))
+    ctx.close()
+    return first_diff
+
+
+def test_c0_logreg_full():
+    w = workloads.c0()
+    first = _run_model_parity(w, w.iters)
+    assert first is None or first > 20
+
+
+def test_c2_shape_logreg54_reduced():
+    w = workloads.c2(n_per=3001, iters=60)      # ragged: not a multiple of the row tile
+    first = _run_model_parity(w, w.iters)
+    assert first is None or first > 20
+
+
+def test_c1_shape_softmax_reduced():
+    w = workloads.c1(n_per=333, iters=40)
+    first = _run_model_parity(w, w.iters)
+    assert first is None or first > 15
+
+
+def test_softmax_small_odd_shapes():
+    w = workloads.c1(n_per=37, F=50, C=3, M=4, iters=15)
+    _run_model_parity(w, w.iters)
+
+
+# ------------------------------------------------------------------------------------------------
+# state round trip, error paths
+# ------------------------------------------------------------------------------------------------
+def test_state_round_trip_resumes_bit_identically():
+    w = workloads.c4(M=6, p=12345, b=4)
+    a = laq.from_workload(w, trace_capacity=8)
+    a.step(7)
+    s = a.get_state()
+    tr_a = a.step(8, trace=True)
+    b_ = laq.from_workload(w, trace_capacity=8)
+    b_.set_state(theta=s["theta"], agg=s["agg"], qprev=s["qprev"], n_eps_hat=s["n_eps_hat"], clock=s["clock"],
+                 ring=s["ring"], counters=s["counters"])
+    tr_b = b_.step(8, trace=True)
+    for key in tr_a:
+        np.testing.assert_array_equal(tr_a[key], tr_b[key])
+    sa, sb = a.get_state(codes=True), b_.get_state(codes=True)
+    for key in ("theta", "agg", "qprev", "n_eps_hat", "clock", "ring", "counters", "codes"):
+        np.testing.assert_array_equal(sa[key], sb[key])
+    a.close()
+    b_.close()
+
+
+def test_runs_are_reproducible_bit_for_bit():
+    w = workloads.c4(M=7, p=54321, b=2)
+    outs = []
+    for _ in range(2):
+        c = laq.from_workload(w, trace_capacity=12)
+        tr = c.step(12, trace=True)
+        outs.append((tr, c.get_state()))
+        c.close()
+    for key in outs[0][0]:
+        np.testing.assert_array_equal(outs[0][0][key], outs[1][0][key])
+    for key in ("theta", "agg", "qprev", "ring"):
+        np.testing.assert_array_equal(outs[0][1][key], outs[1][1][key])
+
+
+def test_api_misuse_returns_error_codes():
+    with pytest.raises(laq.LaqError) as e:
+        laq.Laq(model=laq.MODEL_SYNTH, M=4, p=100, b=3)
+    assert e.value.status == laq.LAQ_EINVAL and "b must be" in str(e.value)
+    w = workloads.c0()
+    c = laq.Laq(model=w.model, M=w.M, p=w.p, N=w.N, n_features=w.n_features, alpha=w.alpha, lam=w.lam, b=w.b)
+    with pytest.raises(laq.LaqError) as e:
+        c.step(1)                                            # shards not loaded
+    assert e.value.status == laq.LAQ_ESTATE
+    with pytest.raises(laq.LaqError) as e:
+        c.load_shards(0, w.X[0][:10], w.y[0][:10])           # wrong N_m
+    assert e.value.status == laq.LAQ_EINVAL
+    with pytest.raises(laq.LaqError) as e:
+        c.step(1, trace=True)                                # no trace capacity
+    assert e.value.status in (laq.LAQ_EINVAL, laq.LAQ_ESTATE)
+    c.close()
+    # workspace too small / misaligned
+    import ctypes as C
+    import torch
+    L = laq.load_library()
+    cfg, keep = laq.make_config(model=laq.MODEL_SYNTH, M=4, p=1000, b=4)
+    buf = torch.empty(laq.workspace_bytes(cfg) + 512, dtype=torch.uint8, device="cuda")
+    h = C.c_void_p()
+    assert L.laq_init(C.byref(h), C.byref(cfg), C.c_void_p(buf.data_ptr()), 1024, None, None) == laq.LAQ_EWORKSPACE
+    L.laq_destroy(h)
+    assert L.laq_init(C.byref(h), C.byref(cfg), C.c_void_p(buf.data_ptr() + 4), buf.numel() - 4, None, None) == laq.LAQ_EWORKSPACE
+    L.laq_destroy(h)
+
+
+def test_non_finite_gradient_freezes_state_and_is_reported():
+    M, p = 3, 200
+    g = np.random.default_rng(1).standard_normal((M, p)).astype(np.float32)
+    c = laq.Laq(model=laq.MODEL_EXTERNAL, M=M, p=p, alpha=0.1, b=4, D=2, xi=[0.4, 0.4], tbar=10, trace_capacity=1)
+    c.set_gradients(g)
+    c.step(1, trace=True)
+    before = c.get_state()
+    bad = g.copy()
+    bad[2, 17] = np.nan
+    c.set_gradients(bad)
+    with pytest.raises(laq.LaqError) as e:
+        c.step(1, trace=True)
+    assert e.value.status == laq.LAQ_ENONFINITE
+    with pytest.raises(laq.LaqError):
+        c.get_state()
+    c.close()
+    assert before["k"] == 1
