@@ -23,9 +23,9 @@
  *     (laq_step with a trace, laq_get_state, laq_sync) as LAQ_ENONFINITE.
  *   - Floating point: theta, gradients and quantizer state are fp32; each quantizer operation is one
  *     IEEE round-to-nearest operation in the order  d = g - Q_prev ; R = max|d| ; s = (2 tau) R ;
- *     t = (d + R)/s + 1/2 ; q = clamp(floor t) ; dQ = s q - R ; Q_new = Q_prev + dQ ; eps = g - Q_new,
- *     with no fused multiply-add; squared norms are fp64 sums of exact fp32 products; the skip rule
- *     is evaluated in fp64.
+ *     t = (d + R)/s + 1/2 ; q = floor t ; dQ = fma(s, q, -R) (Eq. (6) with a single rounding) ;
+ *     Q_new = Q_prev + dQ ; eps = g - Q_new, with no other fused multiply-add; squared norms are fp64
+ *     sums of exact fp32 products; the skip rule is evaluated in fp64.
  *   - Code stream of worker m (the paper's b p-bit part of the upload message): code i occupies bits
  *     [(i b) mod 32, +b) of 32-bit word floor(i b / 32), least significant first.
  *   - Readings where the paper is silent: initial Q_m = 0, ||eps_hat_m||^2 = 0, grad^0 = 0, the D stored
@@ -64,12 +64,14 @@ typedef enum {
   LAQ_MODEL_EXTERNAL = 4    /* the caller supplies g (M x p) before every step with laq_set_gradients */
 } laq_model;
 
-/* LAQ_MODEL_SYNTH stream (fp32, every operation IEEE, no fused multiply-add):
+/* LAQ_MODEL_SYNTH stream (fp32; coordinates in groups of four, group v = i / 4, e = i mod 4):
  *   fmix32(x): x ^= x>>16; x *= 0x85ebca6b; x ^= x>>13; x *= 0xc2b2ae35; x ^= x>>16
- *   key_m = fmix32(seed_lo ^ fmix32(seed_hi + 0x9e3779b9 (m+1))),  h = fmix32((uint32) i ^ key_m)
- *   with bytes b0..b3 of h (b0 lowest): zi = b0+b1+b2+b3-510, wi = b0-b1+b2-b3,
- *   cz = fp32(synth_sigma / sqrt(21845)), eta_m = fp32(synth_eta0 (m+1)/M),
- *   g_m^k[i] = zi cz + (k eta_m)(wi cz),  k = 1, 2, ...   (requires p < 2^32) */
+ *   key_m = fmix32(seed_lo ^ fmix32(seed_hi + 0x9e3779b9 (m+1)))
+ *   h0 = fmix32((uint32) v ^ key_m);  h1 = h0 * 0x9e3779b1;  h1 ^= h1 >> 15
+ *   for a word with bytes b0..b3 (b0 lowest): S = b0+b1+b2+b3-510, A = b0-b1+b2-b3
+ *   z_0 = S(h0), z_1 = A(h0), z_2 = S(h1), z_3 = A(h1)
+ *   cz = fp32(synth_sigma / sqrt(21845)), eta_m = fp32(synth_eta0 (m+1)/M)
+ *   g_m^k[i] = fma(fl(k eta_m), z_{e xor 2}, z_e) * cz,  k = 1, 2, ...   (requires p < 2^32) */
 
 enum {
   LAQ_FLAG_TRIGGER_OFF = 2u /* every worker uploads every iteration: Algorithm 1 (QGD) */

@@ -31,8 +31,13 @@ def build(force=False):
     if not force and os.path.exists(_SO) and os.path.getmtime(_SO) >= os.path.getmtime(_SRC):
         return _SO
     tmp = _SO + ".tmp.%d" % os.getpid()
-    cmd = ["g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math", "-shared", "-fPIC",
-           "-o", tmp, _SRC]
+    cmd = ["g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math", "-shared", "-fPIC"]
+    try:  # explicit std::fma calls map to the hardware instruction where there is one (same result, faster)
+        if " fma " in open("/proc/cpuinfo").read():
+            cmd.append("-mfma")
+    except OSError:
+        pass
+    cmd += ["-o", tmp, _SRC]
     subprocess.run(cmd, check=True)
     os.replace(tmp, _SO)
     return _SO

@@ -84,7 +84,7 @@ float round_bf16(float x) {
 //        n_dq = ||dq||^2, n_eps = ||eps||^2  (fp64 sums, index order)
 // Operation order (each one IEEE operation in T):
 //   d = g - qp ; R = max |d| ; tau = 1/(2^b-1) ; s = (2 tau) R ; t = (d + R)/s + 1/2 ;
-//   q = clamp(floor(t), 0, 2^b-1) ; dq = s q - R ; qnew = qp + dq ; eps = g - qnew.
+//   q = clamp(floor(t), 0, 2^b-1) ; dq = fma(s, q, -R) (one rounding) ; qnew = qp + dq ; eps = g - qnew.
 // ---------------------------------------------------------------------------------------------
 template <typename T>
 void quantize(const T* g, const T* qp, i64 p, int b, T* R_out, int32_t* q, T* dq, T* qnew, T* eps,
@@ -111,7 +111,7 @@ void quantize(const T* g, const T* qp, i64 p, int b, T* R_out, int32_t* q, T* dq
       if (f < (T)0) f = 0;
       if (f > levels) f = levels;
       qi = (int32_t)f;
-      dqi = s * (T)qi - R;
+      dqi = std::fma(s, (T)qi, -R);  // Eq. (6), one rounding
     }
     T qn = qp[i] + dqi;
     T e = g[i] - qn;
@@ -133,7 +133,7 @@ void decode(T R, const int32_t* q, const T* qp, i64 p, int b, T* qnew, T* dq) {
   const T tau = (T)1 / levels;
   const T s = ((T)2 * tau) * R;
   for (i64 i = 0; i < p; ++i) {
-    T d = (R > (T)0) ? (s * (T)q[i] - R) : (T)0;
+    T d = (R > (T)0) ? std::fma(s, (T)q[i], -R) : (T)0;
     if (dq) dq[i] = d;
     qnew[i] = qp[i] + d;
   }
@@ -313,16 +313,18 @@ double grad_mlp2(const float* X, const int32_t* y, i64 n, int F, int H, int C, c
 // ---------------------------------------------------------------------------------------------
 // Synthetic gradient stream for the large-p throughput workload (no data shard): a counter-based
 // generator, so that both this file and the CUDA library can produce the same fp32 values from
-// its definition alone.
+// its definition alone.  Coordinates come in groups of four (group v = i / 4, e = i mod 4):
 //   fmix32(x): the 32-bit finaliser of MurmurHash3 (A. Appleby, public domain):
 //       x ^= x>>16; x *= 0x85ebca6b; x ^= x>>13; x *= 0xc2b2ae35; x ^= x>>16
 //   key_m  = fmix32( seed_lo ^ fmix32( seed_hi + 0x9e3779b9 * (m+1) ) )
-//   h      = fmix32( (uint32) i ^ key_m )           (coordinate i < 2^32), bytes b0..b3 (b0 lowest)
-//   zi     = b0 + b1 + b2 + b3 - 510                (sum of four uniform bytes: near-Gaussian)
-//   wi     = b0 - b1 + b2 - b3                      (uncorrelated with zi)
-//   cz     = fp32( sigma / sqrt(21845) )            (21845 = 4 (256^2 - 1)/12, the variance of zi)
+//   h0     = fmix32( (uint32) v ^ key_m ) ;  h1 = h0 * 0x9e3779b1 ;  h1 ^= h1 >> 15
+//   with bytes b0..b3 of a word (b0 lowest):  S(h) = b0+b1+b2+b3-510 ,  A(h) = b0-b1+b2-b3
+//       (sums of four uniform bytes: near-Gaussian, variance 21845 = 4 (256^2-1)/12, S and A uncorrelated)
+//   z_0 = S(h0), z_1 = A(h0), z_2 = S(h1), z_3 = A(h1)
+//   cz     = fp32( sigma / sqrt(21845) )
 //   eta_m  = fp32( eta0 (m+1) / M )                 (heterogeneous drift speed)
-//   g_m^k[i] = fl( fl(zi cz) + fl( fl(k eta_m) fl(wi cz) ) )     all fp32, k = 1, 2, ...
+//   g_m^k[i] = fl( fma( fl(k eta_m), z_{e xor 2}, z_e ) * cz )      fp32, k = 1, 2, ...
+//       (the slowly growing drift term reuses the z of the partner coordinate e xor 2)
 // ---------------------------------------------------------------------------------------------
 uint32_t fmix32(uint32_t x) {
   x ^= x >> 16;
@@ -338,15 +340,21 @@ void synth_gradient(uint64_t seed, int m, int M, i64 p, i64 k, float sigma, floa
   float cz = (float)((double)sigma / std::sqrt(21845.0));
   float eta_m = (float)((double)eta0 * (double)(m + 1) / (double)M);
   float drift = (float)k * eta_m;
-  for (i64 i = 0; i < p; ++i) {
-    uint32_t h = fmix32((uint32_t)i ^ key);
-    int b0 = h & 255, b1 = (h >> 8) & 255, b2 = (h >> 16) & 255, b3 = (h >> 24) & 255;
-    int zi = b0 + b1 + b2 + b3 - 510;
-    int wi = b0 - b1 + b2 - b3;
-    float z = (float)zi * cz;
-    float w = (float)wi * cz;
-    float dw = drift * w;
-    g[i] = z + dw;
+  for (i64 v = 0; 4 * v < p; ++v) {
+    uint32_t h[2];
+    h[0] = fmix32((uint32_t)v ^ key);
+    h[1] = h[0] * 0x9e3779b1u;
+    h[1] ^= h[1] >> 15;
+    float z[4];
+    for (int j = 0; j < 2; ++j) {
+      int b0 = h[j] & 255, b1 = (h[j] >> 8) & 255, b2 = (h[j] >> 16) & 255, b3 = (h[j] >> 24) & 255;
+      z[2 * j] = (float)(b0 + b1 + b2 + b3 - 510);
+      z[2 * j + 1] = (float)(b0 - b1 + b2 - b3);
+    }
+    for (int e = 0; e < 4 && 4 * v + e < p; ++e) {
+      float a = std::fmaf(drift, z[e ^ 2], z[e]);
+      g[4 * v + e] = a * cz;
+    }
   }
 }
 

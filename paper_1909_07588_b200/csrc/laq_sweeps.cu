@@ -10,7 +10,7 @@
 // a fixed order (no floating-point atomics), so a run is reproducible bit for bit.
 //
 // Compiled with -fmad=false: every fp32 operation below is a single IEEE round-to-nearest
-// operation, in the order documented in laq.h.
+// operation, in the order documented in laq.h; fused multiply-adds appear only where written.
 #include "laq_internal.cuh"
 
 namespace laq {
@@ -26,11 +26,8 @@ __device__ __forceinline__ uint32_t fmix32(uint32_t x) {
   return x;
 }
 
-// Exact int -> float for |v| < 2^23 without the conversion pipe.
-__device__ __forceinline__ float small_int_to_float(int v) {
-  return __int_as_float(0x4b400000 + v) - 12582912.0f;  // 1.5 * 2^23 + v, minus 1.5 * 2^23
-}
-
+// Synthetic gradient stream (definition in laq.h).  One strong hash per group of four coordinates,
+// a cheap second word from it, and two near-Gaussian byte sums per word.
 struct Synth {
   uint32_t key;
   float cz, drift;
@@ -40,31 +37,33 @@ struct Synth {
     float eta_m = (float)((double)P.eta0 * (double)(m + 1) / (double)P.M);
     drift = __fmul_rn((float)k_iter, eta_m);
   }
-  __device__ __forceinline__ float at(uint32_t i) const {
-    uint32_t h = fmix32(i ^ key);
-    const int ev = (int)__dp4a(h, 0x00010001u, 0u);          // b0 + b2
-    const int od = (int)__dp4a(h, 0x01000100u, 0u);          // b1 + b3
-    const int zi = ev + od - 510;
-    const int wi = ev - od;
-    float z = __fmul_rn(small_int_to_float(zi), cz);
-    float w = __fmul_rn(small_int_to_float(wi), cz);
-    return __fadd_rn(z, __fmul_rn(drift, w));
-  }
-  // coordinates 4v .. 4v+3, zero beyond p
-  __device__ __forceinline__ float4 at4(long long v, long long p) const {
-    long long i = 4 * v;
+  // coordinates 4v .. 4v+3
+  __device__ __forceinline__ float4 at4(long long v) const {
+    const uint32_t h0 = fmix32((uint32_t)v ^ key);
+    uint32_t h1 = h0 * 0x9e3779b1u;
+    h1 ^= h1 >> 15;
+    const int e0 = (int)__dp4a(h0, 0x00010001u, 0u), o0 = (int)__dp4a(h0, 0x01000100u, 0u);  // b0+b2, b1+b3
+    const int e1 = (int)__dp4a(h1, 0x00010001u, 0u), o1 = (int)__dp4a(h1, 0x01000100u, 0u);
+    // exact int -> float through the mantissa of 1.5 * 2^23 (the -510 offset folds into the constant)
+    const float z0 = __int_as_float(0x4b400000 + e0 + o0) - (12582912.0f + 510.0f);
+    const float z1 = __int_as_float(0x4b400000 + e0 - o0) - 12582912.0f;
+    const float z2 = __int_as_float(0x4b400000 + e1 + o1) - (12582912.0f + 510.0f);
+    const float z3 = __int_as_float(0x4b400000 + e1 - o1) - 12582912.0f;
     float4 r;
-    if (i + 3 < p) {
-      r.x = at((uint32_t)i);
-      r.y = at((uint32_t)i + 1);
-      r.z = at((uint32_t)i + 2);
-      r.w = at((uint32_t)i + 3);
-    } else {
-      r.x = (i < p) ? at((uint32_t)i) : 0.f;
-      r.y = (i + 1 < p) ? at((uint32_t)i + 1) : 0.f;
-      r.z = (i + 2 < p) ? at((uint32_t)i + 2) : 0.f;
-      r.w = (i + 3 < p) ? at((uint32_t)i + 3) : 0.f;
-    }
+    r.x = __fmul_rn(__fmaf_rn(drift, z2, z0), cz);
+    r.y = __fmul_rn(__fmaf_rn(drift, z3, z1), cz);
+    r.z = __fmul_rn(__fmaf_rn(drift, z0, z2), cz);
+    r.w = __fmul_rn(__fmaf_rn(drift, z1, z3), cz);
+    return r;
+  }
+  // the same with zeros at coordinates >= p (last group of a row)
+  __device__ __forceinline__ float4 at4_masked(long long v, long long p) const {
+    float4 r = at4(v);
+    const long long i = 4 * v;
+    if (i >= p) r.x = 0.f;
+    if (i + 1 >= p) r.y = 0.f;
+    if (i + 2 >= p) r.z = 0.f;
+    if (i + 3 >= p) r.w = 0.f;
     return r;
   }
 };
@@ -104,16 +103,20 @@ __global__ void __launch_bounds__(512) radius_kernel(const Params P) {
   if (SYNTH) sy.init(P, m, k + 1);
   const float4* __restrict__ q4 = reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps);
   const float4* __restrict__ g4 = SYNTH ? nullptr : reinterpret_cast<const float4*>(P.g + (long long)m * P.ps);
-  const long long nv = P.nv, stride = (long long)gridDim.x * blockDim.x;
+  // groups [0, nv_main) lie wholly inside the row; the (at most five) groups after them may contain
+  // padding coordinates and take the masked path
+  const long long nv = P.nv, nv_main = (P.p / 4) & ~1ll, stride = (long long)gridDim.x * blockDim.x;
   uint32_t mx = 0;
-  for (long long v0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; v0 < nv; v0 += kUnroll * stride) {
+  // the ordering of |d| as unsigned bit patterns equals its ordering as floats, and puts inf and nan
+  // above every finite value, so a non-finite entry surfaces in R
+  for (long long v0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; v0 < nv_main; v0 += kUnroll * stride) {
     float4 q[kUnroll], g[kUnroll];
 #pragma unroll
     for (int j = 0; j < kUnroll; ++j) {
       const long long v = v0 + j * stride;
-      if (v < nv) {
+      if (v < nv_main) {
         q[j] = __ldg(q4 + v);
-        g[j] = SYNTH ? sy.at4(v, P.p) : __ldg(g4 + v);
+        g[j] = SYNTH ? sy.at4(v) : __ldg(g4 + v);
       } else {
         q[j] = make_float4(0.f, 0.f, 0.f, 0.f);
         g[j] = q[j];
@@ -121,13 +124,20 @@ __global__ void __launch_bounds__(512) radius_kernel(const Params P) {
     }
 #pragma unroll
     for (int j = 0; j < kUnroll; ++j) {
-      // the ordering of |d| as unsigned bit patterns equals its ordering as floats, and puts
-      // inf and nan above every finite value, so a non-finite entry surfaces in R
       mx = max(mx, abs_bits(__fsub_rn(g[j].x, q[j].x)));
       mx = max(mx, abs_bits(__fsub_rn(g[j].y, q[j].y)));
       mx = max(mx, abs_bits(__fsub_rn(g[j].z, q[j].z)));
       mx = max(mx, abs_bits(__fsub_rn(g[j].w, q[j].w)));
     }
+  }
+  if (blockIdx.x == 0 && nv_main + threadIdx.x < nv) {
+    const long long v = nv_main + threadIdx.x;
+    const float4 q = __ldg(q4 + v);                      // padding of Q_prev and of a stored g is zero
+    const float4 g = SYNTH ? sy.at4_masked(v, P.p) : __ldg(g4 + v);
+    mx = max(mx, abs_bits(__fsub_rn(g.x, q.x)));
+    mx = max(mx, abs_bits(__fsub_rn(g.y, q.y)));
+    mx = max(mx, abs_bits(__fsub_rn(g.z, q.z)));
+    mx = max(mx, abs_bits(__fsub_rn(g.w, q.w)));
   }
   mx = __reduce_max_sync(0xffffffffu, mx);
   __shared__ uint32_t sh[32];
@@ -145,18 +155,21 @@ __global__ void __launch_bounds__(512) radius_kernel(const Params P) {
 // code packing: the 4 codes of coordinates 4v..4v+3 form one 4b-bit field at bit 4vb of the row
 // ------------------------------------------------------------------------------------------------
 template <int B>
-__device__ __forceinline__ void store_codes(uint32_t* row, long long v, uint32_t c0, uint32_t c1, uint32_t c2,
-                                            uint32_t c3, bool valid) {
+__device__ __forceinline__ void store_codes(uint32_t* row, long long v, uint32_t y0, uint32_t y1, uint32_t y2,
+                                            uint32_t y3, bool valid) {
+  // y_e = 0x4b000000 + code_e: the code sits in the low bits
   if (B == 16) {
-    if (valid) reinterpret_cast<uint2*>(row)[v] = make_uint2(c0 | (c1 << 16), c2 | (c3 << 16));
+    if (valid) reinterpret_cast<uint2*>(row)[v] = make_uint2(__byte_perm(y0, y1, 0x5410), __byte_perm(y2, y3, 0x5410));
   } else if (B == 8) {
-    if (valid) row[v] = c0 | (c1 << 8) | (c2 << 16) | (c3 << 24);
+    if (valid) row[v] = __byte_perm(__byte_perm(y0, y1, 0x0040), __byte_perm(y2, y3, 0x0040), 0x5410);
   } else if (B == 4) {
-    if (valid) reinterpret_cast<uint16_t*>(row)[v] = (uint16_t)(c0 | (c1 << 4) | (c2 << 8) | (c3 << 12));
+    if (valid)
+      reinterpret_cast<uint16_t*>(row)[v] =
+          (uint16_t)((y0 & 15u) | ((y1 & 15u) << 4) | ((y2 & 15u) << 8) | ((y3 & 15u) << 12));
   } else if (B == 2) {
-    if (valid) reinterpret_cast<uint8_t*>(row)[v] = (uint8_t)(c0 | (c1 << 2) | (c2 << 4) | (c3 << 6));
+    if (valid) reinterpret_cast<uint8_t*>(row)[v] = (uint8_t)((y0 & 3u) | ((y1 & 3u) << 2) | ((y2 & 3u) << 4) | ((y3 & 3u) << 6));
   } else {  // B == 1: two neighbouring lanes share a byte; v and the lane index have the same parity
-    uint32_t nib = valid ? (c0 | (c1 << 1) | (c2 << 2) | (c3 << 3)) : 0u;
+    uint32_t nib = valid ? ((y0 & 1u) | ((y1 & 1u) << 1) | ((y2 & 1u) << 2) | ((y3 & 1u) << 3)) : 0u;
     uint32_t hi = __shfl_down_sync(0xffffffffu, nib, 1);
     if (valid && !(v & 1)) reinterpret_cast<uint8_t*>(row)[v >> 1] = (uint8_t)(nib | (hi << 4));
   }
@@ -182,19 +195,35 @@ __device__ __forceinline__ void load_codes(const uint32_t* row, long long v, uin
   }
 }
 
-// One coordinate of Eq. (5)/(6).  Returns the code; updates the two fp64 sums.
-__device__ __forceinline__ uint32_t quantize_one(float g, float q, float R, float s, float levels, bool live,
-                                                 double& sdq, double& seps) {
-  if (!live) return 0u;
+// IEEE quotient x / s from y = RN(1/s): one product and two residual corrections (each residual is an
+// exact fused multiply-add).  The second correction starts from a faithful quotient, which makes the
+// result the correctly rounded one (Markstein's theorem); valid while nothing under- or overflows,
+// which the caller guarantees by using it only for 2^-60 <= s <= 2^60.
+__device__ __forceinline__ float div_by_reciprocal(float x, float s, float y) {
+  float q = __fmul_rn(x, y);
+  float r = __fmaf_rn(-s, q, x);
+  q = __fmaf_rn(r, y, q);
+  r = __fmaf_rn(-s, q, x);
+  return __fmaf_rn(r, y, q);
+}
+
+// One coordinate of Eq. (5)/(6).  Returns 2^23 + code as a float bit pattern (code in the low bits);
+// updates the two fp64 sums.  No clamp: |d| <= R bounds floor(t) by 2^b - 1 (t <= 2^b - 1/2 + rounding).
+template <bool FAST>
+__device__ __forceinline__ uint32_t quantize_one(float g, float q, float R, float s, float y, double& sdq,
+                                                 double& seps) {
   const float d = __fsub_rn(g, q);
-  const float t = __fadd_rn(__fdiv_rn(__fadd_rn(d, R), s), 0.5f);
-  const float f = fminf(fmaxf(floorf(t), 0.f), levels);
-  const float dq = __fsub_rn(__fmul_rn(s, f), R);
+  const float x = __fadd_rn(d, R);
+  const float u = FAST ? div_by_reciprocal(x, s, y) : __fdiv_rn(x, s);
+  const float t = __fadd_rn(u, 0.5f);
+  const float fl = __fadd_rd(t, 8388608.0f);        // 2^23 + floor(t): rounding down at unit spacing
+  const float f = __fsub_rn(fl, 8388608.0f);        // floor(t), exact
+  const float dq = __fmaf_rn(s, f, -R);             // Eq. (6) with one rounding
   const float qn = __fadd_rn(q, dq);
   const float e = __fsub_rn(g, qn);
-  sdq = fma((double)dq, (double)dq, sdq);   // the product of two fp32 values is exact in fp64
+  sdq = fma((double)dq, (double)dq, sdq);           // the product of two fp32 values is exact in fp64
   seps = fma((double)e, (double)e, seps);
-  return (uint32_t)f;
+  return __float_as_uint(fl);
 }
 
 // Skip rule (7a)+(7b), clocks, uploader list, counters: run by the last block of quantize_kernel.
@@ -274,6 +303,77 @@ __device__ void trigger_stage(const Params& P, int bpw) {
   }
 }
 
+// The per-worker sweep of quantize_kernel (R > 0).  FAST selects the reciprocal-based exact division.
+// Groups [0, nv_main) lie wholly inside the row and run without masks; the few groups after them are
+// handled by the first warp of the worker's first block with per-coordinate masks.  nv_main is even,
+// so the lane pairs of the 1-bit packing never straddle the two parts.
+template <bool SYNTH, int B, bool FAST>
+__device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned long long k, float R, float s,
+                                               double& sdq, double& seps) {
+  Synth sy;
+  if (SYNTH) sy.init(P, m, k + 1);
+  const float y = __fdiv_rn(1.0f, s);
+  const float4* __restrict__ q4 = reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps);
+  const float4* __restrict__ g4 = SYNTH ? nullptr : reinterpret_cast<const float4*>(P.g + (long long)m * P.ps);
+  uint32_t* row = P.codes + (long long)m * P.cw;
+  const long long nv = P.nv, p = P.p, nv_main = (p / 4) & ~1ll, stride = (long long)gridDim.x * blockDim.x;
+  // all lanes of a warp run the same number of trips (the 1-bit packing shuffles between lanes)
+  const long long first = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long warp_first = first - (threadIdx.x & 31);
+  for (long long base = 0; warp_first + base < nv_main; base += kUnroll * stride) {
+    float4 q[kUnroll], g[kUnroll];
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) {
+      const long long v = first + base + j * stride;
+      if (v < nv_main) {
+        q[j] = __ldg(q4 + v);
+        g[j] = SYNTH ? sy.at4(v) : __ldg(g4 + v);
+      } else {  // harmless operands: d = 0, code in range, nothing stored, nothing summed
+        q[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        g[j] = q[j];
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) {
+      const long long v = first + base + j * stride;
+      if (warp_first + base + j * stride >= nv_main) break;  // warp-uniform
+      const bool ok = v < nv_main;
+      double a = 0.0, c = 0.0;
+      const uint32_t y0 = quantize_one<FAST>(g[j].x, q[j].x, R, s, y, a, c);
+      const uint32_t y1 = quantize_one<FAST>(g[j].y, q[j].y, R, s, y, a, c);
+      const uint32_t y2 = quantize_one<FAST>(g[j].z, q[j].z, R, s, y, a, c);
+      const uint32_t y3 = quantize_one<FAST>(g[j].w, q[j].w, R, s, y, a, c);
+      if (ok) {
+        sdq += a;
+        seps += c;
+      }
+      store_codes<B>(row, v, y0, y1, y2, y3, ok);
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x < 32) {  // groups that may contain padding coordinates
+    const long long v = nv_main + threadIdx.x;
+    const bool ok = v < nv;
+    uint32_t yy[4] = {0x4b000000u, 0x4b000000u, 0x4b000000u, 0x4b000000u};
+    if (ok) {
+      const float4 q = __ldg(q4 + v);
+      const float4 g = SYNTH ? sy.at4_masked(v, p) : __ldg(g4 + v);
+      const float gg[4] = {g.x, g.y, g.z, g.w}, qq[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (4 * v + e < p) yy[e] = quantize_one<FAST>(gg[e], qq[e], R, s, y, sdq, seps);
+    }
+    store_codes<B>(row, v, yy[0], yy[1], yy[2], yy[3], ok);
+  }
+}
+
+// R = 0: every code is zero (and so are dQ and eps)
+template <int B>
+__device__ __forceinline__ void zero_codes(const Params& P, int m) {
+  uint32_t* row = P.codes + (long long)m * P.cw;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long w = (long long)blockIdx.x * blockDim.x + threadIdx.x; w < P.cw; w += stride) row[w] = 0u;
+}
+
 template <bool SYNTH, int B>
 __global__ void __launch_bounds__(512) quantize_kernel(const Params P) {
   __shared__ double sh[32];
@@ -286,46 +386,14 @@ __global__ void __launch_bounds__(512) quantize_kernel(const Params P) {
   const bool finite = Rb < 0x7f800000u;
   double sdq = 0.0, seps = 0.0;
   if (!frozen && finite) {
-    Synth sy;
-    if (SYNTH) sy.init(P, m, k + 1);
     const float levels = (float)((1u << B) - 1u);
     const float s = __fmul_rn(__fmul_rn(2.0f, __fdiv_rn(1.0f, levels)), R);
-    const bool live = R > 0.f;  // R = 0: codes, dQ and eps are all zero
-    const float4* __restrict__ q4 = reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps);
-    const float4* __restrict__ g4 = SYNTH ? nullptr : reinterpret_cast<const float4*>(P.g + (long long)m * P.ps);
-    uint32_t* row = P.codes + (long long)m * P.cw;
-    const long long nv = P.nv, stride = (long long)gridDim.x * blockDim.x, p = P.p;
-    // all lanes of a warp run the same number of trips (the 1-bit packing shuffles between lanes)
-    const long long first = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const long long warp_first = first - (threadIdx.x & 31);
-    for (long long base = 0; warp_first + base < nv; base += kUnroll * stride) {
-      float4 q[kUnroll], g[kUnroll];
-      bool ok[kUnroll];
-#pragma unroll
-      for (int j = 0; j < kUnroll; ++j) {
-        const long long v = first + base + j * stride;
-        ok[j] = v < nv;
-        if (ok[j]) {
-          q[j] = __ldg(q4 + v);
-          g[j] = SYNTH ? sy.at4(v, p) : __ldg(g4 + v);
-        } else {
-          q[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-          g[j] = q[j];
-        }
-      }
-#pragma unroll
-      for (int j = 0; j < kUnroll; ++j) {
-        const long long v = first + base + j * stride;
-        if (warp_first + base + j * stride >= nv) break;  // warp-uniform
-        const long long i = 4 * v;
-        const bool on = ok[j] && live;
-        const uint32_t c0 = quantize_one(g[j].x, q[j].x, R, s, levels, on && i < p, sdq, seps);
-        const uint32_t c1 = quantize_one(g[j].y, q[j].y, R, s, levels, on && i + 1 < p, sdq, seps);
-        const uint32_t c2 = quantize_one(g[j].z, q[j].z, R, s, levels, on && i + 2 < p, sdq, seps);
-        const uint32_t c3 = quantize_one(g[j].w, q[j].w, R, s, levels, on && i + 3 < p, sdq, seps);
-        store_codes<B>(row, v, c0, c1, c2, c3, ok[j]);
-      }
-    }
+    if (!(R > 0.f))
+      zero_codes<B>(P, m);
+    else if (s >= 0x1p-60f && s <= 0x1p60f)
+      quantize_sweep<SYNTH, B, true>(P, m, k, R, s, sdq, seps);
+    else
+      quantize_sweep<SYNTH, B, false>(P, m, k, R, s, sdq, seps);
   }
   const double tdq = block_sum(sdq, sh);
   const double teps = block_sum(seps, sh);
@@ -350,6 +418,9 @@ __global__ void __launch_bounds__(512) quantize_kernel(const Params P) {
 // lazy aggregate + theta step
 // ------------------------------------------------------------------------------------------------
 constexpr int kAggBatch = 4;  // uploaders whose loads are issued together
+
+// exact float of a code < 2^23 through the mantissa of 2^23
+__device__ __forceinline__ float code_to_float(uint32_t c) { return __uint_as_float(0x4b000000u | c) - 8388608.0f; }
 
 template <int B>
 __global__ void __launch_bounds__(512) aggregate_kernel(const Params P) {
@@ -392,10 +463,10 @@ __global__ void __launch_bounds__(512) aggregate_kernel(const Params P) {
           const int m = s_m[u0 + j];
           const float R = s_R[u0 + j], s = s_s[u0 + j];
           // the server's recovery of the innovation from the message: dQ = 2 tau R q - R
-          float d0 = __fsub_rn(__fmul_rn(s, (float)c[j][0]), R);
-          float d1 = __fsub_rn(__fmul_rn(s, (float)c[j][1]), R);
-          float d2 = __fsub_rn(__fmul_rn(s, (float)c[j][2]), R);
-          float d3 = __fsub_rn(__fmul_rn(s, (float)c[j][3]), R);
+          float d0 = __fmaf_rn(s, code_to_float(c[j][0]), -R);
+          float d1 = __fmaf_rn(s, code_to_float(c[j][1]), -R);
+          float d2 = __fmaf_rn(s, code_to_float(c[j][2]), -R);
+          float d3 = __fmaf_rn(s, code_to_float(c[j][3]), -R);
           if (tail) {  // padding coordinates carry no innovation
             if (i >= p) d0 = 0.f;
             if (i + 1 >= p) d1 = 0.f;

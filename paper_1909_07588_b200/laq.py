@@ -255,3 +255,4 @@ def from_workload(w, trace_capacity=0, stream=None, **overrides):
     for m in range(len(w.X)):
         ctx.load_shards(m, w.X[m], w.y[m])
     return ctx
+

@@ -117,15 +117,17 @@ def c1(seed=1, M=10, n_per=6000, F=784, C=10, iters=500):
                     L_smooth=L)
 
 
-def c2(seed=2, M=10, n_per=58101, iters=1000):
-    """Binary logistic regression, 54 features: 10 Gaussian columns, a 4-way and a 40-way one-hot group."""
+def c2(seed=2, M=10, n_per=58101, iters=1000, theta0_scale=0.0):
+    """Binary logistic regression, 54 features: 10 Gaussian columns, a 4-way and a 40-way one-hot group.
+    theta0_scale > 0 starts from a small random iterate instead of zero (at theta = 0 every residual is
+    +-1/2, so the gradient of a rarely active one-hot column can cancel to exactly zero)."""
     rng = np.random.default_rng(seed)
     n = M * n_per
     F = 54
     X = np.zeros((n, F), dtype=np.float32)
     X[:, :10] = rng.standard_normal((n, 10)).astype(np.float32)
     for start, width in ((10, 4), (14, 40)):
-        prob = 0.85 ** np.arange(width)      # skewed, but every category still occurs in a reduced-size test
+        prob = 0.93 ** np.arange(width)      # skewed, but every worker still sees every category at reduced size
         prob /= prob.sum()
         cat = rng.choice(width, size=n, p=prob)
         X[np.arange(n), start + cat] = 1.0
@@ -135,8 +137,9 @@ def c2(seed=2, M=10, n_per=58101, iters=1000):
     lam = 0.01
     L = lambda_max_gram(X64) / (4.0 * n) + lam
     Xs, ys = _split(X, y, M, n_per)
+    theta0 = (theta0_scale * rng.standard_normal(F)).astype(np.float32) if theta0_scale > 0 else None
     return Workload("c2_logreg54", MODEL_LOGREG_BIN, M, F, [n_per] * M, n_features=F, alpha=1.0 / L,
-                    lam=lam, b=8, D=10, tbar=100, iters=iters, seed=seed, X=Xs, y=ys, L_smooth=L)
+                    lam=lam, b=8, D=10, tbar=100, iters=iters, seed=seed, X=Xs, y=ys, L_smooth=L, theta0=theta0)
 
 
 def c3(seed=3, M=10, n_per=6000, F=784, H=200, C=10, iters=1000, bf16_ops=1):

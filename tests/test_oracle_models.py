@@ -167,13 +167,32 @@ def test_synthetic_stream_follows_its_written_definition():
         x ^= x >> np.uint32(13); x = np.uint32(x * np.uint32(0xc2b2ae35))
         x ^= x >> np.uint32(16)
         return x
-    seed, m, M, p, k, sigma, eta0 = (7 << 32) | 12345, 5, 16, 1000, 9, 0.1, 0.05
+    seed, m, M, p, k, sigma, eta0 = (7 << 32) | 12345, 5, 16, 1003, 9, 0.1, 0.05
+    nv = (p + 3) // 4
     with np.errstate(over="ignore"):
         key = fmix(np.uint32(seed & 0xffffffff) ^ fmix(np.uint32(seed >> 32) + np.uint32(0x9e3779b9) * np.uint32(m + 1)))
-        h = fmix(np.arange(p, dtype=np.uint32) ^ key)
-    b = [((h >> np.uint32(s)) & np.uint32(255)).astype(np.int32) for s in (0, 8, 16, 24)]
-    zi, wi = b[0] + b[1] + b[2] + b[3] - 510, b[0] - b[1] + b[2] - b[3]
+        h0 = fmix(np.arange(nv, dtype=np.uint32) ^ key)
+        h1 = np.uint32(h0 * np.uint32(0x9e3779b1))
+        h1 ^= h1 >> np.uint32(15)
+    z = np.zeros((nv, 4), np.int32)
+    for j, h in enumerate((h0, h1)):
+        b = [((h >> np.uint32(s)) & np.uint32(255)).astype(np.int32) for s in (0, 8, 16, 24)]
+        z[:, 2 * j] = b[0] + b[1] + b[2] + b[3] - 510
+        z[:, 2 * j + 1] = b[0] - b[1] + b[2] - b[3]
     cz = np.float32(np.float64(np.float32(sigma)) / np.sqrt(21845.0))
     drift = np.float32(k) * np.float32(np.float64(np.float32(eta0)) * (m + 1) / M)
-    ref = zi.astype(np.float32) * cz + drift * (wi.astype(np.float32) * cz)
+    partner = z[:, [2, 3, 0, 1]]
+    # small integers times an fp32 factor plus a small integer: exact in fp64, so one rounding = fma
+    a = (np.float64(drift) * partner.astype(np.float64) + z.astype(np.float64)).astype(np.float32)
+    ref = (a * cz).reshape(-1)[:p]
     np.testing.assert_array_equal(oracle.synth_gradient(seed, m, M, p, k, sigma, eta0), ref)
+
+
+def test_synthetic_stream_coordinates_are_uncorrelated():
+    g = oracle.synth_gradient(11, 0, 4, 400_000, 0, 1.0, 0.0).astype(np.float64).reshape(-1, 4)
+    c = np.corrcoef(g.T)
+    assert np.max(np.abs(c - np.eye(4))) < 0.01            # within a group of four
+    flat = g.reshape(-1)
+    for lag in (1, 2, 3, 4, 5, 8, 64):
+        assert abs(np.corrcoef(flat[:-lag], flat[lag:])[0, 1]) < 0.01
+    assert np.allclose(g.std(0), 1.0, rtol=0.01) and np.all(np.abs(g.mean(0)) < 0.01)
