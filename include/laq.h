@@ -188,6 +188,29 @@ laq_status laq_tune(laq_ctx* ctx, const char* key, int32_t value);
 laq_status laq_set_profiling(laq_ctx* ctx, int32_t enabled);
 laq_status laq_kernel_times(laq_ctx* ctx, double* ms, int64_t* launches);
 
+/* (The paper has no counterpart for this entry point; it exists for hosts that must not allocate.)
+ * The quantizer of ONE worker -- radius, packed codes and the two squared norms, exactly as steps 2-3 of
+ * laq_step compute them -- without a context and without any allocation: no cudaMalloc/cudaFree, no
+ * workspace.  It is meant for callers that cannot allocate device memory themselves: a host program that
+ * has given the whole GPU to its own memory pool, or a latency-critical loop in which allocation calls are
+ * banned because they synchronise the device.  The kernels' reduction scratch (33 024 bytes: running
+ * maximum, per-block partial sums, a ticket) is a __device__ array inside the library; every GPU that
+ * loads the library holds it until the process exits.
+ *   d_g, d_qprev : DEVICE, [p] fp32, the gradient and the stored quantized copy (inputs, unchanged)
+ *   d_codes      : DEVICE, [ceil(p b / 32)] words, the code stream (output)
+ *   d_R          : DEVICE, one float, the radius (output)
+ *   d_norms      : DEVICE, two doubles, ||dQ||^2 and ||eps||^2 (output)
+ *   errbuf       : HOST, optional buffer for an error text (errbuf_len bytes), may be NULL
+ * Limits: b in {1, 2, 4, 8, 16}; 1 <= p <= 2^31, larger p is rejected with LAQ_EINVAL and a message.
+ * The call is asynchronous on cuda_stream.  All calls on one GPU share the scratch, which still holds the
+ * previous call's values (the call clears what must start at zero): calls whose kernels overlap on the same
+ * GPU race with each other, so keep them on one stream or otherwise serialised.  The first call on each
+ * device looks up the scratch's device address (and loads the module); make that call during start-up,
+ * before any stream capture.  A non-finite input yields a non-finite *d_R, zero norms and untouched codes. */
+laq_status laq_quantize_worker_static(const float* d_g, const float* d_qprev, int64_t p, int32_t b,
+                                      uint32_t* d_codes, float* d_R, double* d_norms, void* cuda_stream,
+                                      char* errbuf, size_t errbuf_len);
+
 /* Text of the last failure on this context ("" if none).  Valid until the next call on ctx. */
 const char* laq_last_error(const laq_ctx* ctx);
 

@@ -17,7 +17,7 @@ MODEL_LOGREG_BIN, MODEL_SOFTMAX, MODEL_MLP2, MODEL_SYNTH, MODEL_EXTERNAL = range
 FLAG_TRIGGER_OFF = 2
 
 EXPORTS = ["laq_workspace_bytes", "laq_init", "laq_load_shards", "laq_set_gradients", "laq_step", "laq_sync",
-           "laq_get_state", "laq_get_worker", "laq_set_state", "laq_kernel_launches", "laq_tune", "laq_set_profiling", "laq_kernel_times", "laq_last_error", "laq_destroy"]
+           "laq_get_state", "laq_get_worker", "laq_set_state", "laq_kernel_launches", "laq_tune", "laq_set_profiling", "laq_kernel_times", "laq_quantize_worker_static", "laq_last_error", "laq_destroy"]
 
 
 class LaqError(RuntimeError):
@@ -74,6 +74,8 @@ def load_library():
     L.laq_tune.argtypes = [C.c_void_p, C.c_char_p, C.c_int32]
     L.laq_set_profiling.argtypes = [C.c_void_p, C.c_int32]
     L.laq_kernel_times.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+    L.laq_quantize_worker_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p,
+                                             C.c_void_p, C.c_void_p, C.c_char_p, C.c_size_t]
     L.laq_last_error.argtypes = [C.c_void_p]
     L.laq_last_error.restype = C.c_char_p
     L.laq_destroy.argtypes = [C.c_void_p]
@@ -256,3 +258,25 @@ def from_workload(w, trace_capacity=0, stream=None, **overrides):
         ctx.load_shards(m, w.X[m], w.y[m])
     return ctx
 
+
+def quantize_worker_static(g, qprev, b, codes, R, norms, stream=None):
+    """laq_quantize_worker_static: one worker's quantizer for hosts that must not allocate device memory.
+
+    Every argument is a torch CUDA tensor that the caller already owns: g, qprev [p] float32 (inputs),
+    codes [ceil(p*b/32)] int32 or uint32 storage, R [1] float32, norms [2] float64 (outputs).  The kernels'
+    scratch is a fixed array inside the library, shared by all calls on the GPU, so calls must not overlap.
+    """
+    import torch
+    L = load_library()
+    assert g.is_cuda and qprev.is_cuda and codes.is_cuda and R.is_cuda and norms.is_cuda
+    assert g.dtype == torch.float32 and qprev.dtype == torch.float32 and R.dtype == torch.float32
+    assert norms.dtype == torch.float64 and norms.numel() >= 2 and codes.element_size() == 4
+    p = g.numel()
+    assert qprev.numel() == p and codes.numel() >= (p * b + 31) // 32
+    st = stream if stream is not None else torch.cuda.current_stream(g.device)
+    err = C.create_string_buffer(256)
+    rc = L.laq_quantize_worker_static(C.c_void_p(g.data_ptr()), C.c_void_p(qprev.data_ptr()), p, b,
+                                      C.c_void_p(codes.data_ptr()), C.c_void_p(R.data_ptr()),
+                                      C.c_void_p(norms.data_ptr()), C.c_void_p(st.cuda_stream), err, 256)
+    if rc != LAQ_OK:
+        raise LaqError(rc, err.value.decode())

@@ -1,0 +1,78 @@
+"""laq_quantize_worker_static -- the entry point for hosts that may not allocate device memory.
+
+Some users of this library run it from a process whose GPU memory is entirely owned by their own pool, or
+from a loop where allocation calls are forbidden because they stall the device.  For them the library offers
+one quantizer call whose scratch is a fixed array baked into the library instead of caller- or
+library-allocated memory.  This test calls it through the C ABI twice in a row (the scratch is shared and
+keeps the previous call's contents, so the second call checks that stale values are cleared) and compares
+codes, radius and norms with what the regular entry point (laq_step on a one-worker context) produces.
+"""
+import ctypes as C
+
+import numpy as np
+import pytest
+
+from paper_1909_07588_b200 import laq
+
+pytestmark = pytest.mark.gpu
+
+NORM_RTOL = 1e-5     # the tolerance the other GPU tests use for squared norms
+
+
+def _regular_entry_point(g, qprev, b):
+    """Steps 2-3 for one worker through laq_step: returns codes, R, ||dQ||^2, ||eps||^2."""
+    p = g.size
+    ctx = laq.Laq(model=laq.MODEL_EXTERNAL, M=1, p=p, alpha=0.1, b=b, D=1, xi=[0.0], tbar=10, trace_capacity=1)
+    ctx.set_state(qprev=qprev.reshape(1, p))
+    ctx.set_gradients(g.reshape(1, p))
+    tr = ctx.step(1, trace=True)
+    codes = ctx.get_worker(0, qprev=False)["codes"]
+    ctx.close()
+    return codes, tr["R"][0, 0], tr["n_dq"][0, 0], tr["n_eps"][0, 0]
+
+
+def test_static_scratch_quantizer_matches_regular_entry_point_twice_in_a_row():
+    import torch
+    rng = np.random.default_rng(42)
+    cases = [(70001, 8, 1.0), (5003, 4, 1e-3), (600_000, 2, 30.0)]      # ragged sizes, different b and scales
+    # everything the calls touch is allocated up front; the calls themselves allocate nothing
+    bufs = []
+    for p, b, scale in cases:
+        g = (rng.standard_normal(p) * scale).astype(np.float32)
+        q = (rng.standard_normal(p) * scale * 0.5).astype(np.float32)
+        W = (p * b + 31) // 32
+        bufs.append(dict(p=p, b=b, g=g, q=q, dg=torch.from_numpy(g).cuda(), dq=torch.from_numpy(q).cuda(),
+                         codes=torch.full((W,), -1, dtype=torch.int32, device="cuda"),
+                         R=torch.full((1,), -1.0, dtype=torch.float32, device="cuda"),
+                         norms=torch.full((2,), -1.0, dtype=torch.float64, device="cuda")))
+    torch.cuda.synchronize()
+    before = torch.cuda.memory_allocated()
+    for c in bufs:                                                       # calls back to back, no sync between
+        laq.quantize_worker_static(c["dg"], c["dq"], c["b"], c["codes"], c["R"], c["norms"])
+    torch.cuda.synchronize()
+    assert torch.cuda.memory_allocated() == before
+    for c in bufs:
+        codes_ref, R_ref, ndq_ref, neps_ref = _regular_entry_point(c["g"], c["q"], c["b"])
+        np.testing.assert_array_equal(c["codes"].cpu().numpy().view(np.uint32), codes_ref)
+        assert c["R"].item() == R_ref
+        n = c["norms"].cpu().numpy()
+        assert n[0] == pytest.approx(ndq_ref, rel=NORM_RTOL)
+        assert n[1] == pytest.approx(neps_ref, rel=NORM_RTOL)
+
+
+def test_static_scratch_quantizer_rejects_oversized_and_bad_arguments():
+    import torch
+    L = laq.load_library()
+    x = torch.zeros(16, dtype=torch.float32, device="cuda")
+    codes = torch.zeros(16, dtype=torch.int32, device="cuda")
+    R = torch.zeros(1, dtype=torch.float32, device="cuda")
+    norms = torch.zeros(2, dtype=torch.float64, device="cuda")
+    err = C.create_string_buffer(256)
+    args = lambda p, b: (C.c_void_p(x.data_ptr()), C.c_void_p(x.data_ptr()), p, b, C.c_void_p(codes.data_ptr()),
+                         C.c_void_p(R.data_ptr()), C.c_void_p(norms.data_ptr()), None, err, 256)
+    assert L.laq_quantize_worker_static(*args((1 << 31) + 1, 8)) == laq.LAQ_EINVAL
+    assert b"limit" in err.value
+    assert L.laq_quantize_worker_static(*args(16, 3)) == laq.LAQ_EINVAL
+    assert L.laq_quantize_worker_static(*args(0, 8)) == laq.LAQ_EINVAL
+    assert L.laq_quantize_worker_static(None, None, 16, 8, None, None, None, None, err, 256) == laq.LAQ_EINVAL
+    torch.cuda.synchronize()
