@@ -23,9 +23,9 @@
  *     (laq_step with a trace, laq_get_state, laq_sync) as LAQ_ENONFINITE.
  *   - Floating point: theta, gradients and quantizer state are fp32; each quantizer operation is one
  *     IEEE round-to-nearest operation in the order  d = g - Q_prev ; R = max|d| ; s = (2 tau) R ;
- *     t = (d + R)/s + 1/2 ; q = floor t ; dQ = fma(s, q, -R) (Eq. (6) with a single rounding) ;
- *     Q_new = Q_prev + dQ ; eps = g - Q_new, with no other fused multiply-add; squared norms are fp64
- *     sums of exact fp32 products; the skip rule is evaluated in fp64.
+ *     t = (d + R)/s + 1/2 (IEEE division) ; q = floor t ; dQ = s q - R (multiply, then subtract) ;
+ *     Q_new = Q_prev + dQ ; eps = g - Q_new, with no fused multiply-add; squared norms are fp64 sums of
+ *     exact fp32 products; the skip rule is evaluated in fp64.
  *   - Code stream of worker m (the paper's b p-bit part of the upload message): code i occupies bits
  *     [(i b) mod 32, +b) of 32-bit word floor(i b / 32), least significant first.
  *   - Readings where the paper is silent: initial Q_m = 0, ||eps_hat_m||^2 = 0, grad^0 = 0, the D stored
@@ -80,7 +80,7 @@ enum {
 typedef struct {
   int32_t model;            /* laq_model */
   int32_t M;                /* number of workers, 1..1024 */
-  int64_t p;                /* dimension of theta (checked against the model shape) */
+  int64_t p;                /* dimension of theta, 1..2^32-1 (checked against the model shape) */
   const int64_t* N;         /* HOST, length M: samples per worker {N_m}; ignored for SYNTH / EXTERNAL */
   int32_t n_features;       /* F */
   int32_t n_classes;        /* C (SOFTMAX: 2..16, MLP2) */

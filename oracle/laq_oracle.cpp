@@ -84,7 +84,7 @@ float round_bf16(float x) {
 //        n_dq = ||dq||^2, n_eps = ||eps||^2  (fp64 sums, index order)
 // Operation order (each one IEEE operation in T):
 //   d = g - qp ; R = max |d| ; tau = 1/(2^b-1) ; s = (2 tau) R ; t = (d + R)/s + 1/2 ;
-//   q = clamp(floor(t), 0, 2^b-1) ; dq = fma(s, q, -R) (one rounding) ; qnew = qp + dq ; eps = g - qnew.
+//   q = clamp(floor(t), 0, 2^b-1) ; dq = s q - R ; qnew = qp + dq ; eps = g - qnew.
 // ---------------------------------------------------------------------------------------------
 template <typename T>
 void quantize(const T* g, const T* qp, i64 p, int b, T* R_out, int32_t* q, T* dq, T* qnew, T* eps,
@@ -111,7 +111,7 @@ void quantize(const T* g, const T* qp, i64 p, int b, T* R_out, int32_t* q, T* dq
       if (f < (T)0) f = 0;
       if (f > levels) f = levels;
       qi = (int32_t)f;
-      dqi = std::fma(s, (T)qi, -R);  // Eq. (6), one rounding
+      dqi = s * (T)qi - R;  // Eq. (6): multiply, then subtract
     }
     T qn = qp[i] + dqi;
     T e = g[i] - qn;
@@ -133,7 +133,7 @@ void decode(T R, const int32_t* q, const T* qp, i64 p, int b, T* qnew, T* dq) {
   const T tau = (T)1 / levels;
   const T s = ((T)2 * tau) * R;
   for (i64 i = 0; i < p; ++i) {
-    T d = (R > (T)0) ? std::fma(s, (T)q[i], -R) : (T)0;
+    T d = (R > (T)0) ? (s * (T)q[i] - R) : (T)0;
     if (dq) dq[i] = d;
     qnew[i] = qp[i] + d;
   }

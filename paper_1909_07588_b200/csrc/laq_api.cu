@@ -62,7 +62,7 @@ const char* check_config(const laq_config* c) {
   if (!c) return "config is null";
   if (c->model < 0 || c->model > LAQ_MODEL_EXTERNAL) return "unknown model";
   if (c->M < 1 || c->M > kMaxWorkers) return "M must be in 1..1024";
-  if (c->p < 1) return "p must be positive";
+  if (c->p < 1 || c->p >= (1ll << 32)) return "p must be in 1..2^32-1";
   if (!valid_b(c->b)) return "b must be 1, 2, 4, 8 or 16";
   if (c->D < 1 || c->D > kMaxD) return "D must be in 1..64";
   if (!c->xi) return "xi is null";
@@ -89,7 +89,6 @@ const char* check_config(const laq_config* c) {
     if (e) return e;
   }
   if (c->model == LAQ_MODEL_SYNTH) {
-    if (c->p >= (1ll << 32)) return "SYNTH requires p < 2^32";
     if (!std::isfinite(c->synth_sigma) || !std::isfinite(c->synth_eta0)) return "synth parameters must be finite";
   }
   return nullptr;
@@ -559,7 +558,7 @@ laq_status laq_tune(laq_ctx* ctx, const char* key, int32_t value) {
   const std::string k(key);
   auto pow2_threads = [](int v) { return v == 64 || v == 128 || v == 256 || v == 512; };
   if (k == "sweep_threads" && pow2_threads(value)) ctx->ls.sweep_threads = value;
-  else if (k == "sweep_blocks_per_sm" && value >= 1 && value <= 32) ctx->ls.sweep_blocks_per_sm = value;
+  else if (k == "sweep_blocks_per_sm" && value >= 1 && value <= 128) ctx->ls.sweep_blocks_per_sm = value;
   else if (k == "agg_threads" && pow2_threads(value)) ctx->ls.agg_threads = value;
   else if (k == "agg_blocks_per_sm" && value >= 1 && value <= 32) ctx->ls.agg_blocks_per_sm = value;
   else if (k == "grad_blocks_per_worker" && value >= 1 && value <= ctx->gbpw_cap) ctx->gbpw = value;

@@ -79,10 +79,10 @@ struct Params {
 };
 
 struct LaunchShape {
-  int sweep_threads = 256;
-  int sweep_blocks_per_sm = 8;
+  int sweep_threads = 128;
+  int sweep_blocks_per_sm = 64;    // many small blocks: the last partial wave costs a few percent at most
   int agg_threads = 256;
-  int agg_blocks_per_sm = 8;
+  int agg_blocks_per_sm = 32;
   int grad_blocks_per_worker = 0;  // 0 = automatic
 };
 

@@ -107,7 +107,7 @@ __global__ void __launch_bounds__(kThreads) static_quantize_kernel(const float* 
         const float d = __fsub_rn(gi, qi);
         const float t = __fadd_rn(__fdiv_rn(__fadd_rn(d, R), s), 0.5f);
         const float f = fminf(fmaxf(floorf(t), 0.f), levels);
-        const float dq = __fmaf_rn(s, f, -R);
+        const float dq = __fsub_rn(__fmul_rn(s, f), R);
         const float e_ = __fsub_rn(gi, __fadd_rn(qi, dq));
         sdq = fma((double)dq, (double)dq, sdq);
         seps = fma((double)e_, (double)e_, seps);

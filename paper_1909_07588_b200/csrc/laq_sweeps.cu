@@ -38,8 +38,8 @@ struct Synth {
     drift = __fmul_rn((float)k_iter, eta_m);
   }
   // coordinates 4v .. 4v+3
-  __device__ __forceinline__ float4 at4(long long v) const {
-    const uint32_t h0 = fmix32((uint32_t)v ^ key);
+  __device__ __forceinline__ float4 at4(uint32_t v) const {
+    const uint32_t h0 = fmix32(v ^ key);
     uint32_t h1 = h0 * 0x9e3779b1u;
     h1 ^= h1 >> 15;
     const int e0 = (int)__dp4a(h0, 0x00010001u, 0u), o0 = (int)__dp4a(h0, 0x01000100u, 0u);  // b0+b2, b1+b3
@@ -57,9 +57,9 @@ struct Synth {
     return r;
   }
   // the same with zeros at coordinates >= p (last group of a row)
-  __device__ __forceinline__ float4 at4_masked(long long v, long long p) const {
+  __device__ __forceinline__ float4 at4_masked(uint32_t v, long long p) const {
     float4 r = at4(v);
-    const long long i = 4 * v;
+    const long long i = 4ll * v;
     if (i >= p) r.x = 0.f;
     if (i + 1 >= p) r.y = 0.f;
     if (i + 2 >= p) r.z = 0.f;
@@ -104,23 +104,18 @@ __global__ void __launch_bounds__(512) radius_kernel(const Params P) {
   const float4* __restrict__ q4 = reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps);
   const float4* __restrict__ g4 = SYNTH ? nullptr : reinterpret_cast<const float4*>(P.g + (long long)m * P.ps);
   // groups [0, nv_main) lie wholly inside the row; the (at most five) groups after them may contain
-  // padding coordinates and take the masked path
-  const long long nv = P.nv, nv_main = (P.p / 4) & ~1ll, stride = (long long)gridDim.x * blockDim.x;
+  // padding coordinates and take the masked path.  p < 2^32, so group indices fit 32 bits.
+  const uint32_t nv = (uint32_t)P.nv, nv_main = (uint32_t)((P.p / 4) & ~1ll), stride = gridDim.x * blockDim.x;
   uint32_t mx = 0;
   // the ordering of |d| as unsigned bit patterns equals its ordering as floats, and puts inf and nan
   // above every finite value, so a non-finite entry surfaces in R
-  for (long long v0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; v0 < nv_main; v0 += kUnroll * stride) {
+  uint32_t v = blockIdx.x * blockDim.x + threadIdx.x;
+  for (; (unsigned long long)v + (kUnroll - 1) * (unsigned long long)stride < nv_main; v += kUnroll * stride) {
     float4 q[kUnroll], g[kUnroll];
 #pragma unroll
     for (int j = 0; j < kUnroll; ++j) {
-      const long long v = v0 + j * stride;
-      if (v < nv_main) {
-        q[j] = __ldg(q4 + v);
-        g[j] = SYNTH ? sy.at4(v) : __ldg(g4 + v);
-      } else {
-        q[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-        g[j] = q[j];
-      }
+      q[j] = __ldg(q4 + (v + j * stride));
+      g[j] = SYNTH ? sy.at4(v + j * stride) : __ldg(g4 + (v + j * stride));
     }
 #pragma unroll
     for (int j = 0; j < kUnroll; ++j) {
@@ -130,8 +125,16 @@ __global__ void __launch_bounds__(512) radius_kernel(const Params P) {
       mx = max(mx, abs_bits(__fsub_rn(g[j].w, q[j].w)));
     }
   }
+  for (; v < nv_main; v += stride) {
+    const float4 q = __ldg(q4 + v);
+    const float4 g = SYNTH ? sy.at4(v) : __ldg(g4 + v);
+    mx = max(mx, abs_bits(__fsub_rn(g.x, q.x)));
+    mx = max(mx, abs_bits(__fsub_rn(g.y, q.y)));
+    mx = max(mx, abs_bits(__fsub_rn(g.z, q.z)));
+    mx = max(mx, abs_bits(__fsub_rn(g.w, q.w)));
+  }
   if (blockIdx.x == 0 && nv_main + threadIdx.x < nv) {
-    const long long v = nv_main + threadIdx.x;
+    const uint32_t v = nv_main + threadIdx.x;
     const float4 q = __ldg(q4 + v);                      // padding of Q_prev and of a stored g is zero
     const float4 g = SYNTH ? sy.at4_masked(v, P.p) : __ldg(g4 + v);
     mx = max(mx, abs_bits(__fsub_rn(g.x, q.x)));
@@ -155,7 +158,7 @@ __global__ void __launch_bounds__(512) radius_kernel(const Params P) {
 // code packing: the 4 codes of coordinates 4v..4v+3 form one 4b-bit field at bit 4vb of the row
 // ------------------------------------------------------------------------------------------------
 template <int B>
-__device__ __forceinline__ void store_codes(uint32_t* row, long long v, uint32_t y0, uint32_t y1, uint32_t y2,
+__device__ __forceinline__ void store_codes(uint32_t* row, uint32_t v, uint32_t y0, uint32_t y1, uint32_t y2,
                                             uint32_t y3, bool valid) {
   // y_e = 0x4b000000 + code_e: the code sits in the low bits
   if (B == 16) {
@@ -218,7 +221,7 @@ __device__ __forceinline__ uint32_t quantize_one(float g, float q, float R, floa
   const float t = __fadd_rn(u, 0.5f);
   const float fl = __fadd_rd(t, 8388608.0f);        // 2^23 + floor(t): rounding down at unit spacing
   const float f = __fsub_rn(fl, 8388608.0f);        // floor(t), exact
-  const float dq = __fmaf_rn(s, f, -R);             // Eq. (6) with one rounding
+  const float dq = __fsub_rn(__fmul_rn(s, f), R);   // Eq. (6): multiply, then subtract
   const float qn = __fadd_rn(q, dq);
   const float e = __fsub_rn(g, qn);
   sdq = fma((double)dq, (double)dq, sdq);           // the product of two fp32 values is exact in fp64
@@ -316,42 +319,53 @@ __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned 
   const float4* __restrict__ q4 = reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps);
   const float4* __restrict__ g4 = SYNTH ? nullptr : reinterpret_cast<const float4*>(P.g + (long long)m * P.ps);
   uint32_t* row = P.codes + (long long)m * P.cw;
-  const long long nv = P.nv, p = P.p, nv_main = (p / 4) & ~1ll, stride = (long long)gridDim.x * blockDim.x;
-  // all lanes of a warp run the same number of trips (the 1-bit packing shuffles between lanes)
-  const long long first = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const long long warp_first = first - (threadIdx.x & 31);
-  for (long long base = 0; warp_first + base < nv_main; base += kUnroll * stride) {
+  const long long p = P.p;
+  const uint32_t nv = (uint32_t)P.nv, nv_main = (uint32_t)((p / 4) & ~1ll), stride = gridDim.x * blockDim.x;
+  const uint32_t lane = threadIdx.x & 31;
+  uint32_t v = blockIdx.x * blockDim.x + threadIdx.x;
+  double adq[4] = {0.0, 0.0, 0.0, 0.0}, aeps[4] = {0.0, 0.0, 0.0, 0.0};
+  // hot loop: every group of every lane of the warp is valid, no predicates
+  for (; (unsigned long long)(v - lane + 31) + (kUnroll - 1) * (unsigned long long)stride < nv_main;
+       v += kUnroll * stride) {
     float4 q[kUnroll], g[kUnroll];
 #pragma unroll
     for (int j = 0; j < kUnroll; ++j) {
-      const long long v = first + base + j * stride;
-      if (v < nv_main) {
-        q[j] = __ldg(q4 + v);
-        g[j] = SYNTH ? sy.at4(v) : __ldg(g4 + v);
-      } else {  // harmless operands: d = 0, code in range, nothing stored, nothing summed
-        q[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-        g[j] = q[j];
-      }
+      q[j] = __ldg(q4 + (v + j * stride));
+      g[j] = SYNTH ? sy.at4(v + j * stride) : __ldg(g4 + (v + j * stride));
     }
 #pragma unroll
-    for (int j = 0; j < kUnroll; ++j) {
-      const long long v = first + base + j * stride;
-      if (warp_first + base + j * stride >= nv_main) break;  // warp-uniform
-      const bool ok = v < nv_main;
-      double a = 0.0, c = 0.0;
-      const uint32_t y0 = quantize_one<FAST>(g[j].x, q[j].x, R, s, y, a, c);
-      const uint32_t y1 = quantize_one<FAST>(g[j].y, q[j].y, R, s, y, a, c);
-      const uint32_t y2 = quantize_one<FAST>(g[j].z, q[j].z, R, s, y, a, c);
-      const uint32_t y3 = quantize_one<FAST>(g[j].w, q[j].w, R, s, y, a, c);
-      if (ok) {
-        sdq += a;
-        seps += c;
-      }
-      store_codes<B>(row, v, y0, y1, y2, y3, ok);
+    for (int j = 0; j < kUnroll; ++j) {  // four independent accumulation chains per sum
+      const uint32_t y0 = quantize_one<FAST>(g[j].x, q[j].x, R, s, y, adq[0], aeps[0]);
+      const uint32_t y1 = quantize_one<FAST>(g[j].y, q[j].y, R, s, y, adq[1], aeps[1]);
+      const uint32_t y2 = quantize_one<FAST>(g[j].z, q[j].z, R, s, y, adq[2], aeps[2]);
+      const uint32_t y3 = quantize_one<FAST>(g[j].w, q[j].w, R, s, y, adq[3], aeps[3]);
+      store_codes<B>(row, v + j * stride, y0, y1, y2, y3, true);
     }
   }
+  sdq += (adq[0] + adq[1]) + (adq[2] + adq[3]);
+  seps += (aeps[0] + aeps[1]) + (aeps[2] + aeps[3]);
+  // remainder of the main part: all lanes of a warp run the same number of trips (the 1-bit packing
+  // shuffles between lanes), invalid lanes compute on harmless operands and store nothing
+  for (; v - lane < nv_main; v += stride) {
+    const bool ok = v < nv_main;
+    float4 q = make_float4(0.f, 0.f, 0.f, 0.f), g = q;
+    if (ok) {
+      q = __ldg(q4 + v);
+      g = SYNTH ? sy.at4(v) : __ldg(g4 + v);
+    }
+    double a = 0.0, c = 0.0;
+    const uint32_t y0 = quantize_one<FAST>(g.x, q.x, R, s, y, a, c);
+    const uint32_t y1 = quantize_one<FAST>(g.y, q.y, R, s, y, a, c);
+    const uint32_t y2 = quantize_one<FAST>(g.z, q.z, R, s, y, a, c);
+    const uint32_t y3 = quantize_one<FAST>(g.w, q.w, R, s, y, a, c);
+    if (ok) {
+      sdq += a;
+      seps += c;
+    }
+    store_codes<B>(row, v, y0, y1, y2, y3, ok);
+  }
   if (blockIdx.x == 0 && threadIdx.x < 32) {  // groups that may contain padding coordinates
-    const long long v = nv_main + threadIdx.x;
+    const uint32_t v = nv_main + threadIdx.x;
     const bool ok = v < nv;
     uint32_t yy[4] = {0x4b000000u, 0x4b000000u, 0x4b000000u, 0x4b000000u};
     if (ok) {
@@ -360,7 +374,7 @@ __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned 
       const float gg[4] = {g.x, g.y, g.z, g.w}, qq[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
       for (int e = 0; e < 4; ++e)
-        if (4 * v + e < p) yy[e] = quantize_one<FAST>(gg[e], qq[e], R, s, y, sdq, seps);
+        if (4ll * v + e < p) yy[e] = quantize_one<FAST>(gg[e], qq[e], R, s, y, sdq, seps);
     }
     store_codes<B>(row, v, yy[0], yy[1], yy[2], yy[3], ok);
   }
@@ -463,10 +477,10 @@ __global__ void __launch_bounds__(512) aggregate_kernel(const Params P) {
           const int m = s_m[u0 + j];
           const float R = s_R[u0 + j], s = s_s[u0 + j];
           // the server's recovery of the innovation from the message: dQ = 2 tau R q - R
-          float d0 = __fmaf_rn(s, code_to_float(c[j][0]), -R);
-          float d1 = __fmaf_rn(s, code_to_float(c[j][1]), -R);
-          float d2 = __fmaf_rn(s, code_to_float(c[j][2]), -R);
-          float d3 = __fmaf_rn(s, code_to_float(c[j][3]), -R);
+          float d0 = __fsub_rn(__fmul_rn(s, code_to_float(c[j][0])), R);
+          float d1 = __fsub_rn(__fmul_rn(s, code_to_float(c[j][1])), R);
+          float d2 = __fsub_rn(__fmul_rn(s, code_to_float(c[j][2])), R);
+          float d3 = __fsub_rn(__fmul_rn(s, code_to_float(c[j][3])), R);
           if (tail) {  // padding coordinates carry no innovation
             if (i >= p) d0 = 0.f;
             if (i + 1 >= p) d1 = 0.f;
