@@ -319,6 +319,7 @@ laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, siz
     LAQ_CUDA(ctx, cudaMemcpyAsync(ws + pl.Ndev, ctx->N.data(), 8 * (size_t)c.M, cudaMemcpyHostToDevice, ctx->st));
     if (c.model == LAQ_MODEL_MLP2) {
       laq_status s = mlp_setup(ctx->mlp, P, ws + pl.mlp, ctx->st);
+      if (s == LAQ_OK) s = mlp_set_row_offsets(ctx->mlp, (const long long*)ctx->N.data(), c.M, ctx->st);
       if (s != LAQ_OK) return fail(ctx, s, "network scratch set-up failed");
     }
   }
@@ -345,7 +346,9 @@ laq_status laq_load_shards(laq_ctx* ctx, int32_t m, const float* X, const int32_
   LAQ_CUDA(ctx, cudaMemcpyAsync((void*)ctx->Xptr[m], X, (size_t)N_m * ctx->cfg.n_features * 4, kind, ctx->st));
   LAQ_CUDA(ctx, cudaMemcpyAsync((void*)ctx->yptr[m], y, (size_t)N_m * 4, kind, ctx->st));
   if (ctx->cfg.model == LAQ_MODEL_MLP2) {
-    ctx->launches += mlp_convert_shard(ctx->mlp, ctx->P, m, ctx->Xptr[m], N_m, ctx->st);
+    long long row_offset = 0;
+    for (int i = 0; i < m; ++i) row_offset += ctx->N[i];
+    ctx->launches += mlp_convert_shard(ctx->mlp, ctx->P, m, ctx->Xptr[m], N_m, row_offset, ctx->st);
   }
   LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));  // the caller may reuse its buffers on return
   ctx->shard_loaded[m] = 1;
@@ -397,7 +400,7 @@ laq_status laq_step(laq_ctx* ctx, int32_t n_iters, const laq_trace* trace) {
         ctx->launches += launch_grad_finalize(P, ctx->gbpw, &P.sc->theta_sq, ctx->st);
         break;
       case LAQ_MODEL_MLP2:
-        ctx->launches += mlp_launch_gradients(ctx->mlp, P, ctx->st);
+        ctx->launches += mlp_launch_gradients(ctx->mlp, P, &P.sc->theta_sq, ctx->st);
         break;
       default: break;
     }

@@ -1,13 +1,422 @@
-// Step 1 of the LAQ iteration for the one-hidden-layer ReLU network of the paper's supplement.
+// Step 1 of the LAQ iteration for the one-hidden-layer ReLU network of the paper's supplement
+// ("Simulation details": 784-200-10, softmax cross-entropy, l2 regulariser).
+//
+// Parameter layout: W1 [H x F] row-major, b1 [H], W2 [C x H] row-major, b2 [C].
+// The two large products take bf16 operands (round to nearest even) and accumulate in fp32:
+//   hidden pre-activation  X~ W1~^T      (X~ = bf16(X), W1~ = bf16(W1))
+//   W1 gradient            dH~^T X~      (dH~ = bf16(dH))
+// everything else (output layer, softmax, bias gradients, regulariser) is fp32.
+//
+// Kernels per iteration:
+//   mlp_pack_w1_kernel     W1 (fp32, [H][F]) -> W1T (bf16, [F][H]) so that a thread reads 8 hidden units in one load
+//   mlp_forward_kernel     per tile of rows: hidden layer, logits, softmax, loss, dZ, dH (stored as bf16),
+//                          block partials of the b1 / W2 / b2 gradients
+//   mlp_dw1_kernel         dW1_m = dH~_m^T X~_m per worker, written straight into g (scaled, regularised)
+//   mlp_finalize_kernel    block partials -> g for b1, W2, b2, and the worker's loss term
+#include <cuda_bf16.h>
+
 #include "laq_internal.cuh"
 
 namespace laq {
 
-const char* mlp_check_shape(int, int, int) { return "LAQ_MODEL_MLP2 is not available in this build"; }
-size_t mlp_scratch_bytes(const laq_config&) { return 0; }
-laq_status mlp_setup(MlpPlan&, const Params&, void*, cudaStream_t) { return LAQ_EINVAL; }
-int mlp_convert_shard(MlpPlan&, const Params&, int, const float*, long long, cudaStream_t) { return 0; }
-int mlp_launch_gradients(MlpPlan&, const Params&, cudaStream_t) { return 0; }
-void mlp_teardown(MlpPlan&) {}
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kMaxC = 16;
+
+struct MlpDev {          // device pointers inside the scratch area
+  __nv_bfloat16* W1T;    // [F][H]
+  __nv_bfloat16* Xb;     // all shards, bf16, worker m at row offset rowoff[m]
+  __nv_bfloat16* dHb;    // [Ntot][H]
+  float* spart;          // [M][gb][H + C*H + C]   block partials of db1, dW2, db2
+  double* lpart;         // [M][gb]
+  long long* rowoff;     // [M+1] prefix sums of N_m
+  int gb;                // forward blocks per worker
+};
+
+__global__ void __launch_bounds__(256) mlp_pack_w1_kernel(const float* __restrict__ theta, __nv_bfloat16* __restrict__ W1T,
+                                                          int F, int H) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;  // index into W1T: k * H + j
+  if (i < F * H) {
+    const int k = i / H, j = i - k * H;
+    W1T[i] = __float2bfloat16_rn(theta[(long long)j * F + k]);
+  }
+}
+
+__global__ void __launch_bounds__(256) mlp_pack_x_kernel(const float* __restrict__ X, __nv_bfloat16* __restrict__ Xb,
+                                                         long long n) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
+    Xb[i] = __float2bfloat16_rn(__ldg(X + i));
+}
+
+// Thread layout of the two tile products: CG = H/8 column groups of 8 hidden units, RG = 256/CG row groups of
+// 4 rows; a tile has TR = 4 RG rows.
+__global__ void __launch_bounds__(kThreads) mlp_forward_kernel(const Params P, const MlpDev D) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int F = P.F, H = P.H, C = P.C, m = blockIdx.y, t = threadIdx.x, lane = t & 31, w = t >> 5;
+  const int CG = H >> 3, RG = kThreads / CG, TR = 4 * RG;
+  const int cg = t % CG, rg = t / CG;
+  const bool active = rg < RG;
+  __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(smem_raw);                 // [TR][F]
+  float* hs = reinterpret_cast<float*>(smem_raw + (((size_t)TR * F * 2 + 15) & ~(size_t)15));  // [TR][H]
+  float* dz = hs + (size_t)TR * H;                                                 // [TR][kMaxC]
+  __shared__ double shd[32];
+  const float* __restrict__ theta = P.theta;
+  const float* __restrict__ b1 = theta + (long long)H * F;
+  const float* __restrict__ W2 = b1 + H;
+  const float* __restrict__ b2 = W2 + (long long)C * H;
+  const long long n = P.N[m], row0 = D.rowoff[m];
+  const __nv_bfloat16* __restrict__ Xm = D.Xb + row0 * F;
+  const int32_t* __restrict__ y = P.y[m];
+  float acc_db1[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) acc_db1[c] = 0.f;
+  float acc_w2[kMaxC];      // thread t < H owns hidden unit t for the W2 gradient
+#pragma unroll
+  for (int c = 0; c < kMaxC; ++c) acc_w2[c] = 0.f;
+  float acc_b2 = 0.f;       // thread t < C
+  double loss = 0.0;
+  const long long ntiles = (n + TR - 1) / TR;
+  for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    const long long r0 = tile * TR;
+    const int nr = (int)((n - r0 < TR) ? (n - r0) : TR);
+    __syncthreads();
+    {  // stage the rows (contiguous) and zero the unused ones
+      const int cnt = nr * F, tot = TR * F;
+      const __nv_bfloat16* src = Xm + r0 * F;
+      if (((reinterpret_cast<uintptr_t>(src) & 15u) == 0)) {
+        const int n8 = cnt >> 3;
+        const uint4* s4 = reinterpret_cast<const uint4*>(src);
+        uint4* d4 = reinterpret_cast<uint4*>(xs);
+        for (int i = t; i < n8; i += kThreads) d4[i] = __ldg(s4 + i);
+        for (int i = (n8 << 3) + t; i < cnt; i += kThreads) xs[i] = src[i];
+      } else {
+        for (int i = t; i < cnt; i += kThreads) xs[i] = src[i];
+      }
+      for (int i = cnt + t; i < tot; i += kThreads) xs[i] = __float2bfloat16_rn(0.f);
+    }
+    __syncthreads();
+    // hidden layer: 4 rows x 8 hidden units per thread
+    if (active) {
+      float acc[4][8];
+#pragma unroll
+      for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int c = 0; c < 8; ++c) acc[r][c] = 0.f;
+      const __nv_bfloat16* xr = xs + (size_t)(4 * rg) * F;
+      const uint4* wp = reinterpret_cast<const uint4*>(D.W1T) + cg;   // 8 bf16 = 16 bytes per column group
+      for (int k = 0; k < F; ++k) {
+        const uint4 wv = __ldg(wp + (size_t)k * CG);
+        const __nv_bfloat162* w2p = reinterpret_cast<const __nv_bfloat162*>(&wv);
+        float wf[8];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const float2 f2 = __bfloat1622float2(w2p[c]);
+          wf[2 * c] = f2.x;
+          wf[2 * c + 1] = f2.y;
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          const float xv = __bfloat162float(xr[(size_t)r * F + k]);
+#pragma unroll
+          for (int c = 0; c < 8; ++c) acc[r][c] = fmaf(xv, wf[c], acc[r][c]);
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const int j = 8 * cg + c;
+          hs[(size_t)(4 * rg + r) * H + j] = fmaxf(acc[r][c] + __ldg(b1 + j), 0.f);
+        }
+    }
+    __syncthreads();
+    // output layer, softmax, loss, dZ: a warp per row
+    for (int r = w; r < TR; r += kThreads / 32) {
+      float z[kMaxC];
+#pragma unroll
+      for (int c = 0; c < kMaxC; ++c) z[c] = 0.f;
+      if (r < nr) {
+        const float* hr = hs + (size_t)r * H;
+        for (int j = lane; j < H; j += 32) {
+          const float hv = hr[j];
+#pragma unroll
+          for (int c = 0; c < kMaxC; ++c)
+            if (c < C) z[c] = fmaf(hv, __ldg(W2 + (size_t)c * H + j), z[c]);
+        }
+      }
+#pragma unroll
+      for (int c = 0; c < kMaxC; ++c) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) z[c] += __shfl_xor_sync(0xffffffffu, z[c], o);
+      }
+      if (r < nr) {
+        float zmax = -3.0e38f;
+#pragma unroll
+        for (int c = 0; c < kMaxC; ++c)
+          if (c < C) {
+            z[c] += __ldg(b2 + c);
+            zmax = fmaxf(zmax, z[c]);
+          }
+        float e[kMaxC], sum = 0.f;
+#pragma unroll
+        for (int c = 0; c < kMaxC; ++c) {
+          e[c] = (c < C) ? expf(z[c] - zmax) : 0.f;
+          sum += e[c];
+        }
+        const int yv = y[r0 + r];
+        const float inv = 1.0f / sum;
+        float zy = 0.f;
+#pragma unroll
+        for (int c = 0; c < kMaxC; ++c) {
+          if (c == yv) zy = z[c];
+          if (lane == 0 && c < C) dz[r * kMaxC + c] = e[c] * inv - (c == yv ? 1.f : 0.f);
+        }
+        if (lane == 0) loss += (double)((zmax + logf(sum)) - zy);
+      } else if (lane < kMaxC) {
+        dz[r * kMaxC + lane] = 0.f;   // rows beyond the shard contribute nothing
+      }
+    }
+    __syncthreads();
+    // W2 and b2 gradients (thread = hidden unit / class), on the unrounded hidden activations
+    if (t < H) {
+      for (int r = 0; r < nr; ++r) {
+        const float hv = hs[(size_t)r * H + t];
+#pragma unroll
+        for (int c = 0; c < kMaxC; ++c)
+          if (c < C) acc_w2[c] = fmaf(dz[r * kMaxC + c], hv, acc_w2[c]);
+      }
+    }
+    if (t < C)
+      for (int r = 0; r < nr; ++r) acc_b2 += dz[r * kMaxC + t];
+    // dH = (dZ W2) o relu'(H): same 4 x 8 layout; b1 gradient from the unrounded dH; dH stored as bf16
+    if (active) {
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int row = 4 * rg + r;
+        float d[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) d[c] = 0.f;
+        for (int cc = 0; cc < C; ++cc) {
+          const float dzv = dz[row * kMaxC + cc];
+          const float4 wa = __ldg(reinterpret_cast<const float4*>(W2 + (size_t)cc * H + 8 * cg));
+          const float4 wb = __ldg(reinterpret_cast<const float4*>(W2 + (size_t)cc * H + 8 * cg) + 1);
+          d[0] = fmaf(dzv, wa.x, d[0]); d[1] = fmaf(dzv, wa.y, d[1]); d[2] = fmaf(dzv, wa.z, d[2]); d[3] = fmaf(dzv, wa.w, d[3]);
+          d[4] = fmaf(dzv, wb.x, d[4]); d[5] = fmaf(dzv, wb.y, d[5]); d[6] = fmaf(dzv, wb.z, d[6]); d[7] = fmaf(dzv, wb.w, d[7]);
+        }
+        __nv_bfloat16 outv[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const float hv = hs[(size_t)row * H + 8 * cg + c];
+          const float dh = hv > 0.f ? d[c] : 0.f;
+          acc_db1[c] += dh;
+          outv[c] = __float2bfloat16_rn(dh);
+        }
+        if (row < nr)
+          *reinterpret_cast<uint4*>(D.dHb + (row0 + r0 + row) * H + 8 * cg) = *reinterpret_cast<const uint4*>(outv);
+      }
+    }
+  }
+  // block partials: [db1 (H) | dW2 (C*H) | db2 (C)]
+  __syncthreads();
+  float* red = hs;   // reuse the hidden-activation tile: [RG][H]
+  if (active)
+#pragma unroll
+    for (int c = 0; c < 8; ++c) red[rg * H + 8 * cg + c] = acc_db1[c];
+  __syncthreads();
+  float* sp = D.spart + ((long long)m * D.gb + blockIdx.x) * (H + C * H + C);
+  if (t < H) {
+    float s = 0.f;
+    for (int g = 0; g < RG; ++g) s += red[g * H + t];
+    sp[t] = s;
+    for (int c = 0; c < C; ++c) sp[H + c * H + t] = acc_w2[c];
+  }
+  if (t < C) sp[H + C * H + t] = acc_b2;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, o);
+  if (lane == 0) shd[w] = loss;
+  __syncthreads();
+  if (t == 0) {
+    double l = 0.0;
+    for (int i = 0; i < kThreads / 32; ++i) l += shd[i];
+    D.lpart[(long long)m * D.gb + blockIdx.x] = l;
+  }
+}
+
+// dW1_m[j][k] = sum_r dH~[r][j] X~[r][k]: a block owns a 32 x 128 output tile and walks the worker's rows.
+constexpr int kTJ = 32, kTK = 128, kRB = 32;
+
+__global__ void __launch_bounds__(kThreads) mlp_dw1_kernel(const Params P, const MlpDev D) {
+  __shared__ __align__(16) __nv_bfloat16 dhs[kRB][kTJ];
+  __shared__ __align__(16) __nv_bfloat16 xs[kRB][kTK];
+  const int F = P.F, H = P.H, m = blockIdx.z, t = threadIdx.x;
+  const int j0 = blockIdx.y * kTJ, k0 = blockIdx.x * kTK;
+  const int tx = t & 31, ty = t >> 5;       // 4 k per tx, 4 j per ty
+  const long long n = P.N[m], row0 = D.rowoff[m];
+  const __nv_bfloat16* __restrict__ Xm = D.Xb + row0 * F;
+  const __nv_bfloat16* __restrict__ dHm = D.dHb + row0 * H;
+  float acc[4][4];
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+  const __nv_bfloat16 zero = __float2bfloat16_rn(0.f);
+  for (long long r0 = 0; r0 < n; r0 += kRB) {
+    __syncthreads();
+    for (int i = t; i < kRB * kTJ; i += kThreads) {
+      const int r = i / kTJ, j = i - r * kTJ;
+      dhs[r][j] = (r0 + r < n && j0 + j < H) ? dHm[(r0 + r) * H + j0 + j] : zero;
+    }
+    for (int i = t; i < kRB * kTK; i += kThreads) {
+      const int r = i / kTK, k = i - r * kTK;
+      xs[r][k] = (r0 + r < n && k0 + k < F) ? Xm[(r0 + r) * F + k0 + k] : zero;
+    }
+    __syncthreads();
+#pragma unroll 4
+    for (int r = 0; r < kRB; ++r) {
+      const __nv_bfloat162* dp = reinterpret_cast<const __nv_bfloat162*>(&dhs[r][4 * ty]);
+      const __nv_bfloat162* xp = reinterpret_cast<const __nv_bfloat162*>(&xs[r][4 * tx]);
+      const float2 d01 = __bfloat1622float2(dp[0]), d23 = __bfloat1622float2(dp[1]);
+      const float2 x01 = __bfloat1622float2(xp[0]), x23 = __bfloat1622float2(xp[1]);
+      const float dv[4] = {d01.x, d01.y, d23.x, d23.y}, xv[4] = {x01.x, x01.y, x23.x, x23.y};
+#pragma unroll
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(dv[a], xv[b], acc[a][b]);
+    }
+  }
+  const float inv_N = (float)(1.0 / (double)P.Ntot);
+  const float reg = (float)((double)n / (double)P.Ntot * (double)P.lambda);
+#pragma unroll
+  for (int a = 0; a < 4; ++a) {
+    const int j = j0 + 4 * ty + a;
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int k = k0 + 4 * tx + b;
+      if (j < H && k < F) {
+        const long long i = (long long)j * F + k;
+        P.g[(long long)m * P.ps + i] = fmaf(acc[a][b], inv_N, reg * P.theta[i]);
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) mlp_finalize_kernel(const Params P, const MlpDev D, const double* theta_sq) {
+  const int H = P.H, C = P.C, F = P.F, m = blockIdx.y;
+  const int nsmall = H + C * H + C;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  const double inv_N = 1.0 / (double)P.Ntot, share = (double)P.N[m] / (double)P.Ntot;
+  if (i < nsmall) {
+    double s = 0.0;
+    for (int b = 0; b < D.gb; ++b) s += (double)D.spart[((long long)m * D.gb + b) * nsmall + i];
+    const long long pi = (long long)H * F + i;   // b1, W2, b2 follow W1 in theta in the same order as the partials
+    P.g[(long long)m * P.ps + pi] = (float)(s * inv_N + share * (double)P.lambda * (double)P.theta[pi]);
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    double l = 0.0;
+    for (int b = 0; b < D.gb; ++b) l += D.lpart[(long long)m * D.gb + b];
+    P.loss_m[m] = l * inv_N + share * 0.5 * (double)P.lambda * (*theta_sq);
+  }
+}
+
+struct HostPlan {
+  MlpDev d;
+  size_t fwd_smem;
+};
+
+size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+
+int forward_blocks_per_worker(int M) {
+  int g = (2 * kNumSMs + M - 1) / M;
+  return g < 1 ? 1 : (g > 64 ? 64 : g);
+}
+
+size_t forward_smem(int F, int H) {
+  const int CG = H / 8, RG = kThreads / CG, TR = 4 * RG;
+  return (((size_t)TR * F * 2 + 15) & ~(size_t)15) + (size_t)TR * H * 4 + (size_t)TR * kMaxC * 4;
+}
+
+}  // namespace
+
+const char* mlp_check_shape(int F, int H, int C) {
+  if (H < 8 || H > 256 || (H % 8) != 0) return "MLP2 supports n_hidden in 8..256, a multiple of 8";
+  if (C < 2 || C > kMaxC) return "MLP2 supports 2..16 classes";
+  if (F < 1 || forward_smem(F, H) > 200 * 1024) return "MLP2: n_features too large for the row tile";
+  return nullptr;
+}
+
+size_t mlp_scratch_bytes(const laq_config& c) {
+  long long Ntot = 0;
+  for (int m = 0; m < c.M; ++m) Ntot += c.N[m];
+  const int gb = forward_blocks_per_worker(c.M);
+  const size_t nsmall = (size_t)c.n_hidden + (size_t)c.n_classes * c.n_hidden + c.n_classes;
+  size_t b = 0;
+  b += align256((size_t)c.n_features * c.n_hidden * 2);          // W1T
+  b += align256((size_t)Ntot * c.n_features * 2);                // Xb
+  b += align256((size_t)Ntot * c.n_hidden * 2);                  // dHb
+  b += align256((size_t)c.M * gb * nsmall * 4);                  // spart
+  b += align256((size_t)c.M * gb * 8);                           // lpart
+  b += align256((size_t)(c.M + 1) * 8);                          // rowoff
+  return b;
+}
+
+laq_status mlp_setup(MlpPlan& mp, const Params& P, void* scratch, cudaStream_t st) {
+  HostPlan* hp = new HostPlan();
+  char* p = (char*)scratch;
+  const size_t nsmall = (size_t)P.H + (size_t)P.C * P.H + P.C;
+  hp->d.gb = forward_blocks_per_worker(P.M);
+  hp->d.W1T = (__nv_bfloat16*)p; p += align256((size_t)P.F * P.H * 2);
+  hp->d.Xb = (__nv_bfloat16*)p; p += align256((size_t)P.Ntot * P.F * 2);
+  hp->d.dHb = (__nv_bfloat16*)p; p += align256((size_t)P.Ntot * P.H * 2);
+  hp->d.spart = (float*)p; p += align256((size_t)P.M * hp->d.gb * nsmall * 4);
+  hp->d.lpart = (double*)p; p += align256((size_t)P.M * hp->d.gb * 8);
+  hp->d.rowoff = (long long*)p;
+  hp->fwd_smem = forward_smem(P.F, P.H);
+  // prefix sums of the shard sizes (N is not yet on the device when this runs, so it comes from the host copy)
+  mp.scratch = hp;
+  mp.ready = 0;
+  if (cudaFuncSetAttribute(mlp_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hp->fwd_smem) !=
+      cudaSuccess)
+    return LAQ_ECUDA;
+  (void)st;
+  return LAQ_OK;
+}
+
+laq_status mlp_set_row_offsets(MlpPlan& mp, const long long* N_host, int M, cudaStream_t st) {
+  HostPlan* hp = (HostPlan*)mp.scratch;
+  long long off[1025];
+  off[0] = 0;
+  for (int m = 0; m < M; ++m) off[m + 1] = off[m] + N_host[m];
+  if (cudaMemcpyAsync(hp->d.rowoff, off, sizeof(long long) * (M + 1), cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return LAQ_ECUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return LAQ_ECUDA;
+  return LAQ_OK;
+}
+
+int mlp_convert_shard(MlpPlan& mp, const Params& P, int m, const float* X, long long n, long long row_offset,
+                      cudaStream_t st) {
+  HostPlan* hp = (HostPlan*)mp.scratch;
+  const long long cnt = n * P.F;
+  mlp_pack_x_kernel<<<kNumSMs * 4, 256, 0, st>>>(X, hp->d.Xb + row_offset * P.F, cnt);
+  (void)m;
+  return 1;
+}
+
+int mlp_launch_gradients(MlpPlan& mp, const Params& P, const double* theta_sq, cudaStream_t st) {
+  HostPlan* hp = (HostPlan*)mp.scratch;
+  const int F = P.F, H = P.H, C = P.C;
+  mlp_pack_w1_kernel<<<(F * H + 255) / 256, 256, 0, st>>>(P.theta, hp->d.W1T, F, H);
+  mlp_forward_kernel<<<dim3(hp->d.gb, P.M), kThreads, hp->fwd_smem, st>>>(P, hp->d);
+  mlp_dw1_kernel<<<dim3((F + kTK - 1) / kTK, (H + kTJ - 1) / kTJ, P.M), kThreads, 0, st>>>(P, hp->d);
+  const int nsmall = H + C * H + C;
+  mlp_finalize_kernel<<<dim3((nsmall + 255) / 256, P.M), 256, 0, st>>>(P, hp->d, theta_sq);
+  return 4;
+}
+
+void mlp_teardown(MlpPlan& mp) {
+  delete (HostPlan*)mp.scratch;
+  mp.scratch = nullptr;
+}
 
 }  // namespace laq

@@ -89,7 +89,13 @@ __device__ __forceinline__ double block_sum(double v, double* sh /* >= 32 double
   return t;
 }
 
-constexpr int kUnroll = 4;
+#ifndef LAQ_SWEEP_UNROLL
+#define LAQ_SWEEP_UNROLL 2
+#endif
+#ifndef LAQ_QUANT_MIN_BLOCKS
+#define LAQ_QUANT_MIN_BLOCKS 2   // caps the quantize kernel at 64 registers (measured best)
+#endif
+constexpr int kUnroll = LAQ_SWEEP_UNROLL;  // 16-byte groups in flight per thread
 
 // ------------------------------------------------------------------------------------------------
 // radius
@@ -389,7 +395,7 @@ __device__ __forceinline__ void zero_codes(const Params& P, int m) {
 }
 
 template <bool SYNTH, int B>
-__global__ void __launch_bounds__(512) quantize_kernel(const Params P) {
+__global__ void __launch_bounds__(512, LAQ_QUANT_MIN_BLOCKS) quantize_kernel(const Params P) {
   __shared__ double sh[32];
   __shared__ bool is_last;
   const int m = blockIdx.y;

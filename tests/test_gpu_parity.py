@@ -232,8 +232,11 @@ def _run_model_parity(w, iters):
         gs = ctx.get_state(g=True, codes=True)
         # (1)
         g_ref = _oracle_gradients(w, prev["theta"])
+        # the network rounds dH to bf16: an fp32 dH next to a bf16 rounding boundary may round the other way
+        # than the oracle's fp64 dH, which moves single terms of the W1 gradient by 2^-9 relative
+        grad_rtol = 2e-4 if w.model == workloads.MODEL_MLP2 else GRAD_RTOL
         for m in range(w.M):
-            assert np.linalg.norm(gs["g"][m] - g_ref[m]) <= GRAD_RTOL * np.linalg.norm(g_ref[m]), (k, m)
+            assert np.linalg.norm(gs["g"][m] - g_ref[m]) <= grad_rtol * np.linalg.norm(g_ref[m]), (k, m)
         # (2)
         st32 = mir.step_given(gs["g"])
         _assert_trace_row(tr, 0, st32)
@@ -303,6 +306,16 @@ def test_c1_shape_softmax_reduced():
 
 def test_softmax_small_odd_shapes():
     w = workloads.c1(n_per=37, F=50, C=3, M=4, iters=15)
+    _run_model_parity(w, w.iters)
+
+
+def test_c3_shape_mlp_reduced():
+    w = workloads.c3(n_per=96, M=4, iters=8)              # 784-200-10, bf16 operands in the two large products
+    _run_model_parity(w, w.iters)
+
+
+def test_mlp_small_odd_shapes():
+    w = workloads.c3(n_per=37, M=3, F=50, H=24, C=3, iters=10)
     _run_model_parity(w, w.iters)
 
 
