@@ -105,7 +105,8 @@ struct Plan {
 };
 
 int default_gbpw(const laq_config& c) {
-  int g = (2 * kNumSMs + c.M - 1) / c.M;
+  // resident blocks per SM: two for the softmax tiles, four for the narrow logistic tiles; one wave
+  int g = ((c.model == LAQ_MODEL_LOGREG_BIN ? 4 : 2) * kNumSMs) / c.M;
   if (g > kGradBlocksCap) g = kGradBlocksCap;
   return g < 1 ? 1 : g;
 }

@@ -5,6 +5,8 @@
 // (contiguous in memory) in shared memory, computes the residuals (sigma(z) - y, or softmax - onehot)
 // and accumulates residual^T x in registers across its tiles.  Block partials are combined in a
 // fixed order by grad_finalize_kernel, which also adds the regulariser share.
+#include <cuda_pipeline.h>
+
 #include "laq_internal.cuh"
 
 namespace laq {
@@ -22,14 +24,16 @@ __device__ __forceinline__ float warp_sum_f(float v) {
   return v;
 }
 
-// Copy `count` consecutive floats global -> shared with 16-byte loads where alignment allows.
+// Copy `count` consecutive floats global -> shared; where alignment allows as asynchronous 16-byte copies, so
+// that every thread has all of its copies in flight at once.  Ends with the copies complete for this thread;
+// the caller's __syncthreads() makes them visible to the block.
 __device__ __forceinline__ void stage_rows(const float* __restrict__ src, float* dst, int count) {
   if ((reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
     const int n4 = count >> 2;
-    const float4* s4 = reinterpret_cast<const float4*>(src);
-    float4* d4 = reinterpret_cast<float4*>(dst);
-    for (int i = threadIdx.x; i < n4; i += blockDim.x) d4[i] = __ldg(s4 + i);
+    for (int i = threadIdx.x; i < n4; i += blockDim.x) __pipeline_memcpy_async(dst + 4 * i, src + 4 * i, 16);
+    __pipeline_commit();
     for (int i = (n4 << 2) + threadIdx.x; i < count; i += blockDim.x) dst[i] = __ldg(src + i);
+    __pipeline_wait_prior(0);
   } else {
     for (int i = threadIdx.x; i < count; i += blockDim.x) dst[i] = __ldg(src + i);
   }
@@ -205,6 +209,163 @@ __global__ void __launch_bounds__(kSmThreads) grad_softmax_kernel(const Params P
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// C-class softmax regression, fast path: F a multiple of 4, F <= 896, C <= 12.
+// 224 threads (7 warps), tiles of 16 rows staged in shared memory with a row stride of an odd number of
+// 16-byte units (conflict-free 16-byte reads down a column of rows); theta sits in shared memory too.
+//   phase 1  lane = (row, parity of the 16-byte feature group), warp = slice of the feature axis: scores from
+//            16-byte reads of x and broadcast 16-byte reads of theta; the 14 partials per (row, class) are
+//            summed through shared memory, one thread per row then does softmax, residual and loss;
+//   phase 2  thread = four consecutive features: acc[4][C] += residual[r][c] * x[r][f] over the tile's rows,
+//            one 16-byte read of x and the broadcast residuals per row.
+// Two blocks fit on an SM, so one block's loads overlap the other's arithmetic.
+// ------------------------------------------------------------------------------------------------
+constexpr int kS2Threads = 224;
+constexpr int kS2Warps = 7;
+constexpr int kS2Rows = 16;
+constexpr int kS2Parts = 2 * kS2Warps;   // partial scores per (row, class)
+
+template <int C>
+__global__ void __launch_bounds__(kS2Threads, 2) grad_softmax_tile_kernel(const Params P, int gbpw) {
+  extern __shared__ __align__(16) float smem[];
+  const int F = P.F, F4 = F >> 2, FP4 = F4 | 1, FP = FP4 << 2;      // padded row stride (floats)
+  const int m = blockIdx.y, t = threadIdx.x, lane = t & 31, w = t >> 5;
+  float* xs = smem;                                  // [16][FP]
+  float* ths = xs + kS2Rows * FP;                    // [C][F]      theta
+  float* plog = ths + C * F;                         // [14][16][C] partial scores
+  float* res = plog + kS2Parts * kS2Rows * C;        // [16][12]    residuals, padded to 16-byte rows
+  __shared__ double shd[8];
+  __shared__ float zs[kS2Rows * 12];                 // [16][C]     scores
+  static_assert(kS2Rows * C <= kS2Threads, "one thread per (row, class)");
+  const float* __restrict__ X = P.X[m];
+  const int32_t* __restrict__ y = P.y[m];
+  const long long n = P.N[m];
+  for (int i = t; i < C * F4; i += kS2Threads)
+    reinterpret_cast<float4*>(ths)[i] = __ldg(reinterpret_cast<const float4*>(P.theta) + i);
+  const float4* th4 = reinterpret_cast<const float4*>(ths);
+  const int kw = (F4 + kS2Warps - 1) / kS2Warps;     // 16-byte groups of features per warp in phase 1
+  const int row1 = lane & 15, par = lane >> 4;
+  const int k_lo = w * kw + par, k_hi = min(F4, w * kw + kw);
+  const bool owner = t < F4;                         // phase 2: thread t owns features 4t .. 4t+3
+  float acc[4][C];
+#pragma unroll
+  for (int e = 0; e < 4; ++e)
+#pragma unroll
+    for (int c = 0; c < C; ++c) acc[e][c] = 0.f;
+  double loss = 0.0;
+  const long long ntiles = (n + kS2Rows - 1) / kS2Rows;
+  for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    const long long r0 = tile * kS2Rows;
+    const int nr = (int)((n - r0 < kS2Rows) ? (n - r0) : kS2Rows);
+    __syncthreads();
+    {  // stage: contiguous rows in global memory -> padded rows in shared memory, as asynchronous 16-byte
+       // copies so that a thread has all of its copies in flight at once
+      const float4* src = reinterpret_cast<const float4*>(X + r0 * F);
+      const int cnt = nr * F4;
+      int r = t / F4, k = t - r * F4;
+      for (int i = t; i < kS2Rows * F4; i += kS2Threads) {
+        float* dst = xs + r * FP + 4 * k;
+        if (i < cnt)
+          __pipeline_memcpy_async(dst, src + i, 16);
+        else
+          *reinterpret_cast<float4*>(dst) = make_float4(0.f, 0.f, 0.f, 0.f);
+        k += kS2Threads;
+        while (k >= F4) {
+          k -= F4;
+          ++r;
+        }
+      }
+      __pipeline_commit();
+      __pipeline_wait_prior(0);
+    }
+    __syncthreads();
+    {  // phase 1
+      float z[C];
+#pragma unroll
+      for (int c = 0; c < C; ++c) z[c] = 0.f;
+      const float4* xr = reinterpret_cast<const float4*>(xs + row1 * FP);
+      for (int k = k_lo; k < k_hi; k += 2) {
+        const float4 x = xr[k];
+#pragma unroll
+        for (int c = 0; c < C; ++c) {
+          const float4 th = th4[c * F4 + k];
+          z[c] = fmaf(x.x, th.x, z[c]);
+          z[c] = fmaf(x.y, th.y, z[c]);
+          z[c] = fmaf(x.z, th.z, z[c]);
+          z[c] = fmaf(x.w, th.w, z[c]);
+        }
+      }
+#pragma unroll
+      for (int c = 0; c < C; ++c) plog[((2 * w + par) * kS2Rows + row1) * C + c] = z[c];
+    }
+    __syncthreads();
+    if (t < kS2Rows * C) {  // one thread per (row, class): sum the 14 partial scores in a fixed order
+      float s = 0.f;
+#pragma unroll
+      for (int ww = 0; ww < kS2Parts; ++ww) s += plog[ww * kS2Rows * C + t];
+      zs[t] = s;
+    }
+    __syncthreads();
+    if (t < kS2Rows) {  // one thread per row: softmax, residual, loss
+      float z[C];
+#pragma unroll
+      for (int c = 0; c < C; ++c) z[c] = zs[t * C + c];
+      float zmax = z[0];
+#pragma unroll
+      for (int c = 1; c < C; ++c) zmax = fmaxf(zmax, z[c]);
+      float e[C], sum = 0.f;
+#pragma unroll
+      for (int c = 0; c < C; ++c) {
+        e[c] = expf(z[c] - zmax);
+        sum += e[c];
+      }
+      const bool live = t < nr;
+      const int yv = live ? y[r0 + t] : -1;
+      const float inv = 1.0f / sum;
+      float zy = 0.f;
+#pragma unroll
+      for (int c = 0; c < C; ++c) {
+        if (c == yv) zy = z[c];
+        res[t * 12 + c] = live ? (e[c] * inv - (c == yv ? 1.f : 0.f)) : 0.f;
+      }
+      if (live) loss += (double)((zmax + logf(sum)) - zy);
+    }
+    __syncthreads();
+    if (owner) {  // phase 2
+      const float* xc = xs + 4 * t;
+      for (int r = 0; r < nr; ++r) {
+        const float4 x = *reinterpret_cast<const float4*>(xc + r * FP);
+        float rr[12];
+        *reinterpret_cast<float4*>(rr) = *reinterpret_cast<const float4*>(res + r * 12);
+        *reinterpret_cast<float4*>(rr + 4) = *reinterpret_cast<const float4*>(res + r * 12 + 4);
+        *reinterpret_cast<float4*>(rr + 8) = *reinterpret_cast<const float4*>(res + r * 12 + 8);
+#pragma unroll
+        for (int c = 0; c < C; ++c) {
+          acc[0][c] = fmaf(rr[c], x.x, acc[0][c]);
+          acc[1][c] = fmaf(rr[c], x.y, acc[1][c]);
+          acc[2][c] = fmaf(rr[c], x.z, acc[2][c]);
+          acc[3][c] = fmaf(rr[c], x.w, acc[3][c]);
+        }
+      }
+    }
+  }
+  float* gp = P.gpart + ((long long)m * gbpw + blockIdx.x) * P.ps;
+  if (owner) {
+#pragma unroll
+    for (int c = 0; c < C; ++c)
+      *reinterpret_cast<float4*>(gp + c * F + 4 * t) = make_float4(acc[0][c], acc[1][c], acc[2][c], acc[3][c]);
+  }
+  loss = warp_sum_d(loss);
+  __syncthreads();
+  if (lane == 0) shd[w] = loss;
+  __syncthreads();
+  if (t == 0) {
+    double l = 0.0;
+    for (int i = 0; i < kS2Warps; ++i) l += shd[i];
+    P.lpart[(long long)m * gbpw + blockIdx.x] = l;
+  }
+}
+
 }  // namespace
 
 // Combine the block partials of worker blockIdx.y in block order, scale by 1/N and add the
@@ -252,8 +413,23 @@ int launch_grad_logreg(const Params& P, const LaunchShape&, int gbpw, cudaStream
   return 1;
 }
 
+static bool softmax_tile_path(int F, int C) { return (F % 4) == 0 && F / 4 <= kS2Threads && C <= 12; }
+static size_t softmax_tile_smem(int F, int C) {
+  const int FP = ((F >> 2) | 1) << 2;
+  return sizeof(float) * ((size_t)kS2Rows * FP + (size_t)C * F + (size_t)kS2Parts * kS2Rows * C + (size_t)kS2Rows * 12);
+}
+
 template <int C>
 static void launch_sm(const Params& P, int gbpw, cudaStream_t st) {
+  constexpr int CT = (C <= 12 ? C : 2);   // the tile kernel is only instantiated for C <= 12
+  if (softmax_tile_path(P.F, C) && softmax_tile_smem(P.F, C) <= 112 * 1024) {
+    const size_t sm = softmax_tile_smem(P.F, C);
+    cudaFuncSetAttribute(grad_softmax_tile_kernel<CT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    cudaFuncSetAttribute(grad_softmax_tile_kernel<CT>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                         cudaSharedmemCarveoutMaxShared);  // room for two blocks per SM
+    grad_softmax_tile_kernel<CT><<<dim3(gbpw, P.M), kS2Threads, sm, st>>>(P, gbpw);
+    return;
+  }
   const size_t sm = softmax_smem(P.F, C);
   cudaFuncSetAttribute(grad_softmax_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
   grad_softmax_kernel<C><<<dim3(gbpw, P.M), kSmThreads, sm, st>>>(P, gbpw);
