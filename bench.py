@@ -6,7 +6,8 @@
 A step is one LAQ iteration (Algorithm 2: local gradients, quantizer, norms, skip rule, lazy aggregate and
 theta step) over all M workers of the workload.  Prints one JSON line (rank 0).  Workloads:
 c4_b8 (default: M = 64, p = 25.6 M, b = 8, gradients generated in the kernels), c4_b4, c4_b2,
-c4_b8_xi0 (every worker uploads), c4_b8_frozen (no drift: uploads die out), c0, c1, c2 (model workloads).
+c4_b8_xi0 (every worker uploads), c4_b8_frozen (no drift: uploads die out), c4_b8_M8 (8 workers: a small case
+for profiler captures), c0, c1, c2, c3 (model workloads).
 With N > 1 (torchrun) every rank runs an independent replica of the workload on its own GPU: the path does
 not shard across GPUs and has no collective; the timing is the maximum over ranks.
 """
@@ -42,6 +43,9 @@ def make_workload(name):
             kw["xi_scale"] = 0.0
         if "frozen" in parts:
             kw["eta0"] = 0.0
+        for part in parts:                      # e.g. c4_b8_M8: fewer workers, a 1 GB case for profiler captures
+            if part.startswith("M") and part[1:].isdigit():
+                kw["M"] = int(part[1:])
         return W.c4(b=b, **kw)
     return {"c0": W.c0, "c1": W.c1, "c2": W.c2, "c3": W.c3}[name]()
 
@@ -126,8 +130,8 @@ def traffic_for(stage, w):
         src = os.path.join(ROOT, "paper_1909_07588_b200", "csrc", rec["source"])
         if hashlib.sha256(open(src, "rb").read()).hexdigest() != rec["source_sha256"]:
             return None
-        per_coord = rec["bytes_per_worker_coordinate"][w.name.split("_M")[0] + "_b%d" % w.b][stage]
-        return per_coord * float(w.M) * w.p
+        per_coord = rec["bytes_per_worker_coordinate"]["c4_b%d" % w.b][stage]
+        return None if per_coord is None or w.model != 3 else per_coord * float(w.M) * w.p
     except Exception:
         return None
 
