@@ -203,6 +203,7 @@ laq_status check_device_error(laq_ctx* ctx) {
   LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));
   if (err & 1u)
     return fail(ctx, LAQ_ENONFINITE, "a gradient or radius was not finite; the state is frozen at that iteration");
+  if (err & ~1u) return fail(ctx, LAQ_ECUDA, "a bounded wait in the tensor-core pipeline ran out; the state is frozen");
   return LAQ_OK;
 }
 
@@ -321,6 +322,7 @@ laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, siz
     if (c.model == LAQ_MODEL_MLP2) {
       laq_status s = mlp_setup(ctx->mlp, P, ws + pl.mlp, ctx->st);
       if (s == LAQ_OK) s = mlp_set_row_offsets(ctx->mlp, (const long long*)ctx->N.data(), c.M, ctx->st);
+      if (s == LAQ_OK) s = mlp_setup_tensor_path(ctx->mlp, P, ctx->st);
       if (s != LAQ_OK) return fail(ctx, s, "network scratch set-up failed");
     }
   }

@@ -13,9 +13,17 @@
 //                          block partials of the b1 / W2 / b2 gradients
 //   mlp_dw1_kernel         dW1_m = dH~_m^T X~_m per worker, written straight into g (scaled, regularised)
 //   mlp_finalize_kernel    block partials -> g for b1, W2, b2, and the worker's loss term
+// Tensor-core path (n_features a multiple of 8): the two large products run on tcgen05 (laq_umma_gemm.cuh):
+//   umma_hidden_kernel     H = relu(X~ W1~^T + b1) for all workers' rows at once, fp32 to memory
+//   mlp_forward_kernel<1>  as above without the hidden product; writes dH~ transposed ([H][rows], K-major for
+//                          the second product; every worker's row segment padded to a multiple of 64 with zeros)
+//   umma_dw1_kernel        dW1_m = dH~_m^T X~_m from the transposed copies dH~^T and X~^T (made once per shard)
 #include <cuda_bf16.h>
 
+#include <vector>
+
 #include "laq_internal.cuh"
+#include "laq_umma_gemm.cuh"
 
 namespace laq {
 
@@ -32,6 +40,13 @@ struct MlpDev {          // device pointers inside the scratch area
   double* lpart;         // [M][gb]
   long long* rowoff;     // [M+1] prefix sums of N_m
   int gb;                // forward blocks per worker
+  // tensor-core path
+  __nv_bfloat16* W1b;    // [H][F]
+  float* Hbuf;           // [Ntot][H]  hidden activations
+  __nv_bfloat16* dHT;    // [H][ldT]   dH~ transposed
+  __nv_bfloat16* XbT;    // [F][ldT]   X~ transposed
+  long long* rowoffT;    // [M+1] prefix sums of N_m rounded up to 64
+  long long ldT;         // sum of the rounded shard sizes
 };
 
 __global__ void __launch_bounds__(256) mlp_pack_w1_kernel(const float* __restrict__ theta, __nv_bfloat16* __restrict__ W1T,
@@ -52,14 +67,15 @@ __global__ void __launch_bounds__(256) mlp_pack_x_kernel(const float* __restrict
 
 // Thread layout of the two tile products: CG = H/8 column groups of 8 hidden units, RG = 256/CG row groups of
 // 4 rows; a tile has TR = 4 RG rows.
+template <bool TC>
 __global__ void __launch_bounds__(kThreads) mlp_forward_kernel(const Params P, const MlpDev D) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int F = P.F, H = P.H, C = P.C, m = blockIdx.y, t = threadIdx.x, lane = t & 31, w = t >> 5;
   const int CG = H >> 3, RG = kThreads / CG, TR = 4 * RG;
   const int cg = t % CG, rg = t / CG;
   const bool active = rg < RG;
-  __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(smem_raw);                 // [TR][F]
-  float* hs = reinterpret_cast<float*>(smem_raw + (((size_t)TR * F * 2 + 15) & ~(size_t)15));  // [TR][H]
+  __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(smem_raw);                 // [TR][F]   (not for TC)
+  float* hs = reinterpret_cast<float*>(smem_raw + (TC ? 0 : (((size_t)TR * F * 2 + 15) & ~(size_t)15)));  // [TR][H]
   float* dz = hs + (size_t)TR * H;                                                 // [TR][kMaxC]
   __shared__ double shd[32];
   const float* __restrict__ theta = P.theta;
@@ -82,7 +98,12 @@ __global__ void __launch_bounds__(kThreads) mlp_forward_kernel(const Params P, c
     const long long r0 = tile * TR;
     const int nr = (int)((n - r0 < TR) ? (n - r0) : TR);
     __syncthreads();
-    {  // stage the rows (contiguous) and zero the unused ones
+    if (TC) {  // the hidden activations come from the tensor-core product
+      const float4* src = reinterpret_cast<const float4*>(D.Hbuf + (row0 + r0) * H);
+      float4* dst = reinterpret_cast<float4*>(hs);
+      const int cnt4 = nr * H / 4, tot4 = TR * H / 4;
+      for (int i = t; i < tot4; i += kThreads) dst[i] = (i < cnt4) ? __ldg(src + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    } else {  // stage the rows (contiguous) and zero the unused ones
       const int cnt = nr * F, tot = TR * F;
       const __nv_bfloat16* src = Xm + r0 * F;
       if (((reinterpret_cast<uintptr_t>(src) & 15u) == 0)) {
@@ -98,7 +119,7 @@ __global__ void __launch_bounds__(kThreads) mlp_forward_kernel(const Params P, c
     }
     __syncthreads();
     // hidden layer: 4 rows x 8 hidden units per thread
-    if (active) {
+    if (!TC && active) {
       float acc[4][8];
 #pragma unroll
       for (int r = 0; r < 4; ++r)
@@ -192,6 +213,7 @@ __global__ void __launch_bounds__(kThreads) mlp_forward_kernel(const Params P, c
       for (int r = 0; r < nr; ++r) acc_b2 += dz[r * kMaxC + t];
     // dH = (dZ W2) o relu'(H): same 4 x 8 layout; b1 gradient from the unrounded dH; dH stored as bf16
     if (active) {
+      __nv_bfloat16 dht[4][8];
 #pragma unroll
       for (int r = 0; r < 4; ++r) {
         const int row = 4 * rg + r;
@@ -212,9 +234,20 @@ __global__ void __launch_bounds__(kThreads) mlp_forward_kernel(const Params P, c
           const float dh = hv > 0.f ? d[c] : 0.f;
           acc_db1[c] += dh;
           outv[c] = __float2bfloat16_rn(dh);
+          if (TC) dht[r][c] = outv[c];
         }
-        if (row < nr)
+        if (!TC && row < nr)
           *reinterpret_cast<uint4*>(D.dHb + (row0 + r0 + row) * H + 8 * cg) = *reinterpret_cast<const uint4*>(outv);
+      }
+      if (TC) {  // transposed store: four consecutive rows of one hidden unit are 8 contiguous bytes
+        const long long col = D.rowoffT[m] + r0 + 4 * rg;
+        if (col + 3 < D.rowoffT[m + 1]) {
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            __nv_bfloat16 v4[4] = {dht[0][c], dht[1][c], dht[2][c], dht[3][c]};   // rows >= nr hold dh = 0
+            *reinterpret_cast<uint2*>(D.dHT + (long long)(8 * cg + c) * D.ldT + col) = *reinterpret_cast<const uint2*>(v4);
+          }
+        }
       }
     }
   }
@@ -320,9 +353,97 @@ __global__ void __launch_bounds__(256) mlp_finalize_kernel(const Params P, const
   }
 }
 
+// ---- tensor-core path ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) mlp_pack_w1b_kernel(const float* __restrict__ theta, __nv_bfloat16* __restrict__ W1b,
+                                                           int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) W1b[i] = __float2bfloat16_rn(theta[i]);
+}
+
+// XbT[k][col0 + r] = bf16(X[r][k]) for one shard (done once, when the shard is loaded)
+__global__ void __launch_bounds__(256) mlp_transpose_x_kernel(const float* __restrict__ X, __nv_bfloat16* __restrict__ XbT,
+                                                              long long n, int F, long long ldT, long long col0) {
+  __shared__ float tile[32][33];
+  const long long r0 = (long long)blockIdx.x * 32;
+  const int k0 = blockIdx.y * 32, tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int i = ty; i < 32; i += 8)
+    tile[i][tx] = (r0 + i < n && k0 + tx < F) ? __ldg(X + (r0 + i) * F + k0 + tx) : 0.f;
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8)
+    if (k0 + i < F && r0 + tx < n) XbT[(long long)(k0 + i) * ldT + col0 + r0 + tx] = __float2bfloat16_rn(tile[tx][i]);
+}
+
+struct HiddenEpi {
+  float* Hbuf;
+  const float* b1;
+  long long Ntot;
+  int H, i0;
+  __device__ __forceinline__ void operator()(int r, int c0, const float (&acc)[32]) const {
+    const long long row = (long long)i0 + r;
+    if (row >= Ntot) return;
+    float* out = Hbuf + row * H + c0;
+#pragma unroll
+    for (int c = 0; c < 32; c += 4) {
+      if (c0 + c < H) {   // H is a multiple of 8, chunks of 4 columns are all in or all out
+        const float4 b = __ldg(reinterpret_cast<const float4*>(b1 + c0 + c));
+        float4 v;
+        v.x = fmaxf(acc[c] + b.x, 0.f);
+        v.y = fmaxf(acc[c + 1] + b.y, 0.f);
+        v.z = fmaxf(acc[c + 2] + b.z, 0.f);
+        v.w = fmaxf(acc[c + 3] + b.w, 0.f);
+        *reinterpret_cast<float4*>(out + c) = v;
+      }
+    }
+  }
+};
+
+__global__ void __launch_bounds__(umma::kThreads) umma_hidden_kernel(const __grid_constant__ CUtensorMap tmX,
+                                                                     const __grid_constant__ CUtensorMap tmW,
+                                                                     const Params P, const MlpDev D, int nt) {
+  umma::TileCoord tc{(int)blockIdx.x * umma::kTileM, 0, 0, (P.F + umma::kBlockK - 1) / umma::kBlockK};
+  HiddenEpi epi{D.Hbuf, P.theta + (long long)P.H * P.F, P.Ntot, P.H, tc.i0};
+  umma::gemm_tn_tile(&tmX, &tmW, nt, tc, &P.sc->err, epi);
+}
+
+struct Dw1Epi {
+  float* g;            // worker's gradient row
+  const float* theta;
+  float inv_N, reg;
+  int H, F, j0, k0, nt;
+  __device__ __forceinline__ void operator()(int r, int c0, const float (&acc)[32]) const {
+    const int j = j0 + r;
+    if (j >= H) return;
+#pragma unroll
+    for (int c = 0; c < 32; ++c) {
+      const int k = k0 + c0 + c;
+      if (c0 + c < nt && k < F) {
+        const long long i = (long long)j * F + k;
+        g[i] = fmaf(acc[c], inv_N, reg * theta[i]);
+      }
+    }
+  }
+};
+
+__global__ void __launch_bounds__(umma::kThreads) umma_dw1_kernel(const __grid_constant__ CUtensorMap tmD,
+                                                                  const __grid_constant__ CUtensorMap tmXT,
+                                                                  const Params P, const MlpDev D, int nt) {
+  const int m = blockIdx.z;
+  const long long c0 = D.rowoffT[m], c1 = D.rowoffT[m + 1];
+  umma::TileCoord tc{(int)blockIdx.y * umma::kTileM, (int)blockIdx.x * nt, (int)c0, (int)((c1 - c0) / umma::kBlockK)};
+  const long long n = P.N[m];
+  Dw1Epi epi{P.g + (long long)m * P.ps, P.theta, (float)(1.0 / (double)P.Ntot),
+             (float)((double)n / (double)P.Ntot * (double)P.lambda), P.H, P.F, tc.i0, tc.j0, nt};
+  umma::gemm_tn_tile(&tmD, &tmXT, nt, tc, &P.sc->err, epi);
+}
+
 struct HostPlan {
   MlpDev d;
   size_t fwd_smem;
+  char* scratch_tc = nullptr;
+  std::vector<long long> N_host, offT_host;
+  bool tc = false;          // tensor-core path in use
+  int nt1 = 0, nt2 = 0;     // N tiles of the two products
+  CUtensorMap tmX, tmW, tmD, tmXT;
 };
 
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
@@ -330,6 +451,14 @@ size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 int forward_blocks_per_worker(int M) {
   int g = (2 * kNumSMs + M - 1) / M;
   return g < 1 ? 1 : (g > 64 ? 64 : g);
+}
+
+// the tcgen05 path needs 16-byte row pitches for its tensor maps
+bool tc_shape_ok(int F, int H) { return (F % 8) == 0 && (H % 8) == 0 && H >= 16 && H <= 256; }
+
+size_t forward_smem_tc(int H) {
+  const int CG = H / 8, RG = kThreads / CG, TR = 4 * RG;
+  return (size_t)TR * H * 4 + (size_t)TR * kMaxC * 4;
 }
 
 size_t forward_smem(int F, int H) {
@@ -358,6 +487,15 @@ size_t mlp_scratch_bytes(const laq_config& c) {
   b += align256((size_t)c.M * gb * nsmall * 4);                  // spart
   b += align256((size_t)c.M * gb * 8);                           // lpart
   b += align256((size_t)(c.M + 1) * 8);                          // rowoff
+  if (tc_shape_ok(c.n_features, c.n_hidden)) {
+    long long ldT = 0;
+    for (int m = 0; m < c.M; ++m) ldT += (c.N[m] + 63) / 64 * 64;
+    b += align256((size_t)c.n_hidden * c.n_features * 2);        // W1b
+    b += align256((size_t)Ntot * c.n_hidden * 4);                // Hbuf
+    b += align256((size_t)c.n_hidden * ldT * 2);                 // dHT
+    b += align256((size_t)c.n_features * ldT * 2);               // XbT
+    b += align256((size_t)(c.M + 1) * 8);                        // rowoffT
+  }
   return b;
 }
 
@@ -371,12 +509,13 @@ laq_status mlp_setup(MlpPlan& mp, const Params& P, void* scratch, cudaStream_t s
   hp->d.dHb = (__nv_bfloat16*)p; p += align256((size_t)P.Ntot * P.H * 2);
   hp->d.spart = (float*)p; p += align256((size_t)P.M * hp->d.gb * nsmall * 4);
   hp->d.lpart = (double*)p; p += align256((size_t)P.M * hp->d.gb * 8);
-  hp->d.rowoff = (long long*)p;
+  hp->d.rowoff = (long long*)p; p += align256((size_t)(P.M + 1) * 8);
   hp->fwd_smem = forward_smem(P.F, P.H);
+  hp->scratch_tc = p;
   // prefix sums of the shard sizes (N is not yet on the device when this runs, so it comes from the host copy)
   mp.scratch = hp;
   mp.ready = 0;
-  if (cudaFuncSetAttribute(mlp_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hp->fwd_smem) !=
+  if (cudaFuncSetAttribute(mlp_forward_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hp->fwd_smem) !=
       cudaSuccess)
     return LAQ_ECUDA;
   (void)st;
@@ -391,6 +530,52 @@ laq_status mlp_set_row_offsets(MlpPlan& mp, const long long* N_host, int M, cuda
   if (cudaMemcpyAsync(hp->d.rowoff, off, sizeof(long long) * (M + 1), cudaMemcpyHostToDevice, st) != cudaSuccess)
     return LAQ_ECUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return LAQ_ECUDA;
+  hp->N_host.assign(N_host, N_host + M);
+  return LAQ_OK;
+}
+
+// Tensor-core path: carve its buffers, zero the transposed copies (their padding columns must stay zero), build
+// the four tensor maps.  Falls back to the plain kernels if the shape does not fit or a map cannot be made.
+laq_status mlp_setup_tensor_path(MlpPlan& mp, const Params& P, cudaStream_t st) {
+  HostPlan* hp = (HostPlan*)mp.scratch;
+  hp->tc = false;
+  if (!tc_shape_ok(P.F, P.H)) return LAQ_OK;
+  const int M = P.M;
+  long long offT[1025];
+  offT[0] = 0;
+  for (int m = 0; m < M; ++m) offT[m + 1] = offT[m] + (hp->N_host[m] + 63) / 64 * 64;
+  const long long ldT = offT[M];
+  if (ldT >= (1ll << 31) || P.Ntot >= (1ll << 31)) return LAQ_OK;
+  char* p = hp->scratch_tc;
+  hp->d.W1b = (__nv_bfloat16*)p; p += align256((size_t)P.H * P.F * 2);
+  hp->d.Hbuf = (float*)p; p += align256((size_t)P.Ntot * P.H * 4);
+  hp->d.dHT = (__nv_bfloat16*)p; p += align256((size_t)P.H * ldT * 2);
+  hp->d.XbT = (__nv_bfloat16*)p; p += align256((size_t)P.F * ldT * 2);
+  hp->d.rowoffT = (long long*)p;
+  hp->d.ldT = ldT;
+  hp->nt1 = (P.H + 15) / 16 * 16;
+  hp->nt2 = (P.F % 112 == 0) ? 112 : ((P.F >= 128) ? 128 : (P.F + 15) / 16 * 16);
+  if (cudaMemsetAsync(hp->d.dHT, 0, (size_t)P.H * ldT * 2, st) != cudaSuccess) return LAQ_ECUDA;
+  if (cudaMemsetAsync(hp->d.XbT, 0, (size_t)P.F * ldT * 2, st) != cudaSuccess) return LAQ_ECUDA;
+  if (cudaMemcpyAsync(hp->d.rowoffT, offT, sizeof(long long) * (M + 1), cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return LAQ_ECUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return LAQ_ECUDA;
+  bool ok = umma::make_map_bf16_2d(&hp->tmX, hp->d.Xb, (uint64_t)P.Ntot, (uint64_t)P.F, (uint64_t)P.F * 2, umma::kTileM);
+  ok = ok && umma::make_map_bf16_2d(&hp->tmW, hp->d.W1b, (uint64_t)P.H, (uint64_t)P.F, (uint64_t)P.F * 2, hp->nt1);
+  ok = ok && umma::make_map_bf16_2d(&hp->tmD, hp->d.dHT, (uint64_t)P.H, (uint64_t)ldT, (uint64_t)ldT * 2, umma::kTileM);
+  ok = ok && umma::make_map_bf16_2d(&hp->tmXT, hp->d.XbT, (uint64_t)P.F, (uint64_t)ldT, (uint64_t)ldT * 2, hp->nt2);
+  if (!ok) return LAQ_OK;   // plain kernels
+  if (cudaFuncSetAttribute(umma_hidden_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)umma::smem_bytes(hp->nt1)) != cudaSuccess ||
+      cudaFuncSetAttribute(umma_dw1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)umma::smem_bytes(hp->nt2)) != cudaSuccess ||
+      cudaFuncSetAttribute(mlp_forward_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)forward_smem_tc(P.H)) != cudaSuccess) {
+    cudaGetLastError();
+    return LAQ_OK;
+  }
+  hp->offT_host.assign(offT, offT + M + 1);
+  hp->tc = true;
   return LAQ_OK;
 }
 
@@ -399,17 +584,29 @@ int mlp_convert_shard(MlpPlan& mp, const Params& P, int m, const float* X, long 
   HostPlan* hp = (HostPlan*)mp.scratch;
   const long long cnt = n * P.F;
   mlp_pack_x_kernel<<<kNumSMs * 4, 256, 0, st>>>(X, hp->d.Xb + row_offset * P.F, cnt);
-  (void)m;
-  return 1;
+  if (!hp->tc) return 1;
+  mlp_transpose_x_kernel<<<dim3((unsigned)((n + 31) / 32), (unsigned)((P.F + 31) / 32)), 256, 0, st>>>(
+      X, hp->d.XbT, n, P.F, hp->d.ldT, hp->offT_host[m]);
+  return 2;
 }
 
 int mlp_launch_gradients(MlpPlan& mp, const Params& P, const double* theta_sq, cudaStream_t st) {
   HostPlan* hp = (HostPlan*)mp.scratch;
   const int F = P.F, H = P.H, C = P.C;
-  mlp_pack_w1_kernel<<<(F * H + 255) / 256, 256, 0, st>>>(P.theta, hp->d.W1T, F, H);
-  mlp_forward_kernel<<<dim3(hp->d.gb, P.M), kThreads, hp->fwd_smem, st>>>(P, hp->d);
-  mlp_dw1_kernel<<<dim3((F + kTK - 1) / kTK, (H + kTJ - 1) / kTJ, P.M), kThreads, 0, st>>>(P, hp->d);
   const int nsmall = H + C * H + C;
+  if (hp->tc) {
+    mlp_pack_w1b_kernel<<<(F * H + 255) / 256, 256, 0, st>>>(P.theta, hp->d.W1b, F * H);
+    umma_hidden_kernel<<<(unsigned)((P.Ntot + umma::kTileM - 1) / umma::kTileM), umma::kThreads,
+                         umma::smem_bytes(hp->nt1), st>>>(hp->tmX, hp->tmW, P, hp->d, hp->nt1);
+    mlp_forward_kernel<true><<<dim3(hp->d.gb, P.M), kThreads, forward_smem_tc(H), st>>>(P, hp->d);
+    umma_dw1_kernel<<<dim3((F + hp->nt2 - 1) / hp->nt2, (H + umma::kTileM - 1) / umma::kTileM, P.M), umma::kThreads,
+                      umma::smem_bytes(hp->nt2), st>>>(hp->tmD, hp->tmXT, P, hp->d, hp->nt2);
+    mlp_finalize_kernel<<<dim3((nsmall + 255) / 256, P.M), 256, 0, st>>>(P, hp->d, theta_sq);
+    return 5;
+  }
+  mlp_pack_w1_kernel<<<(F * H + 255) / 256, 256, 0, st>>>(P.theta, hp->d.W1T, F, H);
+  mlp_forward_kernel<false><<<dim3(hp->d.gb, P.M), kThreads, hp->fwd_smem, st>>>(P, hp->d);
+  mlp_dw1_kernel<<<dim3((F + kTK - 1) / kTK, (H + kTJ - 1) / kTJ, P.M), kThreads, 0, st>>>(P, hp->d);
   mlp_finalize_kernel<<<dim3((nsmall + 255) / 256, P.M), 256, 0, st>>>(P, hp->d, theta_sq);
   return 4;
 }
