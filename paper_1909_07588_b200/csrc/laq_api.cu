@@ -320,7 +320,7 @@ laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, siz
     LAQ_CUDA(ctx, cudaMemcpyAsync(ws + pl.yptr, ctx->yptr.data(), 8 * (size_t)c.M, cudaMemcpyHostToDevice, ctx->st));
     LAQ_CUDA(ctx, cudaMemcpyAsync(ws + pl.Ndev, ctx->N.data(), 8 * (size_t)c.M, cudaMemcpyHostToDevice, ctx->st));
     if (c.model == LAQ_MODEL_MLP2) {
-      laq_status s = mlp_setup(ctx->mlp, P, ws + pl.mlp, ctx->st);
+      laq_status s = mlp_setup(ctx->mlp, P, (const long long*)ctx->N.data(), ws + pl.mlp, ctx->st);
       if (s == LAQ_OK) s = mlp_set_row_offsets(ctx->mlp, (const long long*)ctx->N.data(), c.M, ctx->st);
       if (s == LAQ_OK) s = mlp_setup_tensor_path(ctx->mlp, P, ctx->st);
       if (s != LAQ_OK) return fail(ctx, s, "network scratch set-up failed");

@@ -401,7 +401,201 @@ __global__ void __launch_bounds__(umma::kThreads) umma_hidden_kernel(const __gri
                                                                      const __grid_constant__ CUtensorMap tmW,
                                                                      const Params P, const MlpDev D, int nt) {
   umma::TileCoord tc{(int)blockIdx.x * umma::kTileM, 0, 0, (P.F + umma::kBlockK - 1) / umma::kBlockK};
-  HiddenEpi epi{D.Hbuf, P.theta + (long long)P.H * P.F, P.Ntot, P.H, tc.i0};
+  umma::ChunkEpilogue<HiddenEpi> epi{HiddenEpi{D.Hbuf, P.theta + (long long)P.H * P.F, P.Ntot, P.H, tc.i0}, nt};
+  umma::gemm_tn_tile(&tmX, &tmW, nt, tc, &P.sc->err, epi);
+}
+
+// Fused epilogue of the hidden product: from the accumulator tile (thread = row) straight to the loss, dZ, the
+// bf16 dH~ (stored transposed: consecutive lanes = consecutive rows = consecutive addresses) and the tile's
+// contributions to the b1 / W2 / b2 gradients, without writing the hidden activations to memory.
+//   pass 1  h = relu(acc + b1); scores z += h W2^T chunk by chunk; softmax, loss, dZ (kept in registers)
+//   pass 2  the accumulator is read again from tensor memory: dh = (dZ W2) o [h > 0] -> bf16 -> dH~^T; the h chunk
+//           goes through shared memory so that a thread per column can sum over the tile's rows
+//               A[c][j] = sum_r dZ[r][c] h[r][j]         (the W2 gradient)
+//               S[c][j] = sum_r dZ[r][c] [h[r][j] > 0]   (then db1[j] = sum_c W2[c][j] S[c][j])
+//           in a fixed order (no atomics).
+__host__ __device__ inline size_t fused_extra_floats(int H) {
+  return (size_t)H * 12 + (size_t)((H + 3) & ~3) + 128 * 33 + 128 * 12 + 2 * (size_t)12 * H + 16;
+}
+
+struct FusedEpi {
+  const Params& P;
+  const MlpDev& D;
+  int nt, m, tile;          // worker and tile index within the worker
+  __device__ __forceinline__ void run(uint32_t tmem_base, int q, int lane) {
+    const int H = P.H, C = P.C, F = P.F;
+    const int tt = q * 32 + lane;            // 0..127: the tile row this thread owns
+    float* base = reinterpret_cast<float*>(umma::extra_smem(nt));
+    float* w2t = base;                       // [H][12]   W2 transposed (j-major), padded rows of 12
+    float* b1s = w2t + (size_t)H * 12;       // [H]
+    float* chunk = b1s + ((H + 3) & ~3);     // [128][33] one 32-column chunk of h
+    float* dzs = chunk + 128 * 33;           // [128][12]
+    float* accA = dzs + 128 * 12;            // [12][H]
+    float* accS = accA + (size_t)12 * H;     // [12][H]
+    double* lossw = reinterpret_cast<double*>(accS + (size_t)12 * H);      // [4] (8-byte aligned: all sizes even)
+    float* red = chunk;                      // [4][2 C][32] partial column sums, reuses the chunk buffer
+    const float* __restrict__ theta = P.theta;
+    const float* __restrict__ b1 = theta + (long long)H * F;
+    const float* __restrict__ W2 = b1 + H;
+    const float* __restrict__ b2 = W2 + (long long)C * H;
+    for (int i = tt; i < H * 12; i += 128) {
+      const int j = i / 12, c = i - 12 * j;
+      w2t[i] = (c < C) ? __ldg(W2 + (size_t)c * H + j) : 0.f;
+    }
+    for (int i = tt; i < H; i += 128) b1s[i] = __ldg(b1 + i);
+    umma::epilogue_sync();
+    const long long n = P.N[m];
+    const long long trow = (long long)tile * umma::kTileM + tt;   // row within the worker's shard
+    const bool valid = trow < n;
+    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+    // ---- pass 1
+    float z[12];
+#pragma unroll
+    for (int c = 0; c < 12; ++c) z[c] = 0.f;
+    for (int c0 = 0; c0 < nt; c0 += 32) {
+      uint32_t v[32];
+      umma::tmem_load_32(taddr + (uint32_t)c0, v);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const int j = c0 + i;
+        if (j < H) {
+          const float h = fmaxf(__uint_as_float(v[i]) + b1s[j], 0.f);
+          const float4 wa = *reinterpret_cast<const float4*>(w2t + j * 12);
+          const float4 wb = *reinterpret_cast<const float4*>(w2t + j * 12 + 4);
+          const float4 wc = *reinterpret_cast<const float4*>(w2t + j * 12 + 8);
+          z[0] = fmaf(h, wa.x, z[0]); z[1] = fmaf(h, wa.y, z[1]); z[2] = fmaf(h, wa.z, z[2]); z[3] = fmaf(h, wa.w, z[3]);
+          z[4] = fmaf(h, wb.x, z[4]); z[5] = fmaf(h, wb.y, z[5]); z[6] = fmaf(h, wb.z, z[6]); z[7] = fmaf(h, wb.w, z[7]);
+          z[8] = fmaf(h, wc.x, z[8]); z[9] = fmaf(h, wc.y, z[9]); z[10] = fmaf(h, wc.z, z[10]); z[11] = fmaf(h, wc.w, z[11]);
+        }
+      }
+    }
+    float dz[12];
+    double loss = 0.0;
+    {
+      float zmax = -3.0e38f;
+#pragma unroll
+      for (int c = 0; c < 12; ++c)
+        if (c < C) {
+          z[c] += __ldg(b2 + c);
+          zmax = fmaxf(zmax, z[c]);
+        }
+      float e[12], sum = 0.f;
+#pragma unroll
+      for (int c = 0; c < 12; ++c) {
+        e[c] = (c < C) ? expf(z[c] - zmax) : 0.f;
+        sum += e[c];
+      }
+      const int yv = valid ? P.y[m][trow] : -1;
+      const float inv = 1.0f / sum;
+      float zy = 0.f;
+#pragma unroll
+      for (int c = 0; c < 12; ++c) {
+        if (c == yv) zy = z[c];
+        dz[c] = (valid && c < C) ? (e[c] * inv - (c == yv ? 1.f : 0.f)) : 0.f;
+        dzs[tt * 12 + c] = dz[c];
+      }
+      if (valid) loss = (double)((zmax + logf(sum)) - zy);
+    }
+    // ---- pass 2
+    const long long col = D.rowoffT[m] + trow;
+    const bool in_segment = col < D.rowoffT[m + 1];        // rows of the padded segment (zeros beyond the shard)
+    const int rq = tt >> 5, cl = tt & 31;                  // reduce phase: column cl, rows 32 rq .. 32 rq + 31
+    for (int c0 = 0; c0 < nt; c0 += 32) {
+      uint32_t v[32];
+      umma::tmem_load_32(taddr + (uint32_t)c0, v);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const int j = c0 + i;
+        float h = 0.f;
+        if (j < H) {
+          h = fmaxf(__uint_as_float(v[i]) + b1s[j], 0.f);
+          const float4 wa = *reinterpret_cast<const float4*>(w2t + j * 12);
+          const float4 wb = *reinterpret_cast<const float4*>(w2t + j * 12 + 4);
+          const float4 wc = *reinterpret_cast<const float4*>(w2t + j * 12 + 8);
+          float d = dz[0] * wa.x;
+          d = fmaf(dz[1], wa.y, d); d = fmaf(dz[2], wa.z, d); d = fmaf(dz[3], wa.w, d);
+          d = fmaf(dz[4], wb.x, d); d = fmaf(dz[5], wb.y, d); d = fmaf(dz[6], wb.z, d); d = fmaf(dz[7], wb.w, d);
+          d = fmaf(dz[8], wc.x, d); d = fmaf(dz[9], wc.y, d); d = fmaf(dz[10], wc.z, d); d = fmaf(dz[11], wc.w, d);
+          const float dh = h > 0.f ? d : 0.f;
+          if (in_segment) D.dHT[(long long)j * D.ldT + col] = __float2bfloat16_rn(dh);
+        }
+        chunk[tt * 33 + i] = h;
+      }
+      umma::epilogue_sync();
+      {  // column sums over this thread's 32 rows
+        float a[12], sgn[12];
+#pragma unroll
+        for (int c = 0; c < 12; ++c) a[c] = sgn[c] = 0.f;
+        for (int r = 32 * rq; r < 32 * rq + 32; ++r) {
+          const float h = chunk[r * 33 + cl];
+          const float pos = h > 0.f ? 1.f : 0.f;
+          const float4 da = *reinterpret_cast<const float4*>(dzs + r * 12);
+          const float4 db = *reinterpret_cast<const float4*>(dzs + r * 12 + 4);
+          const float4 dc = *reinterpret_cast<const float4*>(dzs + r * 12 + 8);
+          const float dv[12] = {da.x, da.y, da.z, da.w, db.x, db.y, db.z, db.w, dc.x, dc.y, dc.z, dc.w};
+#pragma unroll
+          for (int c = 0; c < 12; ++c) {
+            a[c] = fmaf(dv[c], h, a[c]);
+            sgn[c] = fmaf(dv[c], pos, sgn[c]);
+          }
+        }
+        umma::epilogue_sync();      // everybody has read the chunk: reuse it for the partial sums
+#pragma unroll
+        for (int c = 0; c < 12; ++c) {
+          red[(rq * 24 + c) * 32 + cl] = a[c];
+          red[(rq * 24 + 12 + c) * 32 + cl] = sgn[c];
+        }
+      }
+      umma::epilogue_sync();
+      for (int i = tt; i < 24 * 32; i += 128) {   // fixed order over the four row quarters
+        const int k = i >> 5, cc = i & 31, j = c0 + cc;
+        if (j < H) {
+          const float sum4 = ((red[(0 * 24 + k) * 32 + cc] + red[(1 * 24 + k) * 32 + cc]) + red[(2 * 24 + k) * 32 + cc]) +
+                             red[(3 * 24 + k) * 32 + cc];
+          if (k < 12) accA[k * H + j] = sum4; else accS[(k - 12) * H + j] = sum4;
+        }
+      }
+      umma::epilogue_sync();
+    }
+    // ---- the tile's partials: [db1 (H) | dW2 (C H) | db2 (C)] and the loss
+    const int gb = D.gb;
+    float* sp = D.spart + ((long long)m * gb + tile) * (H + C * H + C);
+    for (int j = tt; j < H; j += 128) {
+      float s = 0.f;
+      for (int c = 0; c < C; ++c) s = fmaf(w2t[j * 12 + c], accS[c * H + j], s);
+      sp[j] = s;
+      for (int c = 0; c < C; ++c) sp[H + c * H + j] = accA[c * H + j];
+    }
+    if (tt < C) {
+      float s = 0.f;
+      for (int r = 0; r < 128; ++r) s += dzs[r * 12 + tt];
+      sp[H + C * H + tt] = s;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, o);
+    if (lane == 0) lossw[q] = loss;
+    umma::epilogue_sync();
+    if (tt == 0) D.lpart[(long long)m * gb + tile] = ((lossw[0] + lossw[1]) + lossw[2]) + lossw[3];
+  }
+};
+
+// grid: (tiles per worker, M); tile t of worker m covers the worker's rows 128 t .. 128 t + 127
+__global__ void __launch_bounds__(umma::kThreads) umma_hidden_fused_kernel(const __grid_constant__ CUtensorMap tmX,
+                                                                           const __grid_constant__ CUtensorMap tmW,
+                                                                           const Params P, const MlpDev D, int nt) {
+  const int m = blockIdx.y, tile = blockIdx.x;
+  const long long n = P.N[m];
+  const bool has_rows = (long long)tile * umma::kTileM < n;
+  umma::TileCoord tc{(int)(D.rowoff[m] + (long long)tile * umma::kTileM), 0, 0,
+                     has_rows ? (P.F + umma::kBlockK - 1) / umma::kBlockK : 0};
+  if (!has_rows) {   // a worker with fewer tiles than the grid: its slot holds zeros
+    const int nsmall = P.H + P.C * P.H + P.C;
+    float* sp = D.spart + ((long long)m * D.gb + tile) * nsmall;
+    for (int i = threadIdx.x; i < nsmall; i += blockDim.x) sp[i] = 0.f;
+    if (threadIdx.x == 0) D.lpart[(long long)m * D.gb + tile] = 0.0;
+    return;
+  }
+  FusedEpi epi{P, D, nt, m, tile};
   umma::gemm_tn_tile(&tmX, &tmW, nt, tc, &P.sc->err, epi);
 }
 
@@ -431,8 +625,10 @@ __global__ void __launch_bounds__(umma::kThreads) umma_dw1_kernel(const __grid_c
   const long long c0 = D.rowoffT[m], c1 = D.rowoffT[m + 1];
   umma::TileCoord tc{(int)blockIdx.y * umma::kTileM, (int)blockIdx.x * nt, (int)c0, (int)((c1 - c0) / umma::kBlockK)};
   const long long n = P.N[m];
-  Dw1Epi epi{P.g + (long long)m * P.ps, P.theta, (float)(1.0 / (double)P.Ntot),
-             (float)((double)n / (double)P.Ntot * (double)P.lambda), P.H, P.F, tc.i0, tc.j0, nt};
+  umma::ChunkEpilogue<Dw1Epi> epi{Dw1Epi{P.g + (long long)m * P.ps, P.theta, (float)(1.0 / (double)P.Ntot),
+                                         (float)((double)n / (double)P.Ntot * (double)P.lambda), P.H, P.F, tc.i0,
+                                         tc.j0, nt},
+                                  nt};
   umma::gemm_tn_tile(&tmD, &tmXT, nt, tc, &P.sc->err, epi);
 }
 
@@ -443,6 +639,7 @@ struct HostPlan {
   std::vector<long long> N_host, offT_host;
   bool tc = false;          // tensor-core path in use
   int nt1 = 0, nt2 = 0;     // N tiles of the two products
+  int fused_tiles = 0;      // > 0: the hidden product runs with the fused epilogue, this many tiles per worker
   CUtensorMap tmX, tmW, tmD, tmXT;
 };
 
@@ -459,6 +656,19 @@ bool tc_shape_ok(int F, int H) { return (F % 8) == 0 && (H % 8) == 0 && H >= 16 
 size_t forward_smem_tc(int H) {
   const int CG = H / 8, RG = kThreads / CG, TR = 4 * RG;
   return (size_t)TR * H * 4 + (size_t)TR * kMaxC * 4;
+}
+
+// tiles per worker of the fused hidden kernel, or 0 if the fused epilogue cannot be used for this shape
+int fused_tiles_for(int F, int H, int C, const long long* N, int M) {
+  if (!tc_shape_ok(F, H) || C > 12) return 0;
+  const int nt1 = (H + 15) / 16 * 16;
+  if (umma::smem_bytes(nt1) + fused_extra_floats(H) * 4 > 226 * 1024) return 0;
+  long long tiles = 0;
+  for (int m = 0; m < M; ++m) {
+    const long long t = (N[m] + umma::kTileM - 1) / umma::kTileM;
+    if (t > tiles) tiles = t;
+  }
+  return tiles <= 256 ? (int)tiles : 0;
 }
 
 size_t forward_smem(int F, int H) {
@@ -478,7 +688,9 @@ const char* mlp_check_shape(int F, int H, int C) {
 size_t mlp_scratch_bytes(const laq_config& c) {
   long long Ntot = 0;
   for (int m = 0; m < c.M; ++m) Ntot += c.N[m];
-  const int gb = forward_blocks_per_worker(c.M);
+  std::vector<long long> Nv(c.N, c.N + c.M);
+  const int ft = fused_tiles_for(c.n_features, c.n_hidden, c.n_classes, Nv.data(), c.M);
+  const int gb = ft > forward_blocks_per_worker(c.M) ? ft : forward_blocks_per_worker(c.M);
   const size_t nsmall = (size_t)c.n_hidden + (size_t)c.n_classes * c.n_hidden + c.n_classes;
   size_t b = 0;
   b += align256((size_t)c.n_features * c.n_hidden * 2);          // W1T
@@ -499,16 +711,18 @@ size_t mlp_scratch_bytes(const laq_config& c) {
   return b;
 }
 
-laq_status mlp_setup(MlpPlan& mp, const Params& P, void* scratch, cudaStream_t st) {
+laq_status mlp_setup(MlpPlan& mp, const Params& P, const long long* N_host, void* scratch, cudaStream_t st) {
   HostPlan* hp = new HostPlan();
+  const int ft = fused_tiles_for(P.F, P.H, P.C, N_host, P.M);
+  const int gb_alloc = ft > forward_blocks_per_worker(P.M) ? ft : forward_blocks_per_worker(P.M);
   char* p = (char*)scratch;
   const size_t nsmall = (size_t)P.H + (size_t)P.C * P.H + P.C;
   hp->d.gb = forward_blocks_per_worker(P.M);
   hp->d.W1T = (__nv_bfloat16*)p; p += align256((size_t)P.F * P.H * 2);
   hp->d.Xb = (__nv_bfloat16*)p; p += align256((size_t)P.Ntot * P.F * 2);
   hp->d.dHb = (__nv_bfloat16*)p; p += align256((size_t)P.Ntot * P.H * 2);
-  hp->d.spart = (float*)p; p += align256((size_t)P.M * hp->d.gb * nsmall * 4);
-  hp->d.lpart = (double*)p; p += align256((size_t)P.M * hp->d.gb * 8);
+  hp->d.spart = (float*)p; p += align256((size_t)P.M * gb_alloc * nsmall * 4);
+  hp->d.lpart = (double*)p; p += align256((size_t)P.M * gb_alloc * 8);
   hp->d.rowoff = (long long*)p; p += align256((size_t)(P.M + 1) * 8);
   hp->fwd_smem = forward_smem(P.F, P.H);
   hp->scratch_tc = p;
@@ -576,6 +790,14 @@ laq_status mlp_setup_tensor_path(MlpPlan& mp, const Params& P, cudaStream_t st) 
   }
   hp->offT_host.assign(offT, offT + M + 1);
   hp->tc = true;
+  const int ft = fused_tiles_for(P.F, P.H, P.C, hp->N_host.data(), M);
+  if (ft > 0 && cudaFuncSetAttribute(umma_hidden_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)(umma::smem_bytes(hp->nt1) + fused_extra_floats(P.H) * 4)) == cudaSuccess) {
+    hp->fused_tiles = ft;
+    hp->d.gb = ft;        // one partial slot per tile
+  } else {
+    cudaGetLastError();
+  }
   return LAQ_OK;
 }
 
@@ -596,6 +818,15 @@ int mlp_launch_gradients(MlpPlan& mp, const Params& P, const double* theta_sq, c
   const int nsmall = H + C * H + C;
   if (hp->tc) {
     mlp_pack_w1b_kernel<<<(F * H + 255) / 256, 256, 0, st>>>(P.theta, hp->d.W1b, F * H);
+    if (hp->fused_tiles > 0) {
+      umma_hidden_fused_kernel<<<dim3(hp->fused_tiles, P.M), umma::kThreads,
+                                 umma::smem_bytes(hp->nt1) + fused_extra_floats(H) * 4, st>>>(hp->tmX, hp->tmW, P, hp->d,
+                                                                                              hp->nt1);
+      umma_dw1_kernel<<<dim3((F + hp->nt2 - 1) / hp->nt2, (H + umma::kTileM - 1) / umma::kTileM, P.M), umma::kThreads,
+                        umma::smem_bytes(hp->nt2), st>>>(hp->tmD, hp->tmXT, P, hp->d, hp->nt2);
+      mlp_finalize_kernel<<<dim3((nsmall + 255) / 256, P.M), 256, 0, st>>>(P, hp->d, theta_sq);
+      return 4;
+    }
     umma_hidden_kernel<<<(unsigned)((P.Ntot + umma::kTileM - 1) / umma::kTileM), umma::kThreads,
                          umma::smem_bytes(hp->nt1), st>>>(hp->tmX, hp->tmW, P, hp->d, hp->nt1);
     mlp_forward_kernel<true><<<dim3(hp->d.gb, P.M), kThreads, forward_smem_tc(H), st>>>(P, hp->d);

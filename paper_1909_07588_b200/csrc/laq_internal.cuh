@@ -102,7 +102,7 @@ struct MlpPlan {
 };
 const char* mlp_check_shape(int F, int H, int C);   // null if supported, else the reason
 size_t mlp_scratch_bytes(const laq_config& c);
-laq_status mlp_setup(MlpPlan& mp, const Params& P, void* scratch, cudaStream_t st);
+laq_status mlp_setup(MlpPlan& mp, const Params& P, const long long* N_host, void* scratch, cudaStream_t st);
 laq_status mlp_set_row_offsets(MlpPlan& mp, const long long* N_host, int M, cudaStream_t st);
 laq_status mlp_setup_tensor_path(MlpPlan& mp, const Params& P, cudaStream_t st);
 int mlp_convert_shard(MlpPlan& mp, const Params& P, int m, const float* X, long long n, long long row_offset,

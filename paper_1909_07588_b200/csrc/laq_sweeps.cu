@@ -258,6 +258,7 @@ __device__ void trigger_stage(const Params& P, int bpw) {
   for (int m = threadIdx.x; m < P.M; m += blockDim.x) {
     double n_dq = 0.0, n_eps = 0.0;
     const double* pq = P.part_q + (long long)m * kMaxSweepBlocksPerWorker * 2;
+#pragma unroll 8
     for (int i = 0; i < bpw; ++i) {  // fixed order
       n_dq += __ldcg(pq + 2 * i);
       n_eps += __ldcg(pq + 2 * i + 1);
@@ -577,7 +578,8 @@ void launch_quant_b(const Params& P, dim3 grid, int threads, cudaStream_t st) {
 int sweep_blocks_per_worker(const Params& P, const LaunchShape& ls) {
   // one resident wave: M x bpw blocks ~ SMs x blocks per SM, never more blocks than 16-byte groups
   long long want = ((long long)kNumSMs * ls.sweep_blocks_per_sm + P.M - 1) / P.M;
-  long long need = (P.nv + ls.sweep_threads - 1) / ls.sweep_threads;
+  // a thread should have at least 8 groups of 16 bytes: below that the per-block reductions dominate
+  long long need = (P.nv + 8ll * ls.sweep_threads - 1) / (8ll * ls.sweep_threads);
   long long bpw = want < need ? want : need;
   if (bpw < 1) bpw = 1;
   if (bpw > kMaxSweepBlocksPerWorker) bpw = kMaxSweepBlocksPerWorker;

@@ -118,9 +118,38 @@ struct TileCoord {
   int i0, j0, k0, nkb;
 };
 
-// Epi::operator()(row_in_tile, col0, const float (&acc)[32]) is called by the thread that owns accumulator row
+// Epi::run(tmem_base, q, lane) is executed by the four epilogue warps once the accumulator is complete; warp
+// quarter q (0..3) may read TMEM lanes 32 q .. 32 q + 31, i.e. accumulator rows 32 q + lane.  The epilogue warps
+// are threads 64..191 of the block; they may synchronise among themselves with named barrier 1 (128 threads).
+__device__ __forceinline__ void epilogue_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// Shared memory that follows the stage ring (for an epilogue's own buffers); pass the extra bytes at launch.
+__device__ __forceinline__ unsigned char* extra_smem(int nt) {
+  extern __shared__ unsigned char umma_smem_raw[];
+  const uint32_t base = smem_u32(umma_smem_raw);
+  const uint32_t aligned = (base + 1023u) & ~1023u;
+  return umma_smem_raw + (aligned - base) + kStages * stage_bytes(nt);
+}
+
+// Adapter: f(row_in_tile, col0, const float (&acc)[32]) is called by the thread that owns accumulator row
 // `row_in_tile` (0..127) for the 32-column chunks col0 = 0, 32, ... < NT.  The last chunk may reach past NT:
-// entries at columns >= NT are undefined and the functor must ignore them.
+// entries at columns >= NT are undefined and f must ignore them.
+template <class F>
+struct ChunkEpilogue {
+  F f;
+  int nt;
+  __device__ __forceinline__ void run(uint32_t tmem_base, int q, int lane) {
+    for (int c0 = 0; c0 < nt; c0 += 32) {
+      uint32_t v[32];
+      tmem_load_32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+      float acc[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) acc[i] = __uint_as_float(v[i]);
+      f(q * 32 + lane, c0, acc);
+    }
+  }
+};
+
 template <class Epi>
 __device__ __forceinline__ void gemm_tn_tile(const CUtensorMap* tmA, const CUtensorMap* tmB, int nt, TileCoord tc,
                                              uint32_t* err_flag, Epi& epi) {
@@ -184,16 +213,12 @@ __device__ __forceinline__ void gemm_tn_tile(const CUtensorMap* tmA, const CUten
     const int q = warp & 3;                         // the TMEM lane quarter this warp may read
     const bool ok = __all_sync(0xffffffffu, mbar_wait(accum, 0u, err_flag, 8u));
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (ok && tc.nkb > 0) {
-      for (int c0 = 0; c0 < nt; c0 += 32) {
-        uint32_t v[32];
-        tmem_load_32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
-        float acc[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) acc[i] = __uint_as_float(v[i]);
-        epi(q * 32 + lane, c0, acc);
-      }
-    }
+    // all four epilogue warps take the same branch (the verdicts are combined), so an epilogue may use
+    // its named barrier
+    __shared__ int epi_ok[4];
+    if (lane == 0) epi_ok[q] = (ok && tc.nkb > 0) ? 1 : 0;
+    epilogue_sync();
+    if (epi_ok[0] & epi_ok[1] & epi_ok[2] & epi_ok[3]) epi.run(tmem_base, q, lane);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
