@@ -306,6 +306,12 @@ laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, siz
   for (int m = 0; m < c.M; ++m) P.Ntot += ctx->N[m];
   ctx->gbpw_cap = pl.gbpw_cap;
   ctx->gbpw = default_gbpw(c);
+  if (c.model == LAQ_MODEL_LOGREG_BIN || c.model == LAQ_MODEL_SOFTMAX) {
+    long long n_max = 1;
+    for (int m = 0; m < c.M; ++m) n_max = ctx->N[m] > n_max ? ctx->N[m] : n_max;
+    const int tiles = grad_tiles_per_worker(c.model, c.n_features, n_max);
+    if (ctx->gbpw > tiles) ctx->gbpw = tiles;
+  }
 
   LAQ_CUDA(ctx, cudaMemsetAsync(ws, 0, pl.state_end, ctx->st));
   if (needs_shards(ctx)) {
@@ -393,14 +399,19 @@ laq_status laq_step(laq_ctx* ctx, int32_t n_iters, const laq_trace* trace) {
       cudaEventRecord(ev[0], ctx->st);
     }
     const int64_t l0 = ctx->launches;
+    // small problems: steps 2-5 (and, when cheap, the combination of the gradient kernels' block partials)
+    // run in one single-block kernel
+    const bool small = small_iteration_applies(P);
+    const bool linear = c.model == LAQ_MODEL_LOGREG_BIN || c.model == LAQ_MODEL_SOFTMAX;
+    const bool fuse_finalize = small && linear && ctx->gbpw <= 8;
     switch (c.model) {
       case LAQ_MODEL_LOGREG_BIN:
         ctx->launches += launch_grad_logreg(P, ctx->ls, ctx->gbpw, ctx->st);
-        ctx->launches += launch_grad_finalize(P, ctx->gbpw, &P.sc->theta_sq, ctx->st);
+        if (!fuse_finalize) ctx->launches += launch_grad_finalize(P, ctx->gbpw, &P.sc->theta_sq, ctx->st);
         break;
       case LAQ_MODEL_SOFTMAX:
         ctx->launches += launch_grad_softmax(P, ctx->ls, ctx->gbpw, ctx->st);
-        ctx->launches += launch_grad_finalize(P, ctx->gbpw, &P.sc->theta_sq, ctx->st);
+        if (!fuse_finalize) ctx->launches += launch_grad_finalize(P, ctx->gbpw, &P.sc->theta_sq, ctx->st);
         break;
       case LAQ_MODEL_MLP2:
         ctx->launches += mlp_launch_gradients(ctx->mlp, P, &P.sc->theta_sq, ctx->st);
@@ -411,11 +422,19 @@ laq_status laq_step(laq_ctx* ctx, int32_t n_iters, const laq_trace* trace) {
       cudaEventRecord(ev[1], ctx->st);
       ctx->stage_launches[0] += ctx->launches - l0;
     }
-    ctx->launches += launch_radius(P, ctx->ls, ctx->st);
-    if (ev) cudaEventRecord(ev[2], ctx->st);
-    ctx->launches += launch_quantize_trigger(P, ctx->ls, ctx->st);
-    if (ev) cudaEventRecord(ev[3], ctx->st);
-    ctx->launches += launch_aggregate(P, ctx->ls, ctx->st);
+    if (small) {
+      if (ev) {
+        cudaEventRecord(ev[2], ctx->st);
+        cudaEventRecord(ev[3], ctx->st);
+      }
+      ctx->launches += launch_small_iteration(P, fuse_finalize ? ctx->gbpw : 0, ctx->st);
+    } else {
+      ctx->launches += launch_radius(P, ctx->ls, ctx->st);
+      if (ev) cudaEventRecord(ev[2], ctx->st);
+      ctx->launches += launch_quantize_trigger(P, ctx->ls, ctx->st);
+      if (ev) cudaEventRecord(ev[3], ctx->st);
+      ctx->launches += launch_aggregate(P, ctx->ls, ctx->st);
+    }
     if (ev) {
       cudaEventRecord(ev[4], ctx->st);
       for (int s = 1; s < 4; ++s) ctx->stage_launches[s] += 1;

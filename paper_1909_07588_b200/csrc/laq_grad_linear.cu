@@ -392,6 +392,9 @@ __global__ void __launch_bounds__(256) grad_finalize_kernel(const Params P, int 
 
 bool softmax_classes_supported(int C) { return C >= 2 && C <= 16; }
 
+// Row tiles of the largest shard: more gradient blocks per worker than this would only write zeros.
+int grad_tiles_per_worker(int model, int F, long long n_max);
+
 // rows per tile: a multiple of 4 (so every tile starts 16-byte aligned), at most 160 KB of samples
 static int logreg_rows(int F) {
   int r = (40960 / F) & ~3;
@@ -401,6 +404,12 @@ static size_t logreg_smem(int F) {
   return sizeof(float) * ((size_t)logreg_rows(F) * F + ((F + 3) & ~3) + kLrMaxRows + kLrThreads);
 }
 static size_t softmax_smem(int F, int C) { return sizeof(float) * ((size_t)kSmRows * F + (size_t)kSmRows * C); }
+
+int grad_tiles_per_worker(int model, int F, long long n_max) {
+  const long long rows = (model == LAQ_MODEL_LOGREG_BIN) ? logreg_rows(F) : 16;
+  const long long t = (n_max + rows - 1) / rows;
+  return (int)(t > 1024 ? 1024 : (t < 1 ? 1 : t));
+}
 
 int launch_grad_logreg(const Params& P, const LaunchShape&, int gbpw, cudaStream_t st) {
   const size_t sm = logreg_smem(P.F);

@@ -88,12 +88,15 @@ struct LaunchShape {
 
 // kernels' host-side launchers (each returns the number of kernels it launched)
 int launch_radius(const Params& P, const LaunchShape& ls, cudaStream_t st);
+bool small_iteration_applies(const Params& P);
+int launch_small_iteration(const Params& P, int gbpw_finalize, cudaStream_t st);
 int launch_quantize_trigger(const Params& P, const LaunchShape& ls, cudaStream_t st);
 int launch_aggregate(const Params& P, const LaunchShape& ls, cudaStream_t st);
 int launch_grad_logreg(const Params& P, const LaunchShape& ls, int gbpw, cudaStream_t st);
 int launch_grad_softmax(const Params& P, const LaunchShape& ls, int gbpw, cudaStream_t st);
 int launch_grad_finalize(const Params& P, int gbpw, const double* theta_sq, cudaStream_t st);
 bool softmax_classes_supported(int C);
+int grad_tiles_per_worker(int model, int F, long long n_max);
 
 // one-hidden-layer ReLU network (laq_grad_mlp.cu)
 struct MlpPlan {

@@ -562,6 +562,242 @@ __global__ void __launch_bounds__(512) aggregate_kernel(const Params P) {
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Small problems (M p up to 8192 padded coordinates): steps 2-5 of one iteration in ONE block, so that the
+// iteration is not a chain of launches and cross-block hand-overs.  A warp owns a worker in the radius and
+// quantize phases; the arithmetic and its order are those of the three sweep kernels.  With gbpw > 0 the block
+// first combines the gbpw block partials of the linear-model gradient kernels (what grad_finalize_kernel does).
+// ------------------------------------------------------------------------------------------------
+constexpr int kSmallThreads = 1024;
+
+template <int B>
+__global__ void __launch_bounds__(kSmallThreads) small_iteration_kernel(const Params P, int gbpw) {
+  __shared__ uint32_t s_Rb[kMaxWorkers];
+  __shared__ double s_ndq[kMaxWorkers], s_neps[kMaxWorkers];
+  __shared__ int s_m[kMaxWorkers];
+  __shared__ float s_R[kMaxWorkers], s_s[kMaxWorkers];
+  __shared__ uint8_t s_skip[kMaxWorkers];
+  __shared__ double sh[32];
+  __shared__ int s_nup, s_bad;
+  DevScalars* sc = P.sc;
+  if (*(volatile uint32_t*)&sc->err) return;
+  const int t = threadIdx.x, lane = t & 31, w = t >> 5, nw = kSmallThreads / 32, M = P.M;
+  const long long p = P.p;
+  const uint32_t nv = (uint32_t)P.nv;
+  const unsigned long long k = sc->k;
+  const int par = (int)(k & 1ull);
+  if (t == 0) s_bad = 0;
+  // ---- step 1 (tail): block partials of the gradient kernels -> g_m, loss_m
+  if (gbpw > 0) {
+    const double inv_N = 1.0 / (double)P.Ntot;
+    for (long long idx = t; idx < (long long)M * p; idx += kSmallThreads) {
+      const int m = (int)(idx / p);
+      const long long i = idx - (long long)m * p;
+      const float* gp = P.gpart + (long long)m * gbpw * P.ps + i;
+      double s = 0.0;
+      for (int blk = 0; blk < gbpw; ++blk) s += (double)gp[(long long)blk * P.ps];
+      const double share = (double)P.N[m] / (double)P.Ntot;
+      P.g[(long long)m * P.ps + i] = (float)(s * inv_N + share * (double)P.lambda * (double)P.theta[i]);
+    }
+    for (int m = t; m < M; m += kSmallThreads) {
+      double l = 0.0;
+      for (int blk = 0; blk < gbpw; ++blk) l += P.lpart[(long long)m * gbpw + blk];
+      const double share = (double)P.N[m] / (double)P.Ntot;
+      P.loss_m[m] = l * inv_N + share * 0.5 * (double)P.lambda * sc->theta_sq;
+    }
+  }
+  __syncthreads();
+  // ---- radius: a warp per worker
+  for (int m = w; m < M; m += nw) {
+    const float4* q4 = reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps);
+    const float4* g4 = reinterpret_cast<const float4*>(P.g + (long long)m * P.ps);
+    uint32_t mx = 0;
+    for (uint32_t v = lane; v < nv; v += 32) {   // padding of Q_prev and g is zero
+      const float4 q = q4[v], g = g4[v];
+      mx = max(mx, abs_bits(__fsub_rn(g.x, q.x)));
+      mx = max(mx, abs_bits(__fsub_rn(g.y, q.y)));
+      mx = max(mx, abs_bits(__fsub_rn(g.z, q.z)));
+      mx = max(mx, abs_bits(__fsub_rn(g.w, q.w)));
+    }
+    mx = __reduce_max_sync(0xffffffffu, mx);
+    if (lane == 0) {
+      s_Rb[m] = mx;
+      if (mx >= 0x7f800000u) s_bad = 1;
+    }
+  }
+  __syncthreads();
+  if (s_bad) {  // freeze: nothing of this iteration is applied
+    if (t == 0) {
+      sc->n_up = 0;
+      atomicOr(&sc->err, 1u);
+    }
+    return;
+  }
+  // ---- codes and the two norms: a warp per worker
+  for (int m = w; m < M; m += nw) {
+    const float R = __uint_as_float(s_Rb[m]);
+    const float levels = (float)((1u << B) - 1u);
+    const float s = __fmul_rn(__fmul_rn(2.0f, __fdiv_rn(1.0f, levels)), R);
+    const bool fast = s >= 0x1p-60f && s <= 0x1p60f;
+    const float y = __fdiv_rn(1.0f, s);
+    const float4* q4 = reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps);
+    const float4* g4 = reinterpret_cast<const float4*>(P.g + (long long)m * P.ps);
+    uint32_t* row = P.codes + (long long)m * P.cw;
+    double sdq = 0.0, seps = 0.0;
+    if (R > 0.f) {
+      for (uint32_t v0 = 0; v0 < nv; v0 += 32) {   // all lanes make the same number of trips
+        const uint32_t v = v0 + lane;
+        const bool ok = v < nv;
+        uint32_t yy[4] = {0x4b000000u, 0x4b000000u, 0x4b000000u, 0x4b000000u};
+        if (ok) {
+          const float4 q = q4[v], g = g4[v];
+          const float gg[4] = {g.x, g.y, g.z, g.w}, qq[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            if (4ll * v + e < p)
+              yy[e] = fast ? quantize_one<true>(gg[e], qq[e], R, s, y, sdq, seps)
+                           : quantize_one<false>(gg[e], qq[e], R, s, y, sdq, seps);
+        }
+        store_codes<B>(row, v, yy[0], yy[1], yy[2], yy[3], ok);
+      }
+    } else {
+      for (long long wd = lane; wd < P.cw; wd += 32) row[wd] = 0u;
+    }
+    sdq = warp_sum(sdq);
+    seps = warp_sum(seps);
+    if (lane == 0) {
+      s_ndq[m] = sdq;
+      s_neps[m] = seps;
+    }
+  }
+  __syncthreads();
+  // ---- skip rule (7a) + clock (7b)
+  const bool tracing = P.trace_cap > 0 && sc->trace_pos < (uint32_t)P.trace_cap;
+  const long long trow = (long long)sc->trace_pos * M;
+  for (int m = t; m < M; m += kSmallThreads) {
+    const double n_dq = s_ndq[m], n_eps = s_neps[m];
+    double acc = 0.0;
+    for (int d = 0; d < P.D; ++d) {
+      const double term = (double)P.xi[d] * P.ring[(sc->ring_head + d) % P.D];
+      acc = acc + term;
+    }
+    const double rhs = acc / P.trig_c + 3.0 * (n_eps + P.n_epshat[m]);
+    const int clk = P.clock[m];
+    const bool crit_a = n_dq <= rhs;
+    const bool crit_b = (P.clock_mode == 0) ? (clk <= P.tbar) : (clk + 2 <= P.tbar);
+    const bool skip = crit_a && crit_b && !(P.flags & LAQ_FLAG_TRIGGER_OFF);
+    if (skip) {
+      P.clock[m] = clk + 1;
+    } else {
+      P.clock[m] = 0;
+      P.n_epshat[m] = n_eps;
+    }
+    s_skip[m] = skip ? 1 : 0;
+    P.skip[m] = skip ? 1 : 0;
+    P.norms[3 * m + 0] = n_dq;
+    P.norms[3 * m + 1] = n_eps;
+    P.norms[3 * m + 2] = rhs;
+    P.Rbits[par * M + m] = s_Rb[m];
+    P.Rbits[(par ^ 1) * M + m] = 0u;
+    if (tracing) {
+      P.t_skip[trow + m] = skip ? 1 : 0;
+      P.t_R[trow + m] = __uint_as_float(s_Rb[m]);
+      P.t_ndq[trow + m] = n_dq;
+      P.t_neps[trow + m] = n_eps;
+      P.t_rhs[trow + m] = rhs;
+    }
+  }
+  __syncthreads();
+  if (t == 0) {
+    const float levels = (float)((1u << B) - 1u);
+    const float two_tau = __fmul_rn(2.0f, __fdiv_rn(1.0f, levels));
+    int n = 0;
+    for (int m = 0; m < M; ++m) {
+      if (!s_skip[m]) {
+        const float R = __uint_as_float(s_Rb[m]);
+        s_m[n] = m;
+        s_R[n] = R;
+        s_s[n] = __fmul_rn(two_tau, R);
+        ++n;
+      }
+    }
+    s_nup = n;
+    sc->n_up = n;
+    sc->uploads += (unsigned long long)n;
+    sc->bits += (unsigned long long)n * (32ull + (unsigned long long)B * (unsigned long long)p);
+    if (tracing) P.t_up[sc->trace_pos] = n;
+  }
+  __syncthreads();
+  // ---- lazy aggregate + theta step
+  const int n_up = s_nup;
+  float4* agg4 = reinterpret_cast<float4*>(P.agg);
+  float4* th4 = reinterpret_cast<float4*>(P.theta);
+  const float alpha = P.alpha;
+  double dsum = 0.0, tsum = 0.0;
+  for (uint32_t v = t; v < nv; v += kSmallThreads) {
+    float4 a = agg4[v];
+    const long long i = 4ll * v;
+    for (int u = 0; u < n_up; ++u) {
+      const int m = s_m[u];
+      const float R = s_R[u], s = s_s[u];
+      float4* qrow = reinterpret_cast<float4*>(P.qp + (long long)m * P.ps) + v;
+      float4 q = *qrow;
+      uint32_t c[4];
+      load_codes<B>(P.codes + (long long)m * P.cw, v, c);
+      float d0 = __fsub_rn(__fmul_rn(s, code_to_float(c[0])), R);
+      float d1 = __fsub_rn(__fmul_rn(s, code_to_float(c[1])), R);
+      float d2 = __fsub_rn(__fmul_rn(s, code_to_float(c[2])), R);
+      float d3 = __fsub_rn(__fmul_rn(s, code_to_float(c[3])), R);
+      if (i >= p) d0 = 0.f;        // padding coordinates carry no innovation
+      if (i + 1 >= p) d1 = 0.f;
+      if (i + 2 >= p) d2 = 0.f;
+      if (i + 3 >= p) d3 = 0.f;
+      q.x = __fadd_rn(q.x, d0);
+      q.y = __fadd_rn(q.y, d1);
+      q.z = __fadd_rn(q.z, d2);
+      q.w = __fadd_rn(q.w, d3);
+      *qrow = q;
+      a.x = __fadd_rn(a.x, d0);
+      a.y = __fadd_rn(a.y, d1);
+      a.z = __fadd_rn(a.z, d2);
+      a.w = __fadd_rn(a.w, d3);
+    }
+    agg4[v] = a;
+    float4 th = th4[v];
+    const float u0 = __fmul_rn(alpha, a.x), u1 = __fmul_rn(alpha, a.y), u2 = __fmul_rn(alpha, a.z),
+                u3 = __fmul_rn(alpha, a.w);
+    th.x = __fsub_rn(th.x, u0);
+    th.y = __fsub_rn(th.y, u1);
+    th.z = __fsub_rn(th.z, u2);
+    th.w = __fsub_rn(th.w, u3);
+    th4[v] = th;
+    dsum = fma((double)u0, (double)u0, dsum);
+    dsum = fma((double)u1, (double)u1, dsum);
+    dsum = fma((double)u2, (double)u2, dsum);
+    dsum = fma((double)u3, (double)u3, dsum);
+    tsum = fma((double)th.x, (double)th.x, tsum);
+    tsum = fma((double)th.y, (double)th.y, tsum);
+    tsum = fma((double)th.z, (double)th.z, tsum);
+    tsum = fma((double)th.w, (double)th.w, tsum);
+  }
+  const double d2 = block_sum(dsum, sh);
+  const double th2 = block_sum(tsum, sh);
+  if (t == 0) {
+    sc->theta_sq = th2;
+    const uint32_t head = (sc->ring_head + (uint32_t)P.D - 1u) % (uint32_t)P.D;
+    P.ring[head] = d2;
+    sc->ring_head = head;
+    if (tracing) {
+      P.t_d2[sc->trace_pos] = d2;
+      double loss = 0.0;
+      for (int m = 0; m < M; ++m) loss += P.loss_m[m];
+      P.t_loss[sc->trace_pos] = loss;
+      sc->trace_pos += 1;
+    }
+    sc->k += 1ull;
+  }
+}
+
 template <bool SYNTH>
 void launch_quant_b(const Params& P, dim3 grid, int threads, cudaStream_t st) {
   switch (P.b) {
@@ -591,6 +827,21 @@ int aggregate_blocks(const Params& P, const LaunchShape& ls) {
   long long need = (P.nv + ls.agg_threads - 1) / ls.agg_threads;
   long long nb = want < need ? want : need;
   return (int)(nb < 1 ? 1 : nb);
+}
+
+bool small_iteration_applies(const Params& P) {
+  return P.model != LAQ_MODEL_SYNTH && (long long)P.M * P.ps <= 8192;
+}
+
+int launch_small_iteration(const Params& P, int gbpw_finalize, cudaStream_t st) {
+  switch (P.b) {
+    case 1: small_iteration_kernel<1><<<1, kSmallThreads, 0, st>>>(P, gbpw_finalize); break;
+    case 2: small_iteration_kernel<2><<<1, kSmallThreads, 0, st>>>(P, gbpw_finalize); break;
+    case 4: small_iteration_kernel<4><<<1, kSmallThreads, 0, st>>>(P, gbpw_finalize); break;
+    case 8: small_iteration_kernel<8><<<1, kSmallThreads, 0, st>>>(P, gbpw_finalize); break;
+    default: small_iteration_kernel<16><<<1, kSmallThreads, 0, st>>>(P, gbpw_finalize); break;
+  }
+  return 1;
 }
 
 int launch_radius(const Params& P, const LaunchShape& ls, cudaStream_t st) {
