@@ -105,8 +105,8 @@ struct Plan {
 };
 
 int default_gbpw(const laq_config& c) {
-  // resident blocks per SM: two for the softmax tiles, four for the narrow logistic tiles; one wave
-  int g = ((c.model == LAQ_MODEL_LOGREG_BIN ? 4 : 2) * kNumSMs) / c.M;
+  // one wave of resident blocks (shared memory decides how many fit on an SM)
+  int g = (grad_blocks_per_sm(c.model, c.n_features) * kNumSMs) / c.M;
   if (g > kGradBlocksCap) g = kGradBlocksCap;
   return g < 1 ? 1 : g;
 }

@@ -24,6 +24,16 @@ __device__ __forceinline__ float warp_sum_f(float v) {
   return v;
 }
 
+// Packed fp32 pairs: sm_100 executes two fused multiply-adds per lane in one instruction.
+__device__ __forceinline__ unsigned long long ffma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+
 // Copy `count` consecutive floats global -> shared; where alignment allows as asynchronous 16-byte copies, so
 // that every thread has all of its copies in flight at once.  Ends with the copies complete for this thread;
 // the caller's __syncthreads() makes them visible to the block.
@@ -211,95 +221,105 @@ __global__ void __launch_bounds__(kSmThreads) grad_softmax_kernel(const Params P
 
 // ------------------------------------------------------------------------------------------------
 // C-class softmax regression, fast path: F a multiple of 4, F <= 896, C <= 12.
-// 224 threads (7 warps), tiles of 16 rows staged in shared memory with a row stride of an odd number of
-// 16-byte units (conflict-free 16-byte reads down a column of rows); theta sits in shared memory too.
-//   phase 1  lane = (row, parity of the 16-byte feature group), warp = slice of the feature axis: scores from
-//            16-byte reads of x and broadcast 16-byte reads of theta; the 14 partials per (row, class) are
-//            summed through shared memory, one thread per row then does softmax, residual and loss;
+// 224 threads (7 warps), tiles of 8 rows in a two-deep ring of shared-memory buffers filled by asynchronous
+// 16-byte copies (the next tile arrives while the current one is worked on); rows are padded to an odd number of
+// 16-byte units so that 16-byte reads down a column of rows are conflict free; theta sits in shared memory too.
+//   phase 1  lane = (row, feature group mod 4), warp = slice of the feature axis: scores from 16-byte reads of x
+//            and broadcast 16-byte reads of theta; the 28 partials per (row, class) are summed through shared
+//            memory, one thread per row then does softmax, residual and loss;
 //   phase 2  thread = four consecutive features: acc[4][C] += residual[r][c] * x[r][f] over the tile's rows,
 //            one 16-byte read of x and the broadcast residuals per row.
-// Two blocks fit on an SM, so one block's loads overlap the other's arithmetic.
+// Two blocks fit on an SM.
 // ------------------------------------------------------------------------------------------------
 constexpr int kS2Threads = 224;
 constexpr int kS2Warps = 7;
-constexpr int kS2Rows = 16;
-constexpr int kS2Parts = 2 * kS2Warps;   // partial scores per (row, class)
+constexpr int kS2Rows = 8;
+constexpr int kS2Parts = 4 * kS2Warps;   // partial scores per (row, class)
 
 template <int C>
 __global__ void __launch_bounds__(kS2Threads, 2) grad_softmax_tile_kernel(const Params P, int gbpw) {
   extern __shared__ __align__(16) float smem[];
   const int F = P.F, F4 = F >> 2, FP4 = F4 | 1, FP = FP4 << 2;      // padded row stride (floats)
   const int m = blockIdx.y, t = threadIdx.x, lane = t & 31, w = t >> 5;
-  float* xs = smem;                                  // [16][FP]
-  float* ths = xs + kS2Rows * FP;                    // [C][F]      theta
-  float* plog = ths + C * F;                         // [14][16][C] partial scores
-  float* res = plog + kS2Parts * kS2Rows * C;        // [16][12]    residuals, padded to 16-byte rows
+  float* xs0 = smem;                                 // [2][8][FP]
+  float* ths = xs0 + 2 * kS2Rows * FP;               // [C][F]      theta
+  float* plog = ths + C * F;                         // [28][8][C]  partial scores
+  float* res = plog + kS2Parts * kS2Rows * C;        // [8][12][2]  residuals, each stored twice (packed pairs)
   __shared__ double shd[8];
-  __shared__ float zs[kS2Rows * 12];                 // [16][C]     scores
+  __shared__ float zs[kS2Rows * 12];                 // [8][C]      scores
   static_assert(kS2Rows * C <= kS2Threads, "one thread per (row, class)");
   const float* __restrict__ X = P.X[m];
   const int32_t* __restrict__ y = P.y[m];
   const long long n = P.N[m];
   for (int i = t; i < C * F4; i += kS2Threads)
     reinterpret_cast<float4*>(ths)[i] = __ldg(reinterpret_cast<const float4*>(P.theta) + i);
-  const float4* th4 = reinterpret_cast<const float4*>(ths);
   const int kw = (F4 + kS2Warps - 1) / kS2Warps;     // 16-byte groups of features per warp in phase 1
-  const int row1 = lane & 15, par = lane >> 4;
+  const int row1 = lane & 7, par = lane >> 3;
   const int k_lo = w * kw + par, k_hi = min(F4, w * kw + kw);
   const bool owner = t < F4;                         // phase 2: thread t owns features 4t .. 4t+3
-  float acc[4][C];
+  unsigned long long acc01[C], acc23[C];            // packed pairs (features 4t, 4t+1) and (4t+2, 4t+3)
 #pragma unroll
-  for (int e = 0; e < 4; ++e)
-#pragma unroll
-    for (int c = 0; c < C; ++c) acc[e][c] = 0.f;
+  for (int c = 0; c < C; ++c) acc01[c] = acc23[c] = 0ull;
   double loss = 0.0;
   const long long ntiles = (n + kS2Rows - 1) / kS2Rows;
-  for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+
+  // asynchronous staging of one tile: contiguous rows in global memory -> padded rows in shared memory
+  auto stage = [&](long long tile, float* xs) {
     const long long r0 = tile * kS2Rows;
     const int nr = (int)((n - r0 < kS2Rows) ? (n - r0) : kS2Rows);
-    __syncthreads();
-    {  // stage: contiguous rows in global memory -> padded rows in shared memory, as asynchronous 16-byte
-       // copies so that a thread has all of its copies in flight at once
-      const float4* src = reinterpret_cast<const float4*>(X + r0 * F);
-      const int cnt = nr * F4;
-      int r = t / F4, k = t - r * F4;
-      for (int i = t; i < kS2Rows * F4; i += kS2Threads) {
-        float* dst = xs + r * FP + 4 * k;
-        if (i < cnt)
-          __pipeline_memcpy_async(dst, src + i, 16);
-        else
-          *reinterpret_cast<float4*>(dst) = make_float4(0.f, 0.f, 0.f, 0.f);
-        k += kS2Threads;
-        while (k >= F4) {
-          k -= F4;
-          ++r;
-        }
+    const float4* src = reinterpret_cast<const float4*>(X + r0 * F);
+    const int cnt = nr * F4;
+    int r = t / F4, k = t - r * F4;
+    for (int i = t; i < kS2Rows * F4; i += kS2Threads) {
+      float* dst = xs + r * FP + 4 * k;
+      if (i < cnt)
+        __pipeline_memcpy_async(dst, src + i, 16);
+      else
+        *reinterpret_cast<float4*>(dst) = make_float4(0.f, 0.f, 0.f, 0.f);
+      k += kS2Threads;
+      while (k >= F4) {
+        k -= F4;
+        ++r;
       }
-      __pipeline_commit();
-      __pipeline_wait_prior(0);
     }
+  };
+
+  int buf = 0;
+  if ((long long)blockIdx.x < ntiles) stage(blockIdx.x, xs0);
+  __pipeline_commit();
+  for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x, buf ^= 1) {
+    const long long r0 = tile * kS2Rows;
+    const int nr = (int)((n - r0 < kS2Rows) ? (n - r0) : kS2Rows);
+    float* xs = xs0 + buf * kS2Rows * FP;
+    __syncthreads();                                  // everybody is done with the buffer refilled below
+    if (tile + gridDim.x < ntiles) stage(tile + gridDim.x, xs0 + (buf ^ 1) * kS2Rows * FP);
+    __pipeline_commit();
+    __pipeline_wait_prior(1);                         // this tile's copies (the older group) have landed
     __syncthreads();
-    {  // phase 1
-      float z[C];
+    {  // phase 1 (packed pairs: the two halves of a score are added at the end)
+      unsigned long long z2[C];
 #pragma unroll
-      for (int c = 0; c < C; ++c) z[c] = 0.f;
-      const float4* xr = reinterpret_cast<const float4*>(xs + row1 * FP);
-      for (int k = k_lo; k < k_hi; k += 2) {
-        const float4 x = xr[k];
+      for (int c = 0; c < C; ++c) z2[c] = 0ull;
+      const ulonglong2* xr = reinterpret_cast<const ulonglong2*>(xs + row1 * FP);
+      const ulonglong2* th2 = reinterpret_cast<const ulonglong2*>(ths);
+      for (int k = k_lo; k < k_hi; k += 4) {
+        const ulonglong2 x = xr[k];
 #pragma unroll
         for (int c = 0; c < C; ++c) {
-          const float4 th = th4[c * F4 + k];
-          z[c] = fmaf(x.x, th.x, z[c]);
-          z[c] = fmaf(x.y, th.y, z[c]);
-          z[c] = fmaf(x.z, th.z, z[c]);
-          z[c] = fmaf(x.w, th.w, z[c]);
+          const ulonglong2 th = th2[c * F4 + k];
+          z2[c] = ffma2(x.x, th.x, z2[c]);
+          z2[c] = ffma2(x.y, th.y, z2[c]);
         }
       }
 #pragma unroll
-      for (int c = 0; c < C; ++c) plog[((2 * w + par) * kS2Rows + row1) * C + c] = z[c];
+      for (int c = 0; c < C; ++c) {
+        float lo, hi;
+        unpack2(z2[c], lo, hi);
+        plog[((4 * w + par) * kS2Rows + row1) * C + c] = lo + hi;
+      }
     }
     __syncthreads();
-    if (t < kS2Rows * C) {  // one thread per (row, class): sum the 14 partial scores in a fixed order
+    if (t < kS2Rows * C) {  // one thread per (row, class): sum the 28 partial scores in a fixed order
       float s = 0.f;
 #pragma unroll
       for (int ww = 0; ww < kS2Parts; ++ww) s += plog[ww * kS2Rows * C + t];
@@ -326,34 +346,42 @@ __global__ void __launch_bounds__(kS2Threads, 2) grad_softmax_tile_kernel(const 
 #pragma unroll
       for (int c = 0; c < C; ++c) {
         if (c == yv) zy = z[c];
-        res[t * 12 + c] = live ? (e[c] * inv - (c == yv ? 1.f : 0.f)) : 0.f;
+        const float rv = live ? (e[c] * inv - (c == yv ? 1.f : 0.f)) : 0.f;
+        res[(t * 12 + c) * 2] = rv;
+        res[(t * 12 + c) * 2 + 1] = rv;
       }
       if (live) loss += (double)((zmax + logf(sum)) - zy);
     }
     __syncthreads();
     if (owner) {  // phase 2
       const float* xc = xs + 4 * t;
-      for (int r = 0; r < nr; ++r) {
-        const float4 x = *reinterpret_cast<const float4*>(xc + r * FP);
-        float rr[12];
-        *reinterpret_cast<float4*>(rr) = *reinterpret_cast<const float4*>(res + r * 12);
-        *reinterpret_cast<float4*>(rr + 4) = *reinterpret_cast<const float4*>(res + r * 12 + 4);
-        *reinterpret_cast<float4*>(rr + 8) = *reinterpret_cast<const float4*>(res + r * 12 + 8);
+#pragma unroll 2
+      for (int r = 0; r < kS2Rows; ++r) {             // rows beyond the shard hold zero residuals
+        const ulonglong2 x = *reinterpret_cast<const ulonglong2*>(xc + r * FP);
+        const ulonglong2* rp = reinterpret_cast<const ulonglong2*>(res + r * 24);
 #pragma unroll
-        for (int c = 0; c < C; ++c) {
-          acc[0][c] = fmaf(rr[c], x.x, acc[0][c]);
-          acc[1][c] = fmaf(rr[c], x.y, acc[1][c]);
-          acc[2][c] = fmaf(rr[c], x.z, acc[2][c]);
-          acc[3][c] = fmaf(rr[c], x.w, acc[3][c]);
+        for (int c = 0; c < C; c += 2) {
+          const ulonglong2 rr = rp[c >> 1];           // (r_c, r_c), (r_c+1, r_c+1)
+          acc01[c] = ffma2(rr.x, x.x, acc01[c]);
+          acc23[c] = ffma2(rr.x, x.y, acc23[c]);
+          if (c + 1 < C) {
+            acc01[c + 1] = ffma2(rr.y, x.x, acc01[c + 1]);
+            acc23[c + 1] = ffma2(rr.y, x.y, acc23[c + 1]);
+          }
         }
       }
     }
   }
+  __pipeline_wait_prior(0);
   float* gp = P.gpart + ((long long)m * gbpw + blockIdx.x) * P.ps;
   if (owner) {
 #pragma unroll
-    for (int c = 0; c < C; ++c)
-      *reinterpret_cast<float4*>(gp + c * F + 4 * t) = make_float4(acc[0][c], acc[1][c], acc[2][c], acc[3][c]);
+    for (int c = 0; c < C; ++c) {
+      float4 v;
+      unpack2(acc01[c], v.x, v.y);
+      unpack2(acc23[c], v.z, v.w);
+      *reinterpret_cast<float4*>(gp + c * F + 4 * t) = v;
+    }
   }
   loss = warp_sum_d(loss);
   __syncthreads();
@@ -406,9 +434,16 @@ static size_t logreg_smem(int F) {
 static size_t softmax_smem(int F, int C) { return sizeof(float) * ((size_t)kSmRows * F + (size_t)kSmRows * C); }
 
 int grad_tiles_per_worker(int model, int F, long long n_max) {
-  const long long rows = (model == LAQ_MODEL_LOGREG_BIN) ? logreg_rows(F) : 16;
+  const long long rows = (model == LAQ_MODEL_LOGREG_BIN) ? logreg_rows(F) : 8;
   const long long t = (n_max + rows - 1) / rows;
   return (int)(t > 1024 ? 1024 : (t < 1 ? 1 : t));
+}
+
+// Blocks of the gradient kernel that fit on one SM (shared memory bound): the grid is sized to one such wave.
+int grad_blocks_per_sm(int model, int F) {
+  if (model != LAQ_MODEL_LOGREG_BIN) return 2;
+  const int fit = (int)((227 * 1024) / (logreg_smem(F) + 1024));
+  return fit < 1 ? 1 : (fit > 8 ? 8 : fit);
 }
 
 int launch_grad_logreg(const Params& P, const LaunchShape&, int gbpw, cudaStream_t st) {
@@ -425,7 +460,7 @@ int launch_grad_logreg(const Params& P, const LaunchShape&, int gbpw, cudaStream
 static bool softmax_tile_path(int F, int C) { return (F % 4) == 0 && F / 4 <= kS2Threads && C <= 12; }
 static size_t softmax_tile_smem(int F, int C) {
   const int FP = ((F >> 2) | 1) << 2;
-  return sizeof(float) * ((size_t)kS2Rows * FP + (size_t)C * F + (size_t)kS2Parts * kS2Rows * C + (size_t)kS2Rows * 12);
+  return sizeof(float) * (2 * (size_t)kS2Rows * FP + (size_t)C * F + (size_t)kS2Parts * kS2Rows * C + (size_t)kS2Rows * 24);
 }
 
 template <int C>

@@ -97,6 +97,7 @@ int launch_grad_softmax(const Params& P, const LaunchShape& ls, int gbpw, cudaSt
 int launch_grad_finalize(const Params& P, int gbpw, const double* theta_sq, cudaStream_t st);
 bool softmax_classes_supported(int C);
 int grad_tiles_per_worker(int model, int F, long long n_max);
+int grad_blocks_per_sm(int model, int F);
 
 // one-hidden-layer ReLU network (laq_grad_mlp.cu)
 struct MlpPlan {
