@@ -59,6 +59,15 @@ def hbm_peak():
         return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
 
 
+def tensor_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops_sustained"]), "measured (MEASURED_PEAKS.json bf16_tflops_sustained)"
+    except Exception:
+        return 1400.0, "fallback (earlier measurement on this pool, sustained)"
+
+
 def algorithmic_bytes(w, u):
     """Bytes the method must move per iteration, per stage ("Algorithmic bytes").
     u = uploading fraction |M^k| / M averaged over the timed iterations."""
@@ -317,6 +326,21 @@ def main():
                 "whole_path": {"bytes_per_iter": path_bytes, "GB/s": path_bytes / (path_ms * 1e-3) / 1e9,
                                "frac": path_bytes / (path_ms * 1e-3) / 1e9 / peak}}
 
+    if w.model == 2:
+        # the network's gradient stage is two dense bf16 products (X W1^T and dH^T X): a tensor-core roofline
+        g_stage = [st for st in stages if st["stage"] == "local_gradient"][0]
+        flops = 4.0 * sum(w.N) * w.n_features * w.n_hidden
+        tpeak, tsrc = tensor_peak()
+        tf = flops / (g_stage["ms"] * 1e-3) / 1e12
+        roofline.update({"bound": "tensor", "kernel": "umma_hidden_fused_kernel + umma_dw1_kernel (whole gradient stage)",
+                         "achieved": tf, "peak": tpeak, "unit": "TFLOP/s", "frac": tf / tpeak, "traffic": None,
+                         "peak_source": tsrc, "flops_per_launch": flops, "ms_per_launch": g_stage["ms"]})
+    if w.model != 3 and w.M * ((w.p + 15) // 16 * 16) <= 8192:
+        # small problems run steps 2-5 in one single-block kernel: the radius and quantize slots are empty
+        stages = [st for st in stages if st["stage"] not in ("radius", "quantize_norms_trigger")]
+        stages[-1]["stage"] = "steps_2_to_5_single_block"
+        stages[-1]["kernel"] = "small_iteration_kernel"
+        roofline["stages"] = stages
     line = {"metric": METRIC, "value": world * K / (ms * 1e-3), "unit": "iters/s", "n_gpus": world, "steps": K,
             "warmup": Wm, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
