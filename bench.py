@@ -82,6 +82,22 @@ def algorithmic_bytes(w, u):
     }
 
 
+def max_over_ranks(x, world, device="cuda"):
+    """The slowest rank's time decides: maximum of a per-rank scalar over all ranks (identity for one rank)."""
+    if world <= 1:
+        return float(x)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(x)], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replicas_throughput(world, steps, ms):
+    """Whole-job iterations/s of `world` independent replicas that each ran `steps` iterations in `ms` (max over ranks)."""
+    return world * steps / (ms * 1e-3)
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -272,10 +288,7 @@ def main():
     clocks = sampler.stop()
     if not inline_events:
         s2 = ctx.get_state(big=False)
-    if world > 1:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, world)
     u = (s2["uploads"] - s1["uploads"]) / float(K * w.M)       # of the iterations whose stages were timed
 
     # ---- end to end through the C ABI with host buffers ---------------------------------------------------
@@ -291,10 +304,7 @@ def main():
     theta_out = ctx2.get_state(big=False)["theta"]
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = max_over_ranks(e2e_s, world)
     ctx2.close()
     shard_bytes = sum(x.nbytes + y.nbytes for x, y in zip(w.X, w.y))
     e2e = {"value": world * Ke / e2e_s, "unit": "iters/s", "steps": Ke,
@@ -341,7 +351,7 @@ def main():
         stages[-1]["stage"] = "steps_2_to_5_single_block"
         stages[-1]["kernel"] = "small_iteration_kernel"
         roofline["stages"] = stages
-    line = {"metric": METRIC, "value": world * K / (ms * 1e-3), "unit": "iters/s", "n_gpus": world, "steps": K,
+    line = {"metric": METRIC, "value": replicas_throughput(world, K, ms), "unit": "iters/s", "n_gpus": world, "steps": K,
             "warmup": Wm, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "name": w.name, "M": w.M, "p": w.p, "b": w.b, "D": w.D,
