@@ -161,40 +161,40 @@ def traffic_for(stage, w):
         return None
 
 
-def cpu_baseline(w, name):
-    """The oracle as it stands, one thread, on a bounded sample of the workload."""
+def cpu_baseline(w, name, steps=None, warmup=1, budget_s=12.0):
+    """The oracle as it stands, one thread, on a bounded sample of the workload.  With `steps` given (the
+    reference arm) it runs that many sample iterations after `warmup`, but stops when `budget_s` is used up."""
     import oracle
-    t_build = time.time()
     oracle.build()
     if w.model == 3:
-        p_s = 1_600_000
+        p_s = min(w.p, 1_600_000)
         o = oracle.OracleLaq(32, oracle.MODEL_SYNTH, w.M, p_s, alpha=w.alpha, b=w.b, D=w.D, xi=w.xi, tbar=w.tbar,
                              seed=w.seed, synth_sigma=w.synth_sigma, synth_eta0=w.synth_eta0)
-        o.step()
-        t0 = time.time()
-        n = 0
-        while n < 2 or (time.time() - t0 < 10.0 and n < 50):
-            o.step()
-            n += 1
-        dt = time.time() - t0
         scale = p_s / float(w.p)
-        return {"value": n / dt * scale, "unit": "iters/s", "cores": 1, "kind": "oracle",
-                "sample": "fp32 mirror, M=%d workers, first %d of %d coordinates, %d iterations after 1 warm-up; "
-                          "iterations/s scaled by %g (cost is linear in p)" % (w.M, p_s, w.p, n, scale)}
-    o = oracle.OracleLaq(64, w.model, w.M, w.p, N=w.N, n_features=w.n_features, n_classes=w.n_classes,
-                         n_hidden=w.n_hidden, alpha=w.alpha, lam=w.lam, b=w.b, D=w.D, xi=w.xi, tbar=w.tbar,
-                         bf16_ops=w.bf16_ops, theta0=w.theta0)
-    for m in range(w.M):
-        o.set_shard(m, w.X[m], w.y[m])
-    o.step()
+        what = "fp32 mirror, M=%d workers, first %d of %d coordinates" % (w.M, p_s, w.p)
+    else:
+        o = oracle.OracleLaq(64, w.model, w.M, w.p, N=w.N, n_features=w.n_features, n_classes=w.n_classes,
+                             n_hidden=w.n_hidden, alpha=w.alpha, lam=w.lam, b=w.b, D=w.D, xi=w.xi, tbar=w.tbar,
+                             bf16_ops=w.bf16_ops, theta0=w.theta0)
+        for m in range(w.M):
+            o.set_shard(m, w.X[m], w.y[m])
+        scale = 1.0
+        what = "fp64 oracle, full workload"
+    t_w = time.time()
+    for _ in range(max(1, warmup)):
+        o.step()
+        if time.time() - t_w > budget_s / 3:
+            break
     t0 = time.time()
     n = 0
-    while n < 2 or (time.time() - t0 < 10.0 and n < w.iters):
+    limit = steps if steps is not None else 10 ** 9
+    while n < limit and (n < 2 or time.time() - t0 < budget_s):
         o.step()
         n += 1
     dt = time.time() - t0
-    return {"value": n / dt, "unit": "iters/s", "cores": 1, "kind": "oracle",
-            "sample": "fp64 oracle, full workload, %d iterations after 1 warm-up" % n}
+    return {"value": n / dt * scale, "unit": "iters/s", "cores": 1, "kind": "oracle",
+            "sample": "%s, %d iterations after warm-up%s" % (
+                what, n, "; iterations/s scaled by %g (cost is linear in p)" % scale if scale != 1.0 else "")}
 
 
 def run_reference(args, w, name, rank):
@@ -202,7 +202,7 @@ def run_reference(args, w, name, rank):
     if rank != 0:
         return
     t0 = time.time()
-    base = cpu_baseline(w, name)
+    base = cpu_baseline(w, name, steps=args.steps, warmup=args.warmup, budget_s=150.0)
     val = base["value"]
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "iters/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1000.0 / val, "higher_is_better": True,
