@@ -74,7 +74,11 @@ typedef enum {
  *   g_m^k[i] = fma(fl(k eta_m), z_{e xor 2}, z_e) * cz,  k = 1, 2, ...   (requires p < 2^32) */
 
 enum {
-  LAQ_FLAG_TRIGGER_OFF = 2u /* every worker uploads every iteration: Algorithm 1 (QGD) */
+  LAQ_FLAG_QUANT_OFF = 1u,  /* no quantizer: an upload carries the innovation g_m - Q_m(theta_hat^{k-1}) itself,
+                               32 bits per coordinate, eps = 0 in (7a): the lazily aggregated gradient baseline
+                               (LAG) of Sec. 4.  R is still reported; no codes are written (they stay zero) */
+  LAQ_FLAG_TRIGGER_OFF = 2u /* every worker uploads every iteration: Algorithm 1 (QGD); with LAQ_FLAG_QUANT_OFF
+                               as well: gradient descent, Eq. (2) */
 };
 
 typedef struct {

@@ -69,7 +69,7 @@ const char* check_config(const laq_config* c) {
   if (!(c->alpha > 0.f) || !std::isfinite(c->alpha)) return "alpha must be positive and finite";
   if (c->clock_mode != 0 && c->clock_mode != 1) return "clock_mode must be 0 or 1";
   if (c->trace_capacity < 0) return "trace_capacity must be >= 0";
-  if (c->flags & ~(uint32_t)LAQ_FLAG_TRIGGER_OFF) return "unknown flag";
+  if (c->flags & ~(uint32_t)(LAQ_FLAG_TRIGGER_OFF | LAQ_FLAG_QUANT_OFF)) return "unknown flag";
   const bool data = c->model == LAQ_MODEL_LOGREG_BIN || c->model == LAQ_MODEL_SOFTMAX || c->model == LAQ_MODEL_MLP2;
   if (data) {
     if (!c->N) return "N is null";
@@ -429,9 +429,15 @@ laq_status laq_step(laq_ctx* ctx, int32_t n_iters, const laq_trace* trace) {
       }
       ctx->launches += launch_small_iteration(P, fuse_finalize ? ctx->gbpw : 0, ctx->st);
     } else {
-      ctx->launches += launch_radius(P, ctx->ls, ctx->st);
-      if (ev) cudaEventRecord(ev[2], ctx->st);
-      ctx->launches += launch_quantize_trigger(P, ctx->ls, ctx->st);
+      if (c.flags & LAQ_FLAG_QUANT_OFF) {
+        // no quantizer: one sweep gives the radius, the norm and the skip decisions (the radius slot stays empty)
+        if (ev) cudaEventRecord(ev[2], ctx->st);
+        ctx->launches += launch_innovation_trigger(P, ctx->ls, ctx->st);
+      } else {
+        ctx->launches += launch_radius(P, ctx->ls, ctx->st);
+        if (ev) cudaEventRecord(ev[2], ctx->st);
+        ctx->launches += launch_quantize_trigger(P, ctx->ls, ctx->st);
+      }
       if (ev) cudaEventRecord(ev[3], ctx->st);
       ctx->launches += launch_aggregate(P, ctx->ls, ctx->st);
     }
@@ -584,7 +590,7 @@ laq_status laq_tune(laq_ctx* ctx, const char* key, int32_t value) {
   auto pow2_threads = [](int v) { return v == 64 || v == 128 || v == 256 || v == 512; };
   if (k == "sweep_threads" && pow2_threads(value)) ctx->ls.sweep_threads = value;
   else if (k == "sweep_blocks_per_sm" && value >= 1 && value <= 128) ctx->ls.sweep_blocks_per_sm = value;
-  else if (k == "agg_threads" && pow2_threads(value)) ctx->ls.agg_threads = value;
+  else if (k == "agg_threads" && pow2_threads(value) && value <= 256) ctx->ls.agg_threads = value;
   else if (k == "agg_blocks_per_sm" && value >= 1 && value <= 32) ctx->ls.agg_blocks_per_sm = value;
   else if (k == "grad_blocks_per_worker" && value >= 1 && value <= ctx->gbpw_cap) ctx->gbpw = value;
   else return fail(ctx, LAQ_EINVAL, "unknown tuning key or value outside its limits");

@@ -90,6 +90,7 @@ struct LaunchShape {
 int launch_radius(const Params& P, const LaunchShape& ls, cudaStream_t st);
 bool small_iteration_applies(const Params& P);
 int launch_small_iteration(const Params& P, int gbpw_finalize, cudaStream_t st);
+int launch_innovation_trigger(const Params& P, const LaunchShape& ls, cudaStream_t st);
 int launch_quantize_trigger(const Params& P, const LaunchShape& ls, cudaStream_t st);
 int launch_aggregate(const Params& P, const LaunchShape& ls, cudaStream_t st);
 int launch_grad_logreg(const Params& P, const LaunchShape& ls, int gbpw, cudaStream_t st);

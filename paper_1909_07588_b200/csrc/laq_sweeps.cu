@@ -68,6 +68,9 @@ struct Synth {
   }
 };
 
+// asks for the line of ptr to be brought into L2; no register waits for it
+__device__ __forceinline__ void prefetch_l2(const void* ptr) { asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr)); }
+
 __device__ __forceinline__ uint32_t abs_bits(float x) { return __float_as_uint(x) & 0x7fffffffu; }
 
 __device__ __forceinline__ double warp_sum(double v) {
@@ -308,7 +311,9 @@ __device__ void trigger_stage(const Params& P, int bpw) {
     }
     sc->n_up = n;
     sc->uploads += (unsigned long long)n;
-    sc->bits += (unsigned long long)n * (32ull + (unsigned long long)P.b * (unsigned long long)P.p);
+    sc->bits += (unsigned long long)n * ((P.flags & LAQ_FLAG_QUANT_OFF)
+                                             ? 32ull * (unsigned long long)P.p
+                                             : 32ull + (unsigned long long)P.b * (unsigned long long)P.p);
     if (tracing) P.t_up[sc->trace_pos] = n;
   }
 }
@@ -436,94 +441,121 @@ __global__ void __launch_bounds__(512, LAQ_QUANT_MIN_BLOCKS) quantize_kernel(con
 }
 
 // ------------------------------------------------------------------------------------------------
+// Quantizer off (lazily aggregated gradients without quantization, the LAG baseline of Sec. 4; with the skip
+// rule off as well: plain gradient descent, Eq. (2)).  The innovation g_m - Q_prev is sent as it is, so one
+// sweep gives both its largest magnitude (kept for the report and the non-finite check) and its squared norm;
+// eps is zero.  The last block applies the same skip rule.
+// ------------------------------------------------------------------------------------------------
+template <bool SYNTH>
+__global__ void __launch_bounds__(512) innovation_kernel(const Params P) {
+  __shared__ double sh[32];
+  __shared__ uint32_t shm[32];
+  __shared__ bool is_last;
+  const int m = blockIdx.y;
+  const bool frozen = *(volatile uint32_t*)&P.sc->err != 0;
+  const unsigned long long k = P.sc->k;
+  double sdq = 0.0;
+  uint32_t mx = 0;
+  if (!frozen) {
+    Synth sy;
+    if (SYNTH) sy.init(P, m, k + 1);
+    const float4* __restrict__ q4 = reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps);
+    const float4* __restrict__ g4 = SYNTH ? nullptr : reinterpret_cast<const float4*>(P.g + (long long)m * P.ps);
+    const uint32_t nv = (uint32_t)P.nv, nv_main = (uint32_t)((P.p / 4) & ~1ll), stride = gridDim.x * blockDim.x;
+    double acc[4] = {0.0, 0.0, 0.0, 0.0};
+    auto take = [&](const float4& g, const float4& q) {
+      const float d0 = __fsub_rn(g.x, q.x), d1 = __fsub_rn(g.y, q.y), d2 = __fsub_rn(g.z, q.z), d3 = __fsub_rn(g.w, q.w);
+      mx = max(max(mx, abs_bits(d0)), max(abs_bits(d1), max(abs_bits(d2), abs_bits(d3))));
+      acc[0] = fma((double)d0, (double)d0, acc[0]);
+      acc[1] = fma((double)d1, (double)d1, acc[1]);
+      acc[2] = fma((double)d2, (double)d2, acc[2]);
+      acc[3] = fma((double)d3, (double)d3, acc[3]);
+    };
+    uint32_t v = blockIdx.x * blockDim.x + threadIdx.x;
+    for (; (unsigned long long)v + (kUnroll - 1) * (unsigned long long)stride < nv_main; v += kUnroll * stride) {
+      float4 q[kUnroll], g[kUnroll];
+#pragma unroll
+      for (int j = 0; j < kUnroll; ++j) {
+        q[j] = __ldg(q4 + (v + j * stride));
+        g[j] = SYNTH ? sy.at4(v + j * stride) : __ldg(g4 + (v + j * stride));
+      }
+#pragma unroll
+      for (int j = 0; j < kUnroll; ++j) take(g[j], q[j]);
+    }
+    for (; v < nv_main; v += stride) take(SYNTH ? sy.at4(v) : __ldg(g4 + v), __ldg(q4 + v));
+    if (blockIdx.x == 0 && nv_main + threadIdx.x < nv) {   // padding of Q_prev and of a stored g is zero
+      const uint32_t vt = nv_main + threadIdx.x;
+      take(SYNTH ? sy.at4_masked(vt, P.p) : __ldg(g4 + vt), __ldg(q4 + vt));
+    }
+    sdq = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+  }
+  mx = __reduce_max_sync(0xffffffffu, mx);
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  if (lane == 0) shm[w] = mx;
+  const double tdq = block_sum(sdq, sh);   // its barriers also publish shm
+  if (w == 0) {
+    mx = (lane < ((blockDim.x + 31) >> 5)) ? shm[lane] : 0u;
+    mx = __reduce_max_sync(0xffffffffu, mx);
+  }
+  if (threadIdx.x == 0) {
+    if (!frozen) atomicMax(&P.Rbits[(k & 1ull) * P.M + m], mx);
+    double* pq = P.part_q + ((long long)m * kMaxSweepBlocksPerWorker + blockIdx.x) * 2;
+    __stcg(pq, tdq);
+    __stcg(pq + 1, 0.0);
+    __threadfence();
+    const uint32_t total = gridDim.x * gridDim.y;
+    const uint32_t ticket = atomicAdd(&P.sc->cnt_quant, 1u);
+    is_last = (ticket == total - 1);
+    if (is_last) P.sc->cnt_quant = 0;
+  }
+  __syncthreads();
+  if (is_last && !frozen) {
+    __threadfence();
+    trigger_stage(P, gridDim.x);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // lazy aggregate + theta step
 // ------------------------------------------------------------------------------------------------
-constexpr int kAggBatch = 4;  // uploaders whose loads are issued together
+#ifndef LAQ_AGG_AHEAD
+#define LAQ_AGG_AHEAD 4
+#endif
+#ifndef LAQ_AGG_MIN_BLOCKS
+#define LAQ_AGG_MIN_BLOCKS 5   // 48 registers, no spills
+#endif
+constexpr int kAggAhead = LAQ_AGG_AHEAD;  // uploaders whose row and code lines are requested into L2 ahead of use
 
 // exact float of a code < 2^23 through the mantissa of 2^23
 __device__ __forceinline__ float code_to_float(uint32_t c) { return __uint_as_float(0x4b000000u | c) - 8388608.0f; }
 
-template <int B>
-__global__ void __launch_bounds__(512) aggregate_kernel(const Params P) {
-  __shared__ int s_m[kMaxWorkers];
-  __shared__ float s_R[kMaxWorkers];
-  __shared__ float s_s[kMaxWorkers];
-  __shared__ double sh[32];
-  __shared__ bool is_last;
-  if (*(volatile uint32_t*)&P.sc->err) return;
-  const int n_up = (int)P.sc->n_up;
-  for (int u = threadIdx.x; u < n_up; u += blockDim.x) {
-    s_m[u] = P.up_m[u];
-    s_R[u] = P.up_R[u];
-    s_s[u] = P.up_s[u];
-  }
-  __syncthreads();
-  const long long nv = P.nv, p = P.p, stride = (long long)gridDim.x * blockDim.x;
-  float4* __restrict__ agg4 = reinterpret_cast<float4*>(P.agg);
-  float4* __restrict__ th4 = reinterpret_cast<float4*>(P.theta);
+// grad^k is complete for group v: store it, take the step theta -= alpha grad (Eq. (4)) and add to the fp64 sums
+// of ||alpha grad||^2 and ||theta||^2.
+__device__ __forceinline__ void theta_step(const Params& P, uint32_t v, const float4& a, double& dsum, double& tsum) {
+  reinterpret_cast<float4*>(P.agg)[v] = a;
+  float4* th4 = reinterpret_cast<float4*>(P.theta);
+  float4 th = th4[v];
   const float alpha = P.alpha;
-  double dsum = 0.0, tsum = 0.0;
-  for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < nv; v += stride) {
-    float4 a = agg4[v];
-    const long long i = 4 * v;
-    const bool tail = i + 3 >= p;
-    for (int u0 = 0; u0 < n_up; u0 += kAggBatch) {
-      float4 q[kAggBatch];
-      uint32_t c[kAggBatch][4];
-#pragma unroll
-      for (int j = 0; j < kAggBatch; ++j) {
-        if (u0 + j < n_up) {
-          const int m = s_m[u0 + j];
-          q[j] = *(reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps) + v);
-          load_codes<B>(P.codes + (long long)m * P.cw, v, c[j]);
-        }
-      }
-#pragma unroll
-      for (int j = 0; j < kAggBatch; ++j) {
-        if (u0 + j < n_up) {
-          const int m = s_m[u0 + j];
-          const float R = s_R[u0 + j], s = s_s[u0 + j];
-          // the server's recovery of the innovation from the message: dQ = 2 tau R q - R
-          float d0 = __fsub_rn(__fmul_rn(s, code_to_float(c[j][0])), R);
-          float d1 = __fsub_rn(__fmul_rn(s, code_to_float(c[j][1])), R);
-          float d2 = __fsub_rn(__fmul_rn(s, code_to_float(c[j][2])), R);
-          float d3 = __fsub_rn(__fmul_rn(s, code_to_float(c[j][3])), R);
-          if (tail) {  // padding coordinates carry no innovation
-            if (i >= p) d0 = 0.f;
-            if (i + 1 >= p) d1 = 0.f;
-            if (i + 2 >= p) d2 = 0.f;
-            if (i + 3 >= p) d3 = 0.f;
-          }
-          q[j].x = __fadd_rn(q[j].x, d0);
-          q[j].y = __fadd_rn(q[j].y, d1);
-          q[j].z = __fadd_rn(q[j].z, d2);
-          q[j].w = __fadd_rn(q[j].w, d3);
-          *(reinterpret_cast<float4*>(P.qp + (long long)m * P.ps) + v) = q[j];
-          a.x = __fadd_rn(a.x, d0);  // uploads are applied in ascending worker order
-          a.y = __fadd_rn(a.y, d1);
-          a.z = __fadd_rn(a.z, d2);
-          a.w = __fadd_rn(a.w, d3);
-        }
-      }
-    }
-    agg4[v] = a;
-    float4 th = th4[v];
-    const float u0 = __fmul_rn(alpha, a.x), u1 = __fmul_rn(alpha, a.y), u2 = __fmul_rn(alpha, a.z),
-                u3 = __fmul_rn(alpha, a.w);
-    th.x = __fsub_rn(th.x, u0);
-    th.y = __fsub_rn(th.y, u1);
-    th.z = __fsub_rn(th.z, u2);
-    th.w = __fsub_rn(th.w, u3);
-    th4[v] = th;
-    dsum = fma((double)u0, (double)u0, dsum);
-    dsum = fma((double)u1, (double)u1, dsum);
-    dsum = fma((double)u2, (double)u2, dsum);
-    dsum = fma((double)u3, (double)u3, dsum);
-    tsum = fma((double)th.x, (double)th.x, tsum);
-    tsum = fma((double)th.y, (double)th.y, tsum);
-    tsum = fma((double)th.z, (double)th.z, tsum);
-    tsum = fma((double)th.w, (double)th.w, tsum);
-  }
+  const float u0 = __fmul_rn(alpha, a.x), u1 = __fmul_rn(alpha, a.y), u2 = __fmul_rn(alpha, a.z),
+              u3 = __fmul_rn(alpha, a.w);
+  th.x = __fsub_rn(th.x, u0);
+  th.y = __fsub_rn(th.y, u1);
+  th.z = __fsub_rn(th.z, u2);
+  th.w = __fsub_rn(th.w, u3);
+  th4[v] = th;
+  dsum = fma((double)u0, (double)u0, dsum);
+  dsum = fma((double)u1, (double)u1, dsum);
+  dsum = fma((double)u2, (double)u2, dsum);
+  dsum = fma((double)u3, (double)u3, dsum);
+  tsum = fma((double)th.x, (double)th.x, tsum);
+  tsum = fma((double)th.y, (double)th.y, tsum);
+  tsum = fma((double)th.z, (double)th.z, tsum);
+  tsum = fma((double)th.w, (double)th.w, tsum);
+}
+
+// Block partials of the two sums; the last block to arrive adds them in a fixed order, pushes ||alpha grad||^2 onto
+// the ring of stored differences, writes the trace row and advances k.
+__device__ __forceinline__ void aggregate_finish(const Params& P, double dsum, double tsum, double* sh, bool* is_last_sh) {
   const double bs = block_sum(dsum, sh);
   const double bt = block_sum(tsum, sh);
   if (threadIdx.x == 0) {
@@ -531,11 +563,11 @@ __global__ void __launch_bounds__(512) aggregate_kernel(const Params P) {
     __stcg(P.part_t + blockIdx.x, bt);
     __threadfence();
     const uint32_t ticket = atomicAdd(&P.sc->cnt_agg, 1u);
-    is_last = (ticket == gridDim.x - 1);
-    if (is_last) P.sc->cnt_agg = 0;
+    *is_last_sh = (ticket == gridDim.x - 1);
+    if (*is_last_sh) P.sc->cnt_agg = 0;
   }
   __syncthreads();
-  if (!is_last) return;
+  if (!*is_last_sh) return;
   __threadfence();
   // ||theta^{k+1} - theta^k||^2 = ||alpha grad^k||^2 : fixed-order sum of the block partials
   double t = 0.0, t2 = 0.0;
@@ -560,6 +592,125 @@ __global__ void __launch_bounds__(512) aggregate_kernel(const Params P) {
     }
     sc->k += 1ull;
   }
+}
+
+template <int B>
+__device__ __forceinline__ const void* code_address(const uint32_t* row, uint32_t v) {
+  return reinterpret_cast<const uint8_t*>(row) + ((B == 1) ? (size_t)(v >> 1) : (size_t)v * (size_t)(B / 2));
+}
+
+// A thread owns groups v, v + stride, ...  Per group it holds only the aggregate in registers and walks the
+// uploaders in ascending worker order; latency is covered by occupancy (few registers) and by requesting the
+// lines of the uploaders ahead, and of theta, into L2 before they are needed.
+template <int B>
+__global__ void __launch_bounds__(256, LAQ_AGG_MIN_BLOCKS) aggregate_kernel(const Params P) {
+  __shared__ int s_m[kMaxWorkers];
+  __shared__ float s_R[kMaxWorkers];
+  __shared__ float s_s[kMaxWorkers];
+  __shared__ double sh[32];
+  __shared__ bool is_last;
+  if (*(volatile uint32_t*)&P.sc->err) return;
+  const int n_up = (int)P.sc->n_up;
+  for (int u = threadIdx.x; u < n_up; u += blockDim.x) {
+    s_m[u] = P.up_m[u];
+    s_R[u] = P.up_R[u];
+    s_s[u] = P.up_s[u];
+  }
+  __syncthreads();
+  // p < 2^32, so group indices fit 32 bits; groups >= v_full contain padding coordinates
+  const uint32_t nv = (uint32_t)P.nv, v_full = (uint32_t)(P.p >> 2), stride = gridDim.x * blockDim.x;
+  double dsum = 0.0, tsum = 0.0;
+  for (uint32_t v = blockIdx.x * blockDim.x + threadIdx.x; v < nv; v += stride) {
+    float4 a = reinterpret_cast<const float4*>(P.agg)[v];
+    prefetch_l2(reinterpret_cast<const float4*>(P.theta) + v);
+#pragma unroll
+    for (int j = 0; j < kAggAhead; ++j)
+      if (j < n_up) {
+        const int m = s_m[j];
+        prefetch_l2(reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps) + v);
+        prefetch_l2(code_address<B>(P.codes + (long long)m * P.cw, v));
+      }
+    for (int u = 0; u < n_up; ++u) {
+      if (u + kAggAhead < n_up) {
+        const int m = s_m[u + kAggAhead];
+        prefetch_l2(reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps) + v);
+        prefetch_l2(code_address<B>(P.codes + (long long)m * P.cw, v));
+      }
+      const int m = s_m[u];
+      float4* qptr = reinterpret_cast<float4*>(P.qp + (long long)m * P.ps) + v;
+      float4 q = *qptr;
+      uint32_t c[4];
+      load_codes<B>(P.codes + (long long)m * P.cw, v, c);
+      const float R = s_R[u], s = s_s[u];
+      // the server's recovery of the innovation from the message: dQ = 2 tau R q - R
+      float d0 = __fsub_rn(__fmul_rn(s, code_to_float(c[0])), R);
+      float d1 = __fsub_rn(__fmul_rn(s, code_to_float(c[1])), R);
+      float d2 = __fsub_rn(__fmul_rn(s, code_to_float(c[2])), R);
+      float d3 = __fsub_rn(__fmul_rn(s, code_to_float(c[3])), R);
+      if (v >= v_full) {  // padding coordinates carry no innovation
+        const long long i = 4ll * v;
+        if (i >= P.p) d0 = 0.f;
+        if (i + 1 >= P.p) d1 = 0.f;
+        if (i + 2 >= P.p) d2 = 0.f;
+        d3 = 0.f;
+      }
+      q.x = __fadd_rn(q.x, d0);
+      q.y = __fadd_rn(q.y, d1);
+      q.z = __fadd_rn(q.z, d2);
+      q.w = __fadd_rn(q.w, d3);
+      *qptr = q;
+      a.x = __fadd_rn(a.x, d0);  // uploads are applied in ascending worker order
+      a.y = __fadd_rn(a.y, d1);
+      a.z = __fadd_rn(a.z, d2);
+      a.w = __fadd_rn(a.w, d3);
+    }
+    theta_step(P, v, a, dsum, tsum);
+  }
+  aggregate_finish(P, dsum, tsum, sh, &is_last);
+}
+
+// Quantizer off: an uploader's innovation is g_m - Q_prev itself and Q_prev becomes g_m.
+template <bool SYNTH>
+__global__ void __launch_bounds__(256, 4) aggregate_raw_kernel(const Params P) {
+  __shared__ int s_m[kMaxWorkers];
+  __shared__ double sh[32];
+  __shared__ bool is_last;
+  if (*(volatile uint32_t*)&P.sc->err) return;
+  const int n_up = (int)P.sc->n_up;
+  const unsigned long long k = P.sc->k;
+  for (int u = threadIdx.x; u < n_up; u += blockDim.x) s_m[u] = P.up_m[u];
+  __syncthreads();
+  const uint32_t nv = (uint32_t)P.nv, v_full = (uint32_t)(P.p >> 2), stride = gridDim.x * blockDim.x;
+  double dsum = 0.0, tsum = 0.0;
+  for (uint32_t v = blockIdx.x * blockDim.x + threadIdx.x; v < nv; v += stride) {
+    float4 a = reinterpret_cast<const float4*>(P.agg)[v];
+    prefetch_l2(reinterpret_cast<const float4*>(P.theta) + v);
+    for (int u = 0; u < n_up; ++u) {
+      if (u + 1 < n_up) {
+        const int m1 = s_m[u + 1];
+        prefetch_l2(reinterpret_cast<const float4*>(P.qp + (long long)m1 * P.ps) + v);
+        if (!SYNTH) prefetch_l2(reinterpret_cast<const float4*>(P.g + (long long)m1 * P.ps) + v);
+      }
+      const int m = s_m[u];
+      float4* qptr = reinterpret_cast<float4*>(P.qp + (long long)m * P.ps) + v;
+      const float4 q = *qptr;
+      float4 g;
+      if (SYNTH) {
+        Synth sy;
+        sy.init(P, m, k + 1);
+        g = (v >= v_full) ? sy.at4_masked(v, P.p) : sy.at4(v);
+      } else {
+        g = __ldg(reinterpret_cast<const float4*>(P.g + (long long)m * P.ps) + v);
+      }
+      *qptr = g;
+      a.x = __fadd_rn(a.x, __fsub_rn(g.x, q.x));  // uploads are applied in ascending worker order
+      a.y = __fadd_rn(a.y, __fsub_rn(g.y, q.y));
+      a.z = __fadd_rn(a.z, __fsub_rn(g.z, q.z));
+      a.w = __fadd_rn(a.w, __fsub_rn(g.w, q.w));
+    }
+    theta_step(P, v, a, dsum, tsum);
+  }
+  aggregate_finish(P, dsum, tsum, sh, &is_last);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -830,7 +981,7 @@ int aggregate_blocks(const Params& P, const LaunchShape& ls) {
 }
 
 bool small_iteration_applies(const Params& P) {
-  return P.model != LAQ_MODEL_SYNTH && (long long)P.M * P.ps <= 8192;
+  return P.model != LAQ_MODEL_SYNTH && !(P.flags & LAQ_FLAG_QUANT_OFF) && (long long)P.M * P.ps <= 8192;
 }
 
 int launch_small_iteration(const Params& P, int gbpw_finalize, cudaStream_t st) {
@@ -853,6 +1004,15 @@ int launch_radius(const Params& P, const LaunchShape& ls, cudaStream_t st) {
   return 1;
 }
 
+int launch_innovation_trigger(const Params& P, const LaunchShape& ls, cudaStream_t st) {
+  dim3 grid(sweep_blocks_per_worker(P, ls), P.M);
+  if (P.model == LAQ_MODEL_SYNTH)
+    innovation_kernel<true><<<grid, ls.sweep_threads, 0, st>>>(P);
+  else
+    innovation_kernel<false><<<grid, ls.sweep_threads, 0, st>>>(P);
+  return 1;
+}
+
 int launch_quantize_trigger(const Params& P, const LaunchShape& ls, cudaStream_t st) {
   dim3 grid(sweep_blocks_per_worker(P, ls), P.M);
   if (P.model == LAQ_MODEL_SYNTH)
@@ -864,6 +1024,13 @@ int launch_quantize_trigger(const Params& P, const LaunchShape& ls, cudaStream_t
 
 int launch_aggregate(const Params& P, const LaunchShape& ls, cudaStream_t st) {
   const int nb = aggregate_blocks(P, ls);
+  if (P.flags & LAQ_FLAG_QUANT_OFF) {
+    if (P.model == LAQ_MODEL_SYNTH)
+      aggregate_raw_kernel<true><<<nb, ls.agg_threads, 0, st>>>(P);
+    else
+      aggregate_raw_kernel<false><<<nb, ls.agg_threads, 0, st>>>(P);
+    return 1;
+  }
   switch (P.b) {
     case 1: aggregate_kernel<1><<<nb, ls.agg_threads, 0, st>>>(P); break;
     case 2: aggregate_kernel<2><<<nb, ls.agg_threads, 0, st>>>(P); break;

@@ -14,6 +14,7 @@ LIB_PATH = os.path.join(_HERE, "csrc", "liblaq_b200.so")
 LAQ_OK, LAQ_EINVAL, LAQ_EWORKSPACE, LAQ_ECUDA, LAQ_ENONFINITE, LAQ_ESTATE = range(6)
 STATUS_NAMES = ["LAQ_OK", "LAQ_EINVAL", "LAQ_EWORKSPACE", "LAQ_ECUDA", "LAQ_ENONFINITE", "LAQ_ESTATE"]
 MODEL_LOGREG_BIN, MODEL_SOFTMAX, MODEL_MLP2, MODEL_SYNTH, MODEL_EXTERNAL = range(5)
+FLAG_QUANT_OFF = 1
 FLAG_TRIGGER_OFF = 2
 
 EXPORTS = ["laq_workspace_bytes", "laq_init", "laq_load_shards", "laq_set_gradients", "laq_step", "laq_sync",

@@ -113,6 +113,73 @@ def test_given_gradients_zero_innovation_and_trigger_off():
     ctx.close()
 
 
+@pytest.mark.parametrize("flags", [laq.FLAG_QUANT_OFF, laq.FLAG_QUANT_OFF | laq.FLAG_TRIGGER_OFF])
+@pytest.mark.parametrize("p", [3, 1000, 70001])
+def test_quantizer_off_given_gradients_bit_exact(p, flags):
+    """No quantizer (lazily aggregated gradients; with the skip rule off too: gradient descent, Eq. (2))."""
+    assert (laq.FLAG_QUANT_OFF, laq.FLAG_TRIGGER_OFF) == (oracle.FLAG_QUANT_OFF, oracle.FLAG_TRIGGER_OFF)
+    M, D, tbar, alpha, iters = 5, 4, 6, 0.05, 25 if p < 10000 else 8
+    rng = np.random.default_rng(77 + p)
+    c = rng.standard_normal((M, p))
+    Lm = rng.uniform(0.05, 2.0, M)
+    kw = dict(alpha=alpha, b=4, D=D, xi=np.full(D, 0.2), tbar=tbar, flags=flags)
+    ctx = laq.Laq(model=laq.MODEL_EXTERNAL, M=M, p=p, trace_capacity=1, **kw)
+    mir = oracle.OracleLaq(32, oracle.MODEL_GIVEN, M, p, **kw)
+    theta = np.zeros(p, np.float32)
+    skipped = 0
+    for k in range(iters):
+        g = (Lm[:, None] * (theta.astype(np.float64)[None, :] - c)).astype(np.float32)
+        ctx.set_gradients(g)
+        tr = ctx.step(1, trace=True)
+        st = mir.step_given(g)
+        _assert_trace_row(tr, 0, st)
+        assert not tr["n_eps"].any()
+        gs = ctx.get_state(codes=True)
+        _assert_state_bit_exact(gs, mir.state(), p, 4)         # codes: never written, all zero on both sides
+        theta = gs["theta"]
+        skipped += int(st["skip"].sum())
+    assert (skipped > 0) == (flags == laq.FLAG_QUANT_OFF)
+    assert ctx.get_state()["bits"] == ctx.get_state()["uploads"] * 32 * p
+    ctx.close()
+
+
+def test_quantizer_off_synthetic_stream_bit_exact():
+    M, p, iters = 8, 70001, 30
+    w = workloads.c4(M=M, p=p, b=8, iters=iters)
+    ctx = laq.from_workload(w, trace_capacity=iters, flags=laq.FLAG_QUANT_OFF)
+    mir = _mirror_for(w, flags=oracle.FLAG_QUANT_OFF)
+    tr = ctx.step(iters, trace=True)
+    for j in range(iters):
+        _assert_trace_row(tr, j, mir.step())
+    _assert_state_bit_exact(ctx.get_state(codes=True), mir.state(), p, 8)
+    assert 0 < tr["skip"].sum() < M * iters
+    ctx.close()
+
+
+def test_quantizer_off_model_workload_follows_the_fp64_oracle():
+    """C0 without the quantizer: the library's own gradients, skip masks and theta against the fp64 oracle."""
+    w = workloads.c0()
+    ctx = laq.from_workload(w, trace_capacity=1, flags=laq.FLAG_QUANT_OFF)
+    o64 = _mirror_for(w, 64, flags=oracle.FLAG_QUANT_OFF)
+    mir = oracle.OracleLaq(32, oracle.MODEL_GIVEN, w.M, w.p, alpha=w.alpha, b=w.b, D=w.D, xi=w.xi, tbar=w.tbar,
+                           theta0=w.theta0, flags=oracle.FLAG_QUANT_OFF)
+    agree = 0
+    for k in range(120):
+        tr = ctx.step(1, trace=True)
+        gs = ctx.get_state(g=True, codes=True)
+        _assert_trace_row(tr, 0, mir.step_given(gs["g"]))       # steps 2-5 on the library's own gradients
+        _assert_state_bit_exact(gs, mir.state(), w.p, w.b)
+        st = o64.step()
+        if agree == k and np.array_equal(st["skip"].astype(np.uint8), tr["skip"][0]):
+            agree += 1
+            th = o64.state(big=False)["theta"]
+            assert np.linalg.norm(gs["theta"] - th) <= TRAJ_RTOL * np.linalg.norm(th)
+            assert tr["loss"][0] == pytest.approx(st["loss"], rel=TRAJ_RTOL)
+    print("quantizer off, C0: skip masks equal to the fp64 oracle's for the first %d of 120 iterations" % agree)
+    assert agree >= 20
+    ctx.close()
+
+
 def test_strict_clock_tbar_one_never_skips():
     M, p = 4, 64
     rng = np.random.default_rng(3)

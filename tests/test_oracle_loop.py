@@ -107,6 +107,65 @@ def test_trigger_off_is_qgd(precision):
     assert s["bits"] == M * K * (32 + b * p)          # cost of a message, text after Eq. (6)
 
 
+def test_quantizer_and_trigger_off_is_gradient_descent():
+    """Eq. (2): with no quantizer and no skipping, theta^{k+1} = theta^k - alpha sum_m grad f_m(theta^k)."""
+    rng = np.random.default_rng(5)
+    M, p, K, alpha = 5, 12, 40, 0.0625
+    _, grad = _quadratic_problem(rng, M, p, rng.uniform(0.5, 1.5, M))
+    o = oracle.OracleLaq(64, oracle.MODEL_GIVEN, M, p, alpha=alpha, b=4, D=3, tbar=10,
+                         flags=oracle.FLAG_TRIGGER_OFF | oracle.FLAG_QUANT_OFF)
+    theta = np.zeros(p)
+    for k in range(K):
+        g = grad(theta)
+        st = o.step_given(g)
+        assert not st["skip"].any() and not st["n_eps"].any()
+        np.testing.assert_allclose(st["R"], np.abs(g - (grad_prev if k else 0.0)).max(1), rtol=1e-12)
+        grad_prev = g
+        theta = theta - alpha * g.sum(0)
+        np.testing.assert_allclose(o.state(big=False)["theta"], theta, rtol=1e-11, atol=1e-13)
+    s = o.state()
+    np.testing.assert_array_equal(s["qp"], grad_prev)           # the server holds the exact last gradients
+    assert s["uploads"] == M * K and s["bits"] == M * K * 32 * p
+
+
+def test_quantizer_off_is_lazily_aggregated_gradient_descent():
+    """Without the quantizer the skip rule (7a) has eps = 0 and reads
+    ||grad f_m(theta^k) - grad f_m(theta_hat_m)||^2 <= (1 / (alpha^2 M^2)) sum_d xi_d ||theta^{k+1-d} - theta^{k-d}||^2,
+    the worker-side rule of the lazily aggregated gradient method that Sec. 4 compares with; simulated here directly."""
+    rng = np.random.default_rng(6)
+    M, p, K, alpha, D, tbar = 6, 10, 80, 0.0625, 4, 7
+    xi = np.array([0.3, 0.2, 0.15, 0.1])
+    _, grad = _quadratic_problem(rng, M, p, rng.uniform(0.1, 2.0, M))
+    o = oracle.OracleLaq(64, oracle.MODEL_GIVEN, M, p, alpha=alpha, b=4, D=D, xi=xi, tbar=tbar,
+                         flags=oracle.FLAG_QUANT_OFF)
+    theta = np.zeros(p)
+    held = np.zeros((M, p))                  # grad f_m(theta_hat_m) as the server holds it
+    clock = np.full(M, tbar + 1)
+    diffs = [0.0] * D                        # newest first
+    total_skips = 0
+    for k in range(K):
+        g = grad(theta)
+        st = o.step_given(g)
+        rhs = float(np.dot(xi, diffs)) / (alpha * alpha * M * M)
+        skip = np.zeros(M, bool)
+        for m in range(M):
+            skip[m] = (np.sum((g[m] - held[m]) ** 2) <= rhs) and clock[m] <= tbar
+            if skip[m]:
+                clock[m] += 1
+            else:
+                held[m] = g[m]
+                clock[m] = 0
+        np.testing.assert_array_equal(st["skip"].astype(bool), skip)
+        new_theta = theta - alpha * held.sum(0)
+        diffs = [float(np.sum((new_theta - theta) ** 2))] + diffs[:-1]
+        theta = new_theta
+        np.testing.assert_allclose(o.state(big=False)["theta"], theta, rtol=1e-10, atol=1e-13)
+        total_skips += int(skip.sum())
+    assert 0 < total_skips < M * K
+    s = o.state(big=False)
+    assert s["uploads"] == M * K - total_skips and s["bits"] == s["uploads"] * 32 * p
+
+
 def test_first_iteration_uploads_and_staleness_clock():
     rng = np.random.default_rng(2)
     M, p = 6, 20
