@@ -27,7 +27,8 @@
  *     Q_new = Q_prev + dQ ; eps = g - Q_new, with no fused multiply-add; squared norms are fp64 sums of
  *     exact fp32 products; the skip rule is evaluated in fp64.
  *   - Code stream of worker m (the paper's b p-bit part of the upload message): code i occupies bits
- *     [(i b) mod 32, +b) of 32-bit word floor(i b / 32), least significant first.
+ *     [i b, (i+1) b) of the stream, bit j of the stream being bit (j mod 32) of 32-bit word floor(j / 32)
+ *     (least significant first; for b = 3 a code may straddle two words).
  *   - Readings where the paper is silent: initial Q_m = 0, ||eps_hat_m||^2 = 0, grad^0 = 0, the D stored
  *     squared parameter differences start at 0, clocks start at t_bar + 1 (every worker uploads at
  *     k = 1); R_m = 0 yields q = 0, dQ = 0; ||theta^{k+1}-theta^k||^2 is taken as ||alpha grad^k||^2.
@@ -91,7 +92,7 @@ typedef struct {
   int32_t n_hidden;         /* H (MLP2) */
   float alpha;              /* step size */
   float lambda;             /* l2 regulariser */
-  int32_t b;                /* bits per coordinate: 1, 2, 4, 8 or 16 */
+  int32_t b;                /* bits per coordinate: 1, 2, 3, 4, 8 or 16 */
   int32_t D;                /* number of stored parameter differences, 1..64; the paper requires D <= t_bar */
   const float* xi;          /* HOST, length D: weights xi_1..xi_D of (7a), xi[0] pairs with the newest difference */
   int32_t tbar;             /* staleness bound of (7b) */

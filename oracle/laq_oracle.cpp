@@ -139,22 +139,24 @@ void decode(T R, const int32_t* q, const T* qp, i64 p, int b, T* qnew, T* dq) {
   }
 }
 
-// The upload message's code stream: code i occupies bits [(i b) mod 32, +b) of 32-bit word
-// floor(i b / 32), least significant first.  b must divide 32 here (1,2,4,8,16,32).
+// The upload message's code stream (the b p bits of the message, text after Eq. (6)): code i occupies
+// bits [i b, (i+1) b) of the stream; stream bit j is bit (j mod 32) of 32-bit word floor(j / 32), least
+// significant first.  Written bit by bit, so a code may straddle two words (b = 3).
 void pack_codes(const int32_t* q, i64 p, int b, uint32_t* words, i64 n_words) {
   for (i64 w = 0; w < n_words; ++w) words[w] = 0;
-  for (i64 i = 0; i < p; ++i) {
-    i64 bit = i * (i64)b;
-    uint32_t v = (uint32_t)q[i];
-    if (b < 32) v &= ((1u << b) - 1u);
-    words[bit / 32] |= v << (bit % 32);
-  }
+  for (i64 i = 0; i < p; ++i)
+    for (int t = 0; t < b; ++t) {
+      i64 bit = i * (i64)b + t;
+      if (((uint32_t)q[i] >> t) & 1u) words[bit / 32] |= 1u << (bit % 32);
+    }
 }
 void unpack_codes(const uint32_t* words, i64 p, int b, int32_t* q) {
   for (i64 i = 0; i < p; ++i) {
-    i64 bit = i * (i64)b;
-    uint32_t v = words[bit / 32] >> (bit % 32);
-    if (b < 32) v &= ((1u << b) - 1u);
+    uint32_t v = 0;
+    for (int t = 0; t < b; ++t) {
+      i64 bit = i * (i64)b + t;
+      v |= ((words[bit / 32] >> (bit % 32)) & 1u) << t;
+    }
     q[i] = (int32_t)v;
   }
 }

@@ -46,7 +46,7 @@ constexpr int kProfIters = 512;
 
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
-bool valid_b(int b) { return b == 1 || b == 2 || b == 4 || b == 8 || b == 16; }
+bool valid_b(int b) { return b == 1 || b == 2 || b == 3 || b == 4 || b == 8 || b == 16; }
 
 long long model_p(const laq_config& c) {
   switch (c.model) {
@@ -63,7 +63,7 @@ const char* check_config(const laq_config* c) {
   if (c->model < 0 || c->model > LAQ_MODEL_EXTERNAL) return "unknown model";
   if (c->M < 1 || c->M > kMaxWorkers) return "M must be in 1..1024";
   if (c->p < 1 || c->p >= (1ll << 32)) return "p must be in 1..2^32-1";
-  if (!valid_b(c->b)) return "b must be 1, 2, 4, 8 or 16";
+  if (!valid_b(c->b)) return "b must be 1, 2, 3, 4, 8 or 16";
   if (c->D < 1 || c->D > kMaxD) return "D must be in 1..64";
   if (!c->xi) return "xi is null";
   if (!(c->alpha > 0.f) || !std::isfinite(c->alpha)) return "alpha must be positive and finite";

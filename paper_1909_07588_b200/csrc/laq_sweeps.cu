@@ -166,11 +166,27 @@ __global__ void __launch_bounds__(512) radius_kernel(const Params P) {
 // ------------------------------------------------------------------------------------------------
 // code packing: the 4 codes of coordinates 4v..4v+3 form one 4b-bit field at bit 4vb of the row
 // ------------------------------------------------------------------------------------------------
+// All 32 lanes of a warp call this together with v = (a multiple of 32) + lane (the 1-bit and 3-bit packings
+// combine neighbouring lanes); cw is the number of words of the row.
 template <int B>
 __device__ __forceinline__ void store_codes(uint32_t* row, uint32_t v, uint32_t y0, uint32_t y1, uint32_t y2,
-                                            uint32_t y3, bool valid) {
+                                            uint32_t y3, bool valid, long long cw) {
   // y_e = 0x4b000000 + code_e: the code sits in the low bits
-  if (B == 16) {
+  if (B == 3) {
+    // eight neighbouring groups (32 coordinates) fill three words: the 12-bit field of group v starts at bit
+    // 12 (v mod 8) of that 96-bit chunk and may straddle two of its words
+    const uint32_t field = valid ? ((y0 & 7u) | ((y1 & 7u) << 3) | ((y2 & 7u) << 6) | ((y3 & 7u) << 9)) : 0u;
+    const uint32_t r = v & 7u, off = 12u * r, wi = off >> 5;
+    const unsigned long long t = (unsigned long long)field << (off & 31u);
+    const uint32_t lo = (uint32_t)t, hi = (uint32_t)(t >> 32);
+    const uint32_t octet = 0xffu << (threadIdx.x & 24u);
+    const uint32_t w0 = __reduce_or_sync(octet, wi == 0 ? lo : 0u);
+    const uint32_t w1 = __reduce_or_sync(octet, wi == 1 ? lo : (wi == 0 ? hi : 0u));
+    const uint32_t w2 = __reduce_or_sync(octet, wi == 2 ? lo : (wi == 1 ? hi : 0u));
+    const bool any_valid = __ballot_sync(octet, valid) != 0u;
+    const long long word = 3ll * (v >> 3) + r;
+    if (any_valid && r < 3u && word < cw) row[word] = r == 0 ? w0 : (r == 1 ? w1 : w2);
+  } else if (B == 16) {
     if (valid) reinterpret_cast<uint2*>(row)[v] = make_uint2(__byte_perm(y0, y1, 0x5410), __byte_perm(y2, y3, 0x5410));
   } else if (B == 8) {
     if (valid) row[v] = __byte_perm(__byte_perm(y0, y1, 0x0040), __byte_perm(y2, y3, 0x0040), 0x5410);
@@ -195,6 +211,13 @@ __device__ __forceinline__ void load_codes(const uint32_t* row, long long v, uin
   } else if (B == 8) {
     uint32_t w = __ldg(row + v);
     c[0] = w & 255u; c[1] = (w >> 8) & 255u; c[2] = (w >> 16) & 255u; c[3] = w >> 24;
+  } else if (B == 3) {
+    const long long bit = 12ll * v;
+    const uint32_t sh = (uint32_t)bit & 31u;
+    const uint32_t lo = __ldg(row + (bit >> 5));
+    const uint32_t hi = sh > 20u ? __ldg(row + (bit >> 5) + 1) : 0u;   // the field ends in the next word
+    const uint32_t w = __funnelshift_r(lo, hi, sh);
+    c[0] = w & 7u; c[1] = (w >> 3) & 7u; c[2] = (w >> 6) & 7u; c[3] = (w >> 9) & 7u;
   } else if (B == 4) {
     uint32_t w = __ldg(reinterpret_cast<const uint16_t*>(row) + v);
     c[0] = w & 15u; c[1] = (w >> 4) & 15u; c[2] = (w >> 8) & 15u; c[3] = (w >> 12) & 15u;
@@ -320,8 +343,9 @@ __device__ void trigger_stage(const Params& P, int bpw) {
 
 // The per-worker sweep of quantize_kernel (R > 0).  FAST selects the reciprocal-based exact division.
 // Groups [0, nv_main) lie wholly inside the row and run without masks; the few groups after them are
-// handled by the first warp of the worker's first block with per-coordinate masks.  nv_main is even,
-// so the lane pairs of the 1-bit packing never straddle the two parts.
+// handled by the first warp of the worker's first block with per-coordinate masks.  nv_main is even (a multiple
+// of 8 for b = 3), so the lane pairs of the 1-bit packing (the lane octets of the 3-bit packing) never straddle
+// the two parts.
 template <bool SYNTH, int B, bool FAST>
 __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned long long k, float R, float s,
                                                double& sdq, double& seps) {
@@ -332,7 +356,8 @@ __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned 
   const float4* __restrict__ g4 = SYNTH ? nullptr : reinterpret_cast<const float4*>(P.g + (long long)m * P.ps);
   uint32_t* row = P.codes + (long long)m * P.cw;
   const long long p = P.p;
-  const uint32_t nv = (uint32_t)P.nv, nv_main = (uint32_t)((p / 4) & ~1ll), stride = gridDim.x * blockDim.x;
+  const uint32_t nv = (uint32_t)P.nv, nv_main = (uint32_t)((p / 4) & (B == 3 ? ~7ll : ~1ll)),
+                 stride = gridDim.x * blockDim.x;
   const uint32_t lane = threadIdx.x & 31;
   uint32_t v = blockIdx.x * blockDim.x + threadIdx.x;
   double adq[4] = {0.0, 0.0, 0.0, 0.0}, aeps[4] = {0.0, 0.0, 0.0, 0.0};
@@ -351,7 +376,7 @@ __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned 
       const uint32_t y1 = quantize_one<FAST>(g[j].y, q[j].y, R, s, y, adq[1], aeps[1]);
       const uint32_t y2 = quantize_one<FAST>(g[j].z, q[j].z, R, s, y, adq[2], aeps[2]);
       const uint32_t y3 = quantize_one<FAST>(g[j].w, q[j].w, R, s, y, adq[3], aeps[3]);
-      store_codes<B>(row, v + j * stride, y0, y1, y2, y3, true);
+      store_codes<B>(row, v + j * stride, y0, y1, y2, y3, true, P.cw);
     }
   }
   sdq += (adq[0] + adq[1]) + (adq[2] + adq[3]);
@@ -374,7 +399,7 @@ __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned 
       sdq += a;
       seps += c;
     }
-    store_codes<B>(row, v, y0, y1, y2, y3, ok);
+    store_codes<B>(row, v, y0, y1, y2, y3, ok, P.cw);
   }
   if (blockIdx.x == 0 && threadIdx.x < 32) {  // groups that may contain padding coordinates
     const uint32_t v = nv_main + threadIdx.x;
@@ -388,7 +413,7 @@ __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned 
       for (int e = 0; e < 4; ++e)
         if (4ll * v + e < p) yy[e] = quantize_one<FAST>(gg[e], qq[e], R, s, y, sdq, seps);
     }
-    store_codes<B>(row, v, yy[0], yy[1], yy[2], yy[3], ok);
+    store_codes<B>(row, v, yy[0], yy[1], yy[2], yy[3], ok, P.cw);
   }
 }
 
@@ -596,7 +621,8 @@ __device__ __forceinline__ void aggregate_finish(const Params& P, double dsum, d
 
 template <int B>
 __device__ __forceinline__ const void* code_address(const uint32_t* row, uint32_t v) {
-  return reinterpret_cast<const uint8_t*>(row) + ((B == 1) ? (size_t)(v >> 1) : (size_t)v * (size_t)(B / 2));
+  return reinterpret_cast<const uint8_t*>(row) +
+         ((B == 1) ? (size_t)(v >> 1) : (B == 3) ? ((size_t)v * 3 / 2) & ~(size_t)3 : (size_t)v * (size_t)(B / 2));
 }
 
 // A thread owns groups v, v + stride, ...  Per group it holds only the aggregate in registers and walks the
@@ -809,7 +835,7 @@ __global__ void __launch_bounds__(kSmallThreads) small_iteration_kernel(const Pa
               yy[e] = fast ? quantize_one<true>(gg[e], qq[e], R, s, y, sdq, seps)
                            : quantize_one<false>(gg[e], qq[e], R, s, y, sdq, seps);
         }
-        store_codes<B>(row, v, yy[0], yy[1], yy[2], yy[3], ok);
+        store_codes<B>(row, v, yy[0], yy[1], yy[2], yy[3], ok, P.cw);
       }
     } else {
       for (long long wd = lane; wd < P.cw; wd += 32) row[wd] = 0u;
@@ -954,6 +980,7 @@ void launch_quant_b(const Params& P, dim3 grid, int threads, cudaStream_t st) {
   switch (P.b) {
     case 1: quantize_kernel<SYNTH, 1><<<grid, threads, 0, st>>>(P); break;
     case 2: quantize_kernel<SYNTH, 2><<<grid, threads, 0, st>>>(P); break;
+    case 3: quantize_kernel<SYNTH, 3><<<grid, threads, 0, st>>>(P); break;
     case 4: quantize_kernel<SYNTH, 4><<<grid, threads, 0, st>>>(P); break;
     case 8: quantize_kernel<SYNTH, 8><<<grid, threads, 0, st>>>(P); break;
     default: quantize_kernel<SYNTH, 16><<<grid, threads, 0, st>>>(P); break;
@@ -988,6 +1015,7 @@ int launch_small_iteration(const Params& P, int gbpw_finalize, cudaStream_t st) 
   switch (P.b) {
     case 1: small_iteration_kernel<1><<<1, kSmallThreads, 0, st>>>(P, gbpw_finalize); break;
     case 2: small_iteration_kernel<2><<<1, kSmallThreads, 0, st>>>(P, gbpw_finalize); break;
+    case 3: small_iteration_kernel<3><<<1, kSmallThreads, 0, st>>>(P, gbpw_finalize); break;
     case 4: small_iteration_kernel<4><<<1, kSmallThreads, 0, st>>>(P, gbpw_finalize); break;
     case 8: small_iteration_kernel<8><<<1, kSmallThreads, 0, st>>>(P, gbpw_finalize); break;
     default: small_iteration_kernel<16><<<1, kSmallThreads, 0, st>>>(P, gbpw_finalize); break;
@@ -1034,6 +1062,7 @@ int launch_aggregate(const Params& P, const LaunchShape& ls, cudaStream_t st) {
   switch (P.b) {
     case 1: aggregate_kernel<1><<<nb, ls.agg_threads, 0, st>>>(P); break;
     case 2: aggregate_kernel<2><<<nb, ls.agg_threads, 0, st>>>(P); break;
+    case 3: aggregate_kernel<3><<<nb, ls.agg_threads, 0, st>>>(P); break;
     case 4: aggregate_kernel<4><<<nb, ls.agg_threads, 0, st>>>(P); break;
     case 8: aggregate_kernel<8><<<nb, ls.agg_threads, 0, st>>>(P); break;
     default: aggregate_kernel<16><<<nb, ls.agg_threads, 0, st>>>(P); break;

@@ -36,7 +36,7 @@ def test_workspace_size_and_config_validation_need_no_gpu(lib):
     nbytes = laq.workspace_bytes(cfg)
     # Q_prev (M p fp32) + code streams (M p bytes) + theta and grad dominate
     assert 64 * 25_600_000 * 5 + 2 * 25_600_000 * 4 <= nbytes <= 64 * 25_600_000 * 5 + 2 * 25_600_000 * 4 + (8 << 20)
-    for bad in (dict(b=3), dict(M=0), dict(D=0), dict(alpha=-1.0), dict(clock_mode=2), dict(p=0)):
+    for bad in (dict(b=5), dict(M=0), dict(D=0), dict(alpha=-1.0), dict(clock_mode=2), dict(p=0)):
         kw = dict(model=laq.MODEL_SYNTH, M=4, p=100, b=4)
         kw.update(bad)
         cfg, keep = laq.make_config(**kw)

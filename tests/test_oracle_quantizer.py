@@ -115,7 +115,7 @@ def test_zero_innovation_gives_zero_message(dtype):
 
 
 @pytest.mark.parametrize("dtype", [np.float64, np.float32])
-@pytest.mark.parametrize("b", [1, 2, 4, 8, 16])
+@pytest.mark.parametrize("b", [1, 2, 3, 4, 8, 16])
 def test_server_recovery_from_message_is_bit_exact(dtype, b):
     """The server rebuilds Q_m(theta^k) from (R, q) and its stored copy (text after Eq. (6))."""
     rng = np.random.default_rng(b)
@@ -141,6 +141,12 @@ def test_pack_layout_little_endian_within_words():
     assert w2.tolist() == [1 | (2 << 2) | (3 << 4) | (0 << 6) | (1 << 8)]
     w8 = oracle.pack_codes(np.array([255, 1, 2, 3, 4], np.int32), 8)
     assert w8.tolist() == [0x030201FF, 0x00000004]
+    # b = 3 (the logistic-regression setting of Sec. 4): code 10 straddles words 0 and 1; written out as one
+    # big integer the stream is sum_i q_i 8^i
+    q3 = np.array([5, 7, 1, 0, 3, 6, 2, 4, 7, 7, 1, 5], np.int32)
+    big = sum(int(c) << (3 * i) for i, c in enumerate(q3))
+    assert oracle.pack_codes(q3, 3).tolist() == [big & 0xFFFFFFFF, big >> 32]
+    np.testing.assert_array_equal(oracle.unpack_codes(oracle.pack_codes(q3, 3), 12, 3), q3)
 
 
 def test_message_cost_formula_reproduces_the_papers_tables():
