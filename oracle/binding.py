@@ -83,6 +83,9 @@ def lib():
                            C.c_uint32, C.c_uint64, C.c_float, C.c_float, C.c_int, _c_f32p]
     L.laqo_new.restype = C.c_void_p
     L.laqo_free.argtypes = [C.c_void_p]
+    L.laqo_set_batch.argtypes = [C.c_void_p, C.c_int]
+    L.laqo_batch_offset.argtypes = [C.c_uint64, C.c_int, C.c_int64, C.c_int64]
+    L.laqo_batch_offset.restype = C.c_int64
     L.laqo_set_shard.argtypes = [C.c_void_p, C.c_int, _c_f32p, _c_i32p, C.c_int64, C.c_int]
     L.laqo_set_shard.restype = C.c_int
     L.laqo_step.argtypes = [C.c_void_p]
@@ -155,6 +158,11 @@ def unpack_codes(words, p, b):
     return q
 
 
+def batch_offset(seed, m, k, n):
+    """First sample of worker m's minibatch window at iteration k = 1, 2, .. (shard of n samples)."""
+    return int(lib().laqo_batch_offset(int(seed), int(m), int(k), int(n)))
+
+
 def trigger(n_dq, n_eps, n_epshat, dtheta2, xi, alpha, M, clock, tbar, clock_mode=0):
     """Eq. (7a)+(7b) for one worker; dtheta2[0] is the newest difference.  Returns (skip, rhs)."""
     L = lib()
@@ -222,7 +230,7 @@ class OracleLaq:
 
     def __init__(self, precision, model, M, p, N=None, n_features=0, n_classes=0, n_hidden=0,
                  alpha=0.02, lam=0.0, b=4, D=10, xi=None, tbar=100, clock_mode=0, flags=0, seed=0,
-                 synth_sigma=0.1, synth_eta0=0.05, bf16_ops=0, theta0=None):
+                 synth_sigma=0.1, synth_eta0=0.05, bf16_ops=0, theta0=None, batch=0):
         L = lib()
         self.L, self.precision, self.M, self.p, self.D, self.b = L, precision, M, int(p), D, b
         self.dtype = np.float64 if precision == 64 else np.float32
@@ -234,6 +242,9 @@ class OracleLaq:
                             seed, synth_sigma, synth_eta0, bf16_ops, _ptr(th0, _c_f32p))
         if not self.h:
             raise ValueError("oracle rejected the configuration")
+
+        if batch:
+            L.laqo_set_batch(self.h, int(batch))
 
     def __del__(self):
         if getattr(self, "h", None):

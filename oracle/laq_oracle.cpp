@@ -363,6 +363,14 @@ void synth_gradient(uint64_t seed, int m, int M, i64 p, i64 k, float sigma, floa
 // ---------------------------------------------------------------------------------------------
 // The LAQ loop (Algorithm 2), state and one iteration.
 // ---------------------------------------------------------------------------------------------
+// Start of worker m's minibatch window at iteration k = 1, 2, ..: a counter-based draw from (seed, m, k)
+// with the 32-bit finalizer fmix32, reduced modulo the shard size n.
+i64 batch_offset(uint64_t seed, int m, i64 k, i64 n) {
+  const uint32_t lo = (uint32_t)seed, hi = (uint32_t)(seed >> 32);
+  const uint32_t h = fmix32(fmix32(lo + (uint32_t)k) ^ (hi + 0x9e3779b9u * (uint32_t)(m + 1)));
+  return (i64)(h % (uint32_t)n);
+}
+
 struct Config {
   int model, M;
   i64 p;
@@ -375,6 +383,7 @@ struct Config {
   uint64_t seed;
   float synth_sigma, synth_eta0;
   int bf16_ops;
+  int batch = 0;  // 0: full local gradients; > 0: minibatch size per worker (the stochastic variant of Sec. 4)
 };
 
 struct IterStats {  // what one iteration reports, per worker unless noted
@@ -440,18 +449,43 @@ struct Laq {
     std::vector<double> th(c.p), gd(c.p);
     for (i64 i = 0; i < c.p; ++i) th[i] = (double)theta[i];
     const double inv_N = 1.0 / (double)Ntot;
+    std::vector<float> Xb;
+    std::vector<int32_t> yb;
     for (int m = 0; m < c.M; ++m) {
       const double share = (double)N[m] / (double)Ntot;
+      // The stochastic variant (Sec. 4, minibatch tests): the sum over the worker's samples is replaced by
+      // N_m / B_m times the sum over a minibatch of B_m samples, here a cyclic window of consecutive samples
+      // with a pseudo-random start; the regulariser's share is unchanged.
+      const float* Xm = X[m].data();
+      const int32_t* ym = y[m].data();
+      i64 n_used = N[m];
+      double inv_Nm = inv_N;
+      if (c.batch > 0) {
+        const i64 B = std::min<i64>(c.batch, N[m]);
+        const i64 o = batch_offset(c.seed, m, k + 1, N[m]);
+        const size_t F = (size_t)c.n_features;
+        Xb.resize((size_t)B * F);
+        yb.resize((size_t)B);
+        for (i64 j = 0; j < B; ++j) {
+          const i64 r = (o + j) % N[m];
+          std::memcpy(&Xb[(size_t)j * F], Xm + (size_t)r * F, sizeof(float) * F);
+          yb[(size_t)j] = ym[r];
+        }
+        Xm = Xb.data();
+        ym = yb.data();
+        n_used = B;
+        inv_Nm = inv_N * ((double)N[m] / (double)B);
+      }
       double loss = 0.0;
       if (c.model == M_LOGREG_BIN)
-        loss = grad_logreg_bin(X[m].data(), y[m].data(), N[m], c.n_features, th.data(), inv_N,
-                               share, (double)c.lambda, gd.data());
+        loss = grad_logreg_bin(Xm, ym, n_used, c.n_features, th.data(), inv_Nm, share, (double)c.lambda,
+                               gd.data());
       else if (c.model == M_SOFTMAX)
-        loss = grad_softmax(X[m].data(), y[m].data(), N[m], c.n_features, c.n_classes, th.data(),
-                            inv_N, share, (double)c.lambda, gd.data());
+        loss = grad_softmax(Xm, ym, n_used, c.n_features, c.n_classes, th.data(), inv_Nm, share,
+                            (double)c.lambda, gd.data());
       else
-        loss = grad_mlp2(X[m].data(), y[m].data(), N[m], c.n_features, c.n_hidden, c.n_classes,
-                         th.data(), inv_N, share, (double)c.lambda, c.bf16_ops, gd.data());
+        loss = grad_mlp2(Xm, ym, n_used, c.n_features, c.n_hidden, c.n_classes, th.data(), inv_Nm, share,
+                         (double)c.lambda, c.bf16_ops, gd.data());
       st.loss_m[m] = loss;
       for (i64 i = 0; i < c.p; ++i) g[(size_t)m * c.p + i] = (T)gd[i];
     }
@@ -638,6 +672,14 @@ void* laqo_new(int precision, int model, int M, int64_t p, const int64_t* N, int
   return h;
 }
 void laqo_free(void* hv) { delete (Handle*)hv; }
+void laqo_set_batch(void* hv, int batch) {
+  Handle* h = (Handle*)hv;
+  if (h->prec == 32)
+    h->f.c.batch = batch;
+  else
+    h->d.c.batch = batch;
+}
+int64_t laqo_batch_offset(uint64_t seed, int m, int64_t k, int64_t n) { return batch_offset(seed, m, k, n); }
 
 int laqo_set_shard(void* hv, int m, const float* X, const int32_t* y, int64_t n, int row_len) {
   Handle* h = (Handle*)hv;

@@ -257,3 +257,79 @@ def test_linear_convergence_on_a_tiny_strongly_convex_problem(precision):
     else:
         assert res[-1] < 1e-9 * max(res[0], 1.0)
         assert err[-1] < 1e-3 * err[0]
+
+
+# ------------------------------------------------------------------------------------------------
+# the stochastic variant (minibatch tests of Sec. 4)
+# ------------------------------------------------------------------------------------------------
+def _tiny_logreg(rng, M, n_per, F):
+    X = [rng.standard_normal((n_per[m], F)).astype(np.float32) for m in range(M)]
+    y = [(rng.random(n_per[m]) < 0.5).astype(np.int32) for m in range(M)]
+    return X, y
+
+
+def test_minibatch_window_start_is_in_range_and_spread_out():
+    n = 37
+    starts = np.array([[oracle.batch_offset(12345, m, k, n) for k in range(1, 2001)] for m in range(3)])
+    assert starts.min() >= 0 and starts.max() < n
+    for m in range(3):                                   # every start occurs, about equally often
+        counts = np.bincount(starts[m], minlength=n)
+        assert counts.min() > 0.5 * 2000 / n and counts.max() < 1.6 * 2000 / n
+    assert not np.array_equal(starts[0], starts[1])      # workers draw different windows
+    assert oracle.batch_offset(1, 0, 5, n) != oracle.batch_offset(2, 0, 5, n) or \
+        oracle.batch_offset(1, 0, 6, n) != oracle.batch_offset(2, 0, 6, n)   # the seed matters
+    assert oracle.batch_offset(9, 4, 7, 1) == 0
+
+
+def test_minibatch_gradient_is_the_scaled_window_sum_and_unbiased():
+    """g_m = (N_m / B)(1/N) sum over the window + the worker's share of the regulariser: checked against the
+    full-shard routine applied to the window's rows, and averaged over all N_m window positions (each sample
+    lies in exactly B windows) it equals the full gradient."""
+    rng = np.random.default_rng(11)
+    M, F, B, lam, alpha = 3, 5, 4, 0.125, 0.0625
+    n_per = [9, 6, 11]
+    N = sum(n_per)
+    X, y = _tiny_logreg(rng, M, n_per, F)
+    theta0 = rng.standard_normal(F).astype(np.float32)
+    o = oracle.OracleLaq(64, oracle.MODEL_LOGREG_BIN, M, F, N=n_per, n_features=F, alpha=alpha, lam=lam, b=8, D=2,
+                         tbar=5, seed=77, theta0=theta0, batch=B, flags=oracle.FLAG_TRIGGER_OFF | oracle.FLAG_QUANT_OFF)
+    for m in range(M):
+        o.set_shard(m, X[m], y[m])
+    theta = theta0.astype(np.float64)
+    for k in range(1, 6):
+        expect = np.zeros(F)
+        for m in range(M):
+            st = oracle.batch_offset(77, m, k, n_per[m])
+            rows = [(st + j) % n_per[m] for j in range(B)]
+            _, g = oracle.grad_logreg_bin(X[m][rows], y[m][rows], theta, (n_per[m] / B) / N, n_per[m] / N, lam)
+            expect += g
+        o.step()                                          # GD mode: theta -= alpha sum_m g_m
+        theta = theta - alpha * expect
+        np.testing.assert_allclose(o.state(big=False)["theta"], theta, rtol=1e-10, atol=1e-12)
+    # unbiasedness by brute force over every window position of worker 0
+    th = rng.standard_normal(F)
+    n0 = n_per[0]
+    _, full = oracle.grad_logreg_bin(X[0], y[0], th, 1.0 / N, n0 / N, lam)
+    mean = np.zeros(F)
+    for st in range(n0):
+        rows = [(st + j) % n0 for j in range(B)]
+        _, g = oracle.grad_logreg_bin(X[0][rows], y[0][rows], th, (n0 / B) / N, n0 / N, lam)
+        mean += g / n0
+    np.testing.assert_allclose(mean, full, rtol=1e-12, atol=1e-14)
+
+
+def test_minibatch_as_large_as_the_shard_is_the_full_gradient():
+    rng = np.random.default_rng(12)
+    M, F = 2, 4
+    n_per = [7, 5]
+    X, y = _tiny_logreg(rng, M, n_per, F)
+    kw = dict(N=n_per, n_features=F, alpha=0.125, lam=0.01, b=4, D=2, tbar=5, seed=3)
+    a = oracle.OracleLaq(64, oracle.MODEL_LOGREG_BIN, M, F, batch=0, **kw)
+    b = oracle.OracleLaq(64, oracle.MODEL_LOGREG_BIN, M, F, batch=100, **kw)    # B_m = min(batch, N_m)
+    for m in range(M):
+        a.set_shard(m, X[m], y[m])
+        b.set_shard(m, X[m], y[m])
+    for k in range(10):
+        sa, sb = a.step(), b.step()
+        np.testing.assert_array_equal(sa["skip"], sb["skip"])
+        np.testing.assert_allclose(b.state(big=False)["theta"], a.state(big=False)["theta"], rtol=1e-11, atol=1e-13)
