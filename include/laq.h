@@ -99,10 +99,16 @@ typedef struct {
   int32_t clock_mode;       /* 0: Algorithm 2 as printed, skip allowed while t_m <= t_bar;
                                1: strict, skip needs t_m + 2 <= t_bar (t_bar = 1 never skips) */
   uint32_t flags;           /* LAQ_FLAG_* */
-  uint64_t seed;            /* SYNTH only */
+  uint64_t seed;            /* SYNTH stream and minibatch windows */
   float synth_sigma;        /* SYNTH only */
   float synth_eta0;         /* SYNTH only */
   int32_t trace_capacity;   /* per-iteration records kept on the device for laq_step's trace (0 = none) */
+  int32_t batch;            /* 0: full local gradients.  > 0 (LOGREG_BIN, SOFTMAX): the minibatch variant of the
+                               Sec. 4 stochastic tests.  At iteration k = 1, 2, .. worker m uses the B_m =
+                               min(batch, N_m) samples (o + j) mod N_m, j < B_m, a cyclic window starting at
+                               o = fmix32(fmix32(seed_lo + (uint32) k) ^ (seed_hi + 0x9e3779b9 (m+1))) mod N_m, and
+                               g_m = (N_m / B_m)(1/N) sum_window grad l_i + (N_m/N) lambda theta; the reported loss
+                               is the same estimate of f */
 } laq_config;
 
 /* Per-iteration report of laq_step.  All pointers HOST, each may be NULL; n = n_iters of that call.

@@ -70,6 +70,9 @@ const char* check_config(const laq_config* c) {
   if (c->clock_mode != 0 && c->clock_mode != 1) return "clock_mode must be 0 or 1";
   if (c->trace_capacity < 0) return "trace_capacity must be >= 0";
   if (c->flags & ~(uint32_t)(LAQ_FLAG_TRIGGER_OFF | LAQ_FLAG_QUANT_OFF)) return "unknown flag";
+  if (c->batch < 0) return "batch must be >= 0";
+  if (c->batch > 0 && c->model != LAQ_MODEL_LOGREG_BIN && c->model != LAQ_MODEL_SOFTMAX)
+    return "batch > 0 needs LAQ_MODEL_LOGREG_BIN or LAQ_MODEL_SOFTMAX";
   const bool data = c->model == LAQ_MODEL_LOGREG_BIN || c->model == LAQ_MODEL_SOFTMAX || c->model == LAQ_MODEL_MLP2;
   if (data) {
     if (!c->N) return "N is null";
@@ -294,6 +297,7 @@ laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, siz
   P.t_up = (int32_t*)(ws + pl.t_up);
   P.seed_lo = (uint32_t)(c.seed & 0xffffffffull);
   P.seed_hi = (uint32_t)(c.seed >> 32);
+  P.batch = c.batch;
   P.cz = (float)((double)c.synth_sigma / std::sqrt(21845.0));
   P.eta0 = c.synth_eta0;
   P.X = (const float* const*)(ws + pl.Xptr);

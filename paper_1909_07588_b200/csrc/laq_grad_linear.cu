@@ -65,17 +65,18 @@ __global__ void __launch_bounds__(kLrThreads) grad_logreg_kernel(const Params P,
   __shared__ double shd[32];
   const float* __restrict__ X = P.X[m];
   const int32_t* __restrict__ y = P.y[m];
-  const long long n = P.N[m];
   for (int f = t; f < F; f += blockDim.x) ths[f] = P.theta[f];
   const int S = kLrThreads / F;              // row slices handled in parallel in the second phase
   const bool active = t < S * F;
   const int f_own = t % F, slice = t / F;
   float acc = 0.f;
   double loss = 0.0;
-  const long long ntiles = (n + rows - 1) / rows;
+  const RowWindow win = row_window(P, m);
+  const long long ntiles = win.tiles(rows);
   for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-    const long long r0 = tile * rows;
-    const int nr = (int)((n - r0 < rows) ? (n - r0) : rows);
+    long long r0;
+    int nr;
+    win.tile(tile, rows, r0, nr);
     __syncthreads();
     stage_rows(X + r0 * F, xs, nr * F);
     __syncthreads();
@@ -136,17 +137,18 @@ __global__ void __launch_bounds__(kSmThreads) grad_softmax_kernel(const Params P
   const float* __restrict__ X = P.X[m];
   const int32_t* __restrict__ y = P.y[m];
   const float* __restrict__ theta = P.theta;
-  const long long n = P.N[m];
   float acc[kSmMaxJ][C];
 #pragma unroll
   for (int j = 0; j < kSmMaxJ; ++j)
 #pragma unroll
     for (int c = 0; c < C; ++c) acc[j][c] = 0.f;
   double loss = 0.0;
-  const long long ntiles = (n + kSmRows - 1) / kSmRows;
+  const RowWindow win = row_window(P, m);
+  const long long ntiles = win.tiles(kSmRows);
   for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-    const long long r0 = tile * kSmRows;
-    const int nr = (int)((n - r0 < kSmRows) ? (n - r0) : kSmRows);
+    long long r0;
+    int nr;
+    win.tile(tile, kSmRows, r0, nr);
     __syncthreads();
     stage_rows(X + r0 * F, xs, nr * F);
     __syncthreads();
@@ -250,7 +252,6 @@ __global__ void __launch_bounds__(kS2Threads, 2) grad_softmax_tile_kernel(const 
   static_assert(kS2Rows * C <= kS2Threads, "one thread per (row, class)");
   const float* __restrict__ X = P.X[m];
   const int32_t* __restrict__ y = P.y[m];
-  const long long n = P.N[m];
   for (int i = t; i < C * F4; i += kS2Threads)
     reinterpret_cast<float4*>(ths)[i] = __ldg(reinterpret_cast<const float4*>(P.theta) + i);
   const int kw = (F4 + kS2Warps - 1) / kS2Warps;     // 16-byte groups of features per warp in phase 1
@@ -261,12 +262,14 @@ __global__ void __launch_bounds__(kS2Threads, 2) grad_softmax_tile_kernel(const 
 #pragma unroll
   for (int c = 0; c < C; ++c) acc01[c] = acc23[c] = 0ull;
   double loss = 0.0;
-  const long long ntiles = (n + kS2Rows - 1) / kS2Rows;
+  const RowWindow win = row_window(P, m);
+  const long long ntiles = win.tiles(kS2Rows);
 
   // asynchronous staging of one tile: contiguous rows in global memory -> padded rows in shared memory
   auto stage = [&](long long tile, float* xs) {
-    const long long r0 = tile * kS2Rows;
-    const int nr = (int)((n - r0 < kS2Rows) ? (n - r0) : kS2Rows);
+    long long r0;
+    int nr;
+    win.tile(tile, kS2Rows, r0, nr);
     const float4* src = reinterpret_cast<const float4*>(X + r0 * F);
     const int cnt = nr * F4;
     int r = t / F4, k = t - r * F4;
@@ -288,8 +291,9 @@ __global__ void __launch_bounds__(kS2Threads, 2) grad_softmax_tile_kernel(const 
   if ((long long)blockIdx.x < ntiles) stage(blockIdx.x, xs0);
   __pipeline_commit();
   for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x, buf ^= 1) {
-    const long long r0 = tile * kS2Rows;
-    const int nr = (int)((n - r0 < kS2Rows) ? (n - r0) : kS2Rows);
+    long long r0;
+    int nr;
+    win.tile(tile, kS2Rows, r0, nr);
     float* xs = xs0 + buf * kS2Rows * FP;
     __syncthreads();                                  // everybody is done with the buffer refilled below
     if (tile + gridDim.x < ntiles) stage(tile + gridDim.x, xs0 + (buf ^ 1) * kS2Rows * FP);
@@ -408,13 +412,13 @@ __global__ void __launch_bounds__(256) grad_finalize_kernel(const Params P, int 
     const float* gp = P.gpart + (long long)m * gbpw * P.ps + i;
     double s = 0.0;
     for (int blk = 0; blk < gbpw; ++blk) s += (double)gp[(long long)blk * P.ps];
-    const double g = s * inv_N + share * (double)P.lambda * (double)P.theta[i];
+    const double g = s * (inv_N * batch_scale(P, m)) + share * (double)P.lambda * (double)P.theta[i];
     P.g[(long long)m * P.ps + i] = (float)g;
   }
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     double l = 0.0;
     for (int blk = 0; blk < gbpw; ++blk) l += P.lpart[(long long)m * gbpw + blk];
-    P.loss_m[m] = l * inv_N + share * 0.5 * (double)P.lambda * (*theta_sq);
+    P.loss_m[m] = l * (inv_N * batch_scale(P, m)) + share * 0.5 * (double)P.lambda * (*theta_sq);
   }
 }
 

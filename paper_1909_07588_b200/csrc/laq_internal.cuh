@@ -66,6 +66,7 @@ struct Params {
   int32_t* t_up;
   // synthetic gradient stream
   uint32_t seed_lo, seed_hi;
+  int batch;                 // 0: full local gradients; > 0: minibatch size per worker
   float cz, eta0;
   // shards
   long long Ntot;
@@ -77,6 +78,69 @@ struct Params {
   double* lpart;             // loss partials [M][gbpw]
   uint32_t* cnt_grad;        // [M] tickets
 };
+
+#ifdef __CUDACC__
+// 32-bit finalizer of MurmurHash3 (public domain)
+__device__ __forceinline__ uint32_t fmix32(uint32_t x) {
+  x ^= x >> 16;
+  x *= 0x85ebca6bu;
+  x ^= x >> 13;
+  x *= 0xc2b2ae35u;
+  x ^= x >> 16;
+  return x;
+}
+
+// Rows of worker m that enter the local gradient of the iteration in progress: all N_m rows, or (minibatch
+// variant of Sec. 4) the cyclic window of B_m = min(batch, N_m) consecutive rows whose start is drawn from
+// (seed, m, k): rows [start, start + len_a) followed by rows [0, len_b).
+struct RowWindow {
+  long long start, len_a, len_b;
+  __device__ __forceinline__ long long tiles(int rows) const {
+    return (len_a + rows - 1) / rows + (len_b + rows - 1) / rows;
+  }
+  // tile t of `rows` rows -> first row and number of rows (tiles never straddle the wrap)
+  __device__ __forceinline__ void tile(long long t, int rows, long long& r0, int& nr) const {
+    const long long ta = (len_a + rows - 1) / rows;
+    long long left;
+    if (t < ta) {
+      r0 = start + t * rows;
+      left = len_a - t * rows;
+    } else {
+      t -= ta;
+      r0 = t * rows;
+      left = len_b - t * rows;
+    }
+    nr = (int)(left < rows ? left : rows);
+  }
+  __device__ __forceinline__ bool contains(long long r) const {
+    return (r >= start && r < start + len_a) || r < len_b;
+  }
+};
+
+__device__ __forceinline__ RowWindow row_window(const Params& P, int m) {
+  const long long n = P.N[m];
+  RowWindow w;
+  if (P.batch <= 0 || P.batch >= n) {
+    w.start = 0;
+    w.len_a = n;
+    w.len_b = 0;
+    return w;
+  }
+  const uint32_t k = (uint32_t)(P.sc->k + 1ull);
+  const uint32_t h = fmix32(fmix32(P.seed_lo + k) ^ (P.seed_hi + 0x9e3779b9u * (uint32_t)(m + 1)));
+  w.start = (long long)(h % (uint32_t)n);
+  const long long to_end = n - w.start;
+  w.len_a = P.batch < to_end ? P.batch : to_end;
+  w.len_b = P.batch - w.len_a;
+  return w;
+}
+
+// N_m / B_m: what the sum over the window is scaled by so that it estimates the sum over the shard
+__device__ __forceinline__ double batch_scale(const Params& P, int m) {
+  const long long n = P.N[m];
+  return (P.batch <= 0 || P.batch >= n) ? 1.0 : (double)n / (double)P.batch;
+}
+#endif
 
 struct LaunchShape {
   int sweep_threads = 128;

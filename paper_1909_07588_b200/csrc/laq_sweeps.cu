@@ -17,15 +17,6 @@ namespace laq {
 
 namespace {
 
-__device__ __forceinline__ uint32_t fmix32(uint32_t x) {
-  x ^= x >> 16;
-  x *= 0x85ebca6bu;
-  x ^= x >> 13;
-  x *= 0xc2b2ae35u;
-  x ^= x >> 16;
-  return x;
-}
-
 // Synthetic gradient stream (definition in laq.h).  One strong hash per group of four coordinates,
 // a cheap second word from it, and two near-Gaussian byte sums per word.
 struct Synth {
@@ -774,13 +765,14 @@ __global__ void __launch_bounds__(kSmallThreads) small_iteration_kernel(const Pa
       double s = 0.0;
       for (int blk = 0; blk < gbpw; ++blk) s += (double)gp[(long long)blk * P.ps];
       const double share = (double)P.N[m] / (double)P.Ntot;
-      P.g[(long long)m * P.ps + i] = (float)(s * inv_N + share * (double)P.lambda * (double)P.theta[i]);
+      P.g[(long long)m * P.ps + i] =
+          (float)(s * (inv_N * batch_scale(P, m)) + share * (double)P.lambda * (double)P.theta[i]);
     }
     for (int m = t; m < M; m += kSmallThreads) {
       double l = 0.0;
       for (int blk = 0; blk < gbpw; ++blk) l += P.lpart[(long long)m * gbpw + blk];
       const double share = (double)P.N[m] / (double)P.Ntot;
-      P.loss_m[m] = l * inv_N + share * 0.5 * (double)P.lambda * sc->theta_sq;
+      P.loss_m[m] = l * (inv_N * batch_scale(P, m)) + share * 0.5 * (double)P.lambda * sc->theta_sq;
     }
   }
   __syncthreads();

@@ -33,7 +33,7 @@ class laq_config(C.Structure):
                 ("alpha", C.c_float), ("lam", C.c_float), ("b", C.c_int32), ("D", C.c_int32),
                 ("xi", C.POINTER(C.c_float)), ("tbar", C.c_int32), ("clock_mode", C.c_int32),
                 ("flags", C.c_uint32), ("seed", C.c_uint64), ("synth_sigma", C.c_float),
-                ("synth_eta0", C.c_float), ("trace_capacity", C.c_int32)]
+                ("synth_eta0", C.c_float), ("trace_capacity", C.c_int32), ("batch", C.c_int32)]
 
 
 class laq_trace(C.Structure):
@@ -87,13 +87,13 @@ def load_library():
 
 def make_config(model, M, p, N=None, n_features=0, n_classes=0, n_hidden=0, alpha=0.02, lam=0.0, b=4, D=10,
                 xi=None, tbar=100, clock_mode=0, flags=0, seed=0, synth_sigma=0.1, synth_eta0=0.05,
-                trace_capacity=0):
+                trace_capacity=0, batch=0):
     """Returns (laq_config, keepalive) -- keepalive holds the numpy arrays the struct points to."""
     N_arr = np.ascontiguousarray(N if N is not None else np.zeros(max(M, 1)), dtype=np.int64)
     xi_arr = np.ascontiguousarray(xi if xi is not None else np.full(max(D, 1), 0.8 / max(D, 1)), dtype=np.float32)
     cfg = laq_config(model, M, p, N_arr.ctypes.data_as(C.POINTER(C.c_int64)), n_features, n_classes, n_hidden,
                      alpha, lam, b, D, xi_arr.ctypes.data_as(C.POINTER(C.c_float)), tbar, clock_mode, flags,
-                     seed, synth_sigma, synth_eta0, trace_capacity)
+                     seed, synth_sigma, synth_eta0, trace_capacity, batch)
     return cfg, (N_arr, xi_arr)
 
 

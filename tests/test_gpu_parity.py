@@ -260,24 +260,29 @@ def test_synthetic_full_size_sampled_workers():
 # ------------------------------------------------------------------------------------------------
 # model workloads: gradients from the library's own kernels
 # ------------------------------------------------------------------------------------------------
-def _oracle_gradients(w, theta):
-    """fp64 model gradients of every worker at the given (fp32) theta, from the oracle's stateless functions."""
+def _oracle_gradients(w, theta, batch=0, k=1):
+    """fp64 model gradients of every worker at the given (fp32) theta, from the oracle's stateless functions;
+    with batch > 0 over the minibatch window of iteration k (rows from the oracle's own draw of the start)."""
     N = float(sum(w.N))
     th = np.asarray(theta, np.float64)
     out = []
     for m in range(w.M):
         share = w.N[m] / N
+        X, y, inv = w.X[m], w.y[m], 1.0 / N
+        if batch and batch < w.N[m]:
+            rows = (oracle.batch_offset(w.seed, m, k, w.N[m]) + np.arange(batch)) % w.N[m]
+            X, y, inv = X[rows], y[rows], (w.N[m] / batch) / N
         if w.model == workloads.MODEL_LOGREG_BIN:
-            _, g = oracle.grad_logreg_bin(w.X[m], w.y[m], th, 1.0 / N, share, w.lam)
+            _, g = oracle.grad_logreg_bin(X, y, th, inv, share, w.lam)
         elif w.model == workloads.MODEL_SOFTMAX:
-            _, g = oracle.grad_softmax(w.X[m], w.y[m], th, w.n_classes, 1.0 / N, share, w.lam)
+            _, g = oracle.grad_softmax(X, y, th, w.n_classes, inv, share, w.lam)
         else:
-            _, g = oracle.grad_mlp2(w.X[m], w.y[m], th, w.n_hidden, w.n_classes, 1.0 / N, share, w.lam, w.bf16_ops)
+            _, g = oracle.grad_mlp2(X, y, th, w.n_hidden, w.n_classes, inv, share, w.lam, w.bf16_ops)
         out.append(g)
     return np.array(out)
 
 
-def _run_model_parity(w, iters):
+def _run_model_parity(w, iters, batch=0):
     """Three comparisons per iteration of a model workload:
       (1) step 1 on identical input: the library's gradients at its own theta^k against the fp64 model gradient;
       (2) steps 2-5 on identical input: the fp32 mirror fed with the library's gradients, bit-exact;
@@ -287,9 +292,10 @@ def _run_model_parity(w, iters):
     Besides, a free-running fp64 oracle follows the same problem from the start; the first iteration at which its
     skip mask differs or theta leaves the TRAJ_RTOL band is reported and returned (None if never): a single
     near-tie code flip moves one coordinate of theta by alpha 2 tau R, which both trajectories then absorb."""
-    ctx = laq.from_workload(w, trace_capacity=1)
-    free64 = _mirror_for(w, 64)
-    step64 = _mirror_for(w, 64)
+    ctx = laq.from_workload(w, trace_capacity=1, batch=batch)
+    free64 = _mirror_for(w, 64, batch=batch)
+    # step64 is stepped once per iteration, so its k (which the window start depends on) stays the library's
+    step64 = _mirror_for(w, 64, batch=batch)
     mir = oracle.OracleLaq(32, oracle.MODEL_GIVEN, w.M, w.p, alpha=w.alpha, b=w.b, D=w.D, xi=w.xi, tbar=w.tbar,
                            theta0=w.theta0)
     first_diff, code_flips, skip_flips, n_resolved = None, 0, 0, 0
@@ -298,7 +304,7 @@ def _run_model_parity(w, iters):
         tr = ctx.step(1, trace=True)
         gs = ctx.get_state(g=True, codes=True)
         # (1)
-        g_ref = _oracle_gradients(w, prev["theta"])
+        g_ref = _oracle_gradients(w, prev["theta"], batch, k + 1)
         # the network rounds dH to bf16: an fp32 dH next to a bf16 rounding boundary may round the other way
         # than the oracle's fp64 dH, which moves single terms of the W1 gradient by 2^-9 relative
         grad_rtol = 2e-4 if w.model == workloads.MODEL_MLP2 else GRAD_RTOL
@@ -354,6 +360,35 @@ def test_c0_logreg_full():
     w = workloads.c0()
     first = _run_model_parity(w, w.iters)
     assert first is None or first > 3
+
+
+def test_minibatch_logreg_windows_wrap_and_ragged_tiles():
+    """The stochastic variant (Sec. 4): batch 500 of 3001 samples per worker, b = 3 as in the paper's logistic
+    runs; windows wrap around the end of the shard in some iterations."""
+    w = workloads.c2(n_per=3001, iters=60, theta0_scale=0.01)
+    w.b = 3
+    wraps = sum(oracle.batch_offset(w.seed, m, k, 3001) + 500 > 3001 for m in range(w.M) for k in range(1, 61))
+    assert wraps > 0
+    first = _run_model_parity(w, w.iters, batch=500)
+    assert first is None or first > 3
+
+
+def test_minibatch_softmax():
+    w = workloads.c1(n_per=1203, iters=40)
+    first = _run_model_parity(w, w.iters, batch=500)
+    assert first is None or first > 3
+
+
+def test_minibatch_small_shards_use_every_sample():
+    """batch >= N_m: the window is the whole shard, the run equals the full-gradient run bit for bit."""
+    w = workloads.c0()
+    a = laq.from_workload(w, trace_capacity=50)
+    b = laq.from_workload(w, trace_capacity=50, batch=10 ** 6)
+    ta, tb = a.step(50, trace=True), b.step(50, trace=True)
+    np.testing.assert_array_equal(ta["skip"], tb["skip"])
+    np.testing.assert_array_equal(a.get_state()["theta"], b.get_state()["theta"])
+    a.close()
+    b.close()
 
 
 def test_c2_shape_logreg54_reduced():
@@ -426,6 +461,9 @@ def test_api_misuse_returns_error_codes():
     with pytest.raises(laq.LaqError) as e:
         laq.Laq(model=laq.MODEL_SYNTH, M=4, p=100, b=5)
     assert e.value.status == laq.LAQ_EINVAL and "b must be" in str(e.value)
+    with pytest.raises(laq.LaqError) as e:
+        laq.Laq(model=laq.MODEL_SYNTH, M=4, p=100, b=4, batch=10)       # a minibatch needs samples
+    assert e.value.status == laq.LAQ_EINVAL
     w = workloads.c0()
     c = laq.Laq(model=w.model, M=w.M, p=w.p, N=w.N, n_features=w.n_features, alpha=w.alpha, lam=w.lam, b=w.b)
     with pytest.raises(laq.LaqError) as e:

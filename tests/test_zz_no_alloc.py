@@ -45,12 +45,19 @@ def test_static_scratch_quantizer_matches_regular_entry_point_twice_in_a_row():
                          codes=torch.full((W,), -1, dtype=torch.int32, device="cuda"),
                          R=torch.full((1,), -1.0, dtype=torch.float32, device="cuda"),
                          norms=torch.full((2,), -1.0, dtype=torch.float64, device="cuda")))
+    # Objects of earlier tests that the collector has not yet freed would make the counters move during the
+    # calls, so collect first.  Two checks: torch's allocator served no request, and the driver handed out no
+    # device memory (which would also catch an allocation made inside the library).
+    import gc
+    gc.collect()
     torch.cuda.synchronize()
-    before = torch.cuda.memory_allocated()
+    requests_before = torch.cuda.memory_stats()["allocation.all.allocated"]
+    free_before = torch.cuda.mem_get_info()[0]
     for c in bufs:                                                       # calls back to back, no sync between
         laq.quantize_worker_static(c["dg"], c["dq"], c["b"], c["codes"], c["R"], c["norms"])
     torch.cuda.synchronize()
-    assert torch.cuda.memory_allocated() == before
+    assert torch.cuda.memory_stats()["allocation.all.allocated"] == requests_before
+    assert torch.cuda.mem_get_info()[0] >= free_before
     for c in bufs:
         codes_ref, R_ref, ndq_ref, neps_ref = _regular_entry_point(c["g"], c["q"], c["b"])
         np.testing.assert_array_equal(c["codes"].cpu().numpy().view(np.uint32), codes_ref)
