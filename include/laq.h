@@ -103,7 +103,7 @@ typedef struct {
   float synth_sigma;        /* SYNTH only */
   float synth_eta0;         /* SYNTH only */
   int32_t trace_capacity;   /* per-iteration records kept on the device for laq_step's trace (0 = none) */
-  int32_t batch;            /* 0: full local gradients.  > 0 (LOGREG_BIN, SOFTMAX): the minibatch variant of the
+  int32_t batch;            /* 0: full local gradients.  > 0 (models with samples): the minibatch variant of the
                                Sec. 4 stochastic tests.  At iteration k = 1, 2, .. worker m uses the B_m =
                                min(batch, N_m) samples (o + j) mod N_m, j < B_m, a cyclic window starting at
                                o = fmix32(fmix32(seed_lo + (uint32) k) ^ (seed_hi + 0x9e3779b9 (m+1))) mod N_m, and

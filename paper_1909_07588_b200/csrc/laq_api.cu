@@ -71,8 +71,8 @@ const char* check_config(const laq_config* c) {
   if (c->trace_capacity < 0) return "trace_capacity must be >= 0";
   if (c->flags & ~(uint32_t)(LAQ_FLAG_TRIGGER_OFF | LAQ_FLAG_QUANT_OFF)) return "unknown flag";
   if (c->batch < 0) return "batch must be >= 0";
-  if (c->batch > 0 && c->model != LAQ_MODEL_LOGREG_BIN && c->model != LAQ_MODEL_SOFTMAX)
-    return "batch > 0 needs LAQ_MODEL_LOGREG_BIN or LAQ_MODEL_SOFTMAX";
+  if (c->batch > 0 && (c->model == LAQ_MODEL_SYNTH || c->model == LAQ_MODEL_EXTERNAL))
+    return "batch > 0 needs a model with samples";
   const bool data = c->model == LAQ_MODEL_LOGREG_BIN || c->model == LAQ_MODEL_SOFTMAX || c->model == LAQ_MODEL_MLP2;
   if (data) {
     if (!c->N) return "N is null";

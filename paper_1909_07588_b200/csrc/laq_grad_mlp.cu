@@ -33,6 +33,7 @@ constexpr int kThreads = 256;
 constexpr int kMaxC = 16;
 
 struct MlpDev {          // device pointers inside the scratch area
+  int window_tiles = 0;  // 1: the fused hidden kernel skips tiles outside the minibatch window
   __nv_bfloat16* W1T;    // [F][H]
   __nv_bfloat16* Xb;     // all shards, bf16, worker m at row offset rowoff[m]
   __nv_bfloat16* dHb;    // [Ntot][H]
@@ -93,6 +94,7 @@ __global__ void __launch_bounds__(kThreads) mlp_forward_kernel(const Params P, c
   for (int c = 0; c < kMaxC; ++c) acc_w2[c] = 0.f;
   float acc_b2 = 0.f;       // thread t < C
   double loss = 0.0;
+  const RowWindow win = row_window(P, m);   // minibatch: rows outside the window contribute nothing
   const long long ntiles = (n + TR - 1) / TR;
   for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
     const long long r0 = tile * TR;
@@ -172,7 +174,7 @@ __global__ void __launch_bounds__(kThreads) mlp_forward_kernel(const Params P, c
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) z[c] += __shfl_xor_sync(0xffffffffu, z[c], o);
       }
-      if (r < nr) {
+      if (r < nr && win.contains(r0 + r)) {
         float zmax = -3.0e38f;
 #pragma unroll
         for (int c = 0; c < kMaxC; ++c)
@@ -196,7 +198,7 @@ __global__ void __launch_bounds__(kThreads) mlp_forward_kernel(const Params P, c
         }
         if (lane == 0) loss += (double)((zmax + logf(sum)) - zy);
       } else if (lane < kMaxC) {
-        dz[r * kMaxC + lane] = 0.f;   // rows beyond the shard contribute nothing
+        dz[r * kMaxC + lane] = 0.f;   // rows beyond the shard or outside the minibatch contribute nothing
       }
     }
     __syncthreads();
@@ -319,7 +321,7 @@ __global__ void __launch_bounds__(kThreads) mlp_dw1_kernel(const Params P, const
         for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(dv[a], xv[b], acc[a][b]);
     }
   }
-  const float inv_N = (float)(1.0 / (double)P.Ntot);
+  const float inv_N = (float)(batch_scale(P, m) / (double)P.Ntot);
   const float reg = (float)((double)n / (double)P.Ntot * (double)P.lambda);
 #pragma unroll
   for (int a = 0; a < 4; ++a) {
@@ -344,12 +346,13 @@ __global__ void __launch_bounds__(256) mlp_finalize_kernel(const Params P, const
     double s = 0.0;
     for (int b = 0; b < D.gb; ++b) s += (double)D.spart[((long long)m * D.gb + b) * nsmall + i];
     const long long pi = (long long)H * F + i;   // b1, W2, b2 follow W1 in theta in the same order as the partials
-    P.g[(long long)m * P.ps + pi] = (float)(s * inv_N + share * (double)P.lambda * (double)P.theta[pi]);
+    P.g[(long long)m * P.ps + pi] =
+        (float)(s * (inv_N * batch_scale(P, m)) + share * (double)P.lambda * (double)P.theta[pi]);
   }
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     double l = 0.0;
     for (int b = 0; b < D.gb; ++b) l += D.lpart[(long long)m * D.gb + b];
-    P.loss_m[m] = l * inv_N + share * 0.5 * (double)P.lambda * (*theta_sq);
+    P.loss_m[m] = l * (inv_N * batch_scale(P, m)) + share * 0.5 * (double)P.lambda * (*theta_sq);
   }
 }
 
@@ -422,6 +425,7 @@ struct FusedEpi {
   const Params& P;
   const MlpDev& D;
   int nt, m, tile;          // worker and tile index within the worker
+  RowWindow win;            // rows of the worker that enter this iteration's gradient
   __device__ __forceinline__ void run(uint32_t tmem_base, int q, int lane) {
     const int H = P.H, C = P.C, F = P.F;
     const int tt = q * 32 + lane;            // 0..127: the tile row this thread owns
@@ -446,7 +450,7 @@ struct FusedEpi {
     umma::epilogue_sync();
     const long long n = P.N[m];
     const long long trow = (long long)tile * umma::kTileM + tt;   // row within the worker's shard
-    const bool valid = trow < n;
+    const bool valid = trow < n && win.contains(trow);
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
     // ---- pass 1
     float z[12];
@@ -585,17 +589,20 @@ __global__ void __launch_bounds__(umma::kThreads) umma_hidden_fused_kernel(const
                                                                            const Params P, const MlpDev D, int nt) {
   const int m = blockIdx.y, tile = blockIdx.x;
   const long long n = P.N[m];
-  const bool has_rows = (long long)tile * umma::kTileM < n;
-  umma::TileCoord tc{(int)(D.rowoff[m] + (long long)tile * umma::kTileM), 0, 0,
-                     has_rows ? (P.F + umma::kBlockK - 1) / umma::kBlockK : 0};
-  if (!has_rows) {   // a worker with fewer tiles than the grid: its slot holds zeros
+  const RowWindow win = row_window(P, m);
+  const long long t0 = (long long)tile * umma::kTileM, t1 = t0 + umma::kTileM;
+  // the tile has rows of the shard that lie in the window (all rows without a minibatch)
+  const bool has_rows = t0 < n && ((t0 < win.start + win.len_a && t1 > win.start) || t0 < win.len_b);
+  umma::TileCoord tc{(int)(D.rowoff[m] + t0), 0, 0, has_rows ? (P.F + umma::kBlockK - 1) / umma::kBlockK : 0};
+  if (!has_rows) {   // nothing to add from this tile: its slot holds zeros (dH~ of its rows is not written, and
+                     // the dW1 product does not read it)
     const int nsmall = P.H + P.C * P.H + P.C;
     float* sp = D.spart + ((long long)m * D.gb + tile) * nsmall;
     for (int i = threadIdx.x; i < nsmall; i += blockDim.x) sp[i] = 0.f;
     if (threadIdx.x == 0) D.lpart[(long long)m * D.gb + tile] = 0.0;
     return;
   }
-  FusedEpi epi{P, D, nt, m, tile};
+  FusedEpi epi{P, D, nt, m, tile, win};
   umma::gemm_tn_tile(&tmX, &tmW, nt, tc, &P.sc->err, epi);
 }
 
@@ -625,7 +632,27 @@ __global__ void __launch_bounds__(umma::kThreads) umma_dw1_kernel(const __grid_c
   const long long c0 = D.rowoffT[m], c1 = D.rowoffT[m + 1];
   umma::TileCoord tc{(int)blockIdx.y * umma::kTileM, (int)blockIdx.x * nt, (int)c0, (int)((c1 - c0) / umma::kBlockK)};
   const long long n = P.N[m];
-  umma::ChunkEpilogue<Dw1Epi> epi{Dw1Epi{P.g + (long long)m * P.ps, P.theta, (float)(1.0 / (double)P.Ntot),
+  if (D.window_tiles) {
+    // minibatch: only the 128-row tiles that meet the window were written by the hidden kernel in this iteration;
+    // K runs over their 64-column blocks, in two pieces when the window wraps
+    const RowWindow win = row_window(P, m);
+    const int nblk = tc.nkb, per = umma::kTileM / umma::kBlockK;
+    const int a0 = (int)(win.start / umma::kTileM) * per;
+    int a1 = (int)((win.start + win.len_a - 1) / umma::kTileM + 1) * per;
+    a1 = a1 < nblk ? a1 : nblk;
+    int b1 = win.len_b > 0 ? (int)((win.len_b - 1) / umma::kTileM + 1) * per : 0;
+    b1 = b1 < nblk ? b1 : nblk;
+    if (b1 >= a0) {             // one piece from the start of the segment (or no wrap at all and a0 = 0)
+      tc.k0 = (int)c0 + (b1 > 0 ? 0 : a0) * umma::kBlockK;
+      tc.nkb = b1 > 0 ? a1 : a1 - a0;
+    } else {
+      tc.k0 = (int)c0 + a0 * umma::kBlockK;
+      tc.nkb_first = a1 - a0;
+      tc.k1 = (int)c0;
+      tc.nkb = (a1 - a0) + b1;
+    }
+  }
+  umma::ChunkEpilogue<Dw1Epi> epi{Dw1Epi{P.g + (long long)m * P.ps, P.theta, (float)(batch_scale(P, m) / (double)P.Ntot),
                                          (float)((double)n / (double)P.Ntot * (double)P.lambda), P.H, P.F, tc.i0,
                                          tc.j0, nt},
                                   nt};
@@ -795,6 +822,7 @@ laq_status mlp_setup_tensor_path(MlpPlan& mp, const Params& P, cudaStream_t st) 
                                      (int)(umma::smem_bytes(hp->nt1) + fused_extra_floats(P.H) * 4)) == cudaSuccess) {
     hp->fused_tiles = ft;
     hp->d.gb = ft;        // one partial slot per tile
+    hp->d.window_tiles = P.batch > 0 ? 1 : 0;
   } else {
     cudaGetLastError();
   }

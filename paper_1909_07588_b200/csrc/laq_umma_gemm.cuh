@@ -113,9 +113,14 @@ __host__ __device__ constexpr size_t smem_bytes(int nt) { return kStages * stage
 __host__ __device__ constexpr uint32_t tmem_cols(int nt) { return nt <= 32 ? 32u : nt <= 64 ? 64u : nt <= 128 ? 128u : 256u; }
 
 // Which part of the problem a CTA works on: tile origin in A rows (i0) and B rows (j0), and the K range
-// [k0, k0 + 64 nkb) in elements.
+// [k0, k0 + 64 nkb) in elements.  With nkb_first < nkb the range is in two pieces: the first nkb_first blocks
+// start at k0, the remaining ones at k1 (a row window that wraps around the end of a shard).
 struct TileCoord {
   int i0, j0, k0, nkb;
+  int k1 = 0, nkb_first = 0x7fffffff;
+  __device__ __forceinline__ int k_of(int kb) const {
+    return kb < nkb_first ? k0 + kb * kBlockK : k1 + (kb - nkb_first) * kBlockK;
+  }
 };
 
 // Epi::run(tmem_base, q, lane) is executed by the four epilogue warps once the accumulator is complete; warp
@@ -187,8 +192,8 @@ __device__ __forceinline__ void gemm_tn_tile(const CUtensorMap* tmA, const CUten
         if (!mbar_wait(empty0 + 8 * s, par, err_flag, 2u)) break;
         mbar_expect_tx(full0 + 8 * s, st_bytes);
         const uint32_t sa = smem0 + s * st_bytes;
-        tma_load_2d(sa, tmA, full0 + 8 * s, tc.k0 + kb * kBlockK, tc.i0);
-        tma_load_2d(sa + a_bytes, tmB, full0 + 8 * s, tc.k0 + kb * kBlockK, tc.j0);
+        tma_load_2d(sa, tmA, full0 + 8 * s, tc.k_of(kb), tc.i0);
+        tma_load_2d(sa + a_bytes, tmB, full0 + 8 * s, tc.k_of(kb), tc.j0);
       }
     }
   } else if (warp == 1) {

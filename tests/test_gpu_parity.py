@@ -421,6 +421,21 @@ def test_mlp_small_odd_shapes():
     _run_model_parity(w, w.iters)
 
 
+def test_minibatch_mlp_tensor_path_skips_tiles_outside_the_window():
+    """784-200-10 with shards of 700 rows (six 128-row tiles, eleven 64-column blocks) and windows of 200 rows:
+    the hidden product runs on the tiles that meet the window only, the W1 product over their columns, in two
+    pieces when the window wraps."""
+    w = workloads.c3(n_per=700, M=3, iters=14)
+    starts = [oracle.batch_offset(w.seed, m, k, 700) for m in range(3) for k in range(1, 15)]
+    assert any(s + 200 > 700 for s in starts) and any(s + 200 <= 700 and s >= 128 for s in starts)
+    _run_model_parity(w, w.iters, batch=200)
+
+
+def test_minibatch_mlp_plain_path():
+    w = workloads.c3(n_per=37, M=3, F=50, H=24, C=3, iters=10)
+    _run_model_parity(w, w.iters, batch=10)
+
+
 # ------------------------------------------------------------------------------------------------
 # state round trip, error paths
 # ------------------------------------------------------------------------------------------------
