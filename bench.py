@@ -33,7 +33,25 @@ STAGE_KERNELS = {"radius": "radius_kernel", "quantize_norms_trigger": "quantize_
                  "aggregate_theta_step": "aggregate_kernel", "local_gradient": "grad_*_kernel"}
 
 
+MODE_FLAGS = {"lag": 1, "qgd": 2, "gd": 3}          # quantizer off, trigger off, both (LAQ_FLAG_*)
+
+
 def make_workload(name):
+    """c4_b8 (default), c4_b{2,3,4}, c4_b8_M8, c0..c3; suffixes _lag, _qgd, _gd select the baseline modes and
+    _batchN minibatch gradients (model workloads), e.g. c1_b3_batch500."""
+    w = _base_workload(name)
+    w.flags, w.batch = 0, 0
+    for part in name.split("_")[1:]:
+        if part in MODE_FLAGS:
+            w.flags = MODE_FLAGS[part]
+        elif part.startswith("batch") and part[5:].isdigit():
+            w.batch = int(part[5:])
+        elif part.startswith("b") and part[1:].isdigit() and not name.startswith("c4"):
+            w.b = int(part[1:])
+    return w
+
+
+def _base_workload(name):
     from paper_1909_07588_b200 import workloads as W
     if name.startswith("c4"):
         parts = name.split("_")
@@ -47,7 +65,7 @@ def make_workload(name):
             if part.startswith("M") and part[1:].isdigit():
                 kw["M"] = int(part[1:])
         return W.c4(b=b, **kw)
-    return {"c0": W.c0, "c1": W.c1, "c2": W.c2, "c3": W.c3}[name]()
+    return {"c0": W.c0, "c1": W.c1, "c2": W.c2, "c3": W.c3}[name.split("_")[0]]()
 
 
 def hbm_peak():
@@ -69,11 +87,21 @@ def tensor_peak():
 
 
 def algorithmic_bytes(w, u):
-    """Bytes the method must move per iteration, per stage ("Algorithmic bytes").
+    """Bytes the method must move per iteration, per stage: Q_prev (and a stored g) read once per sweep, codes
+    written once, and per uploader codes read and Q_prev rewritten; theta and the aggregate read and written.
     u = uploading fraction |M^k| / M averaged over the timed iterations."""
     Mp = float(w.M) * w.p
     g_bytes = 0.0 if w.model == 3 else 4.0          # g read from HBM unless generated in the kernel
-    X_bytes = sum(n * w.n_features * 4.0 + n * 4.0 for n in w.N) if w.X else 0.0
+    batch = getattr(w, "batch", 0)
+    rows = [min(n, batch) if batch else n for n in w.N]
+    X_bytes = sum(n * w.n_features * 4.0 + n * 4.0 for n in rows) if w.X else 0.0
+    if getattr(w, "flags", 0) & 1:                  # quantizer off: one sweep for radius and norm, raw innovations
+        return {
+            "local_gradient": X_bytes + (Mp * 4.0 if w.X else 0.0),
+            "radius": 0.0,
+            "quantize_norms_trigger": Mp * (4.0 + g_bytes),
+            "aggregate_theta_step": u * Mp * (8.0 + g_bytes) + 16.0 * w.p,
+        }
     return {
         "local_gradient": X_bytes + (Mp * 4.0 if w.X else 0.0),
         "radius": Mp * (4.0 + g_bytes),
@@ -169,13 +197,13 @@ def cpu_baseline(w, name, steps=None, warmup=1, budget_s=12.0):
     if w.model == 3:
         p_s = min(w.p, 1_600_000)
         o = oracle.OracleLaq(32, oracle.MODEL_SYNTH, w.M, p_s, alpha=w.alpha, b=w.b, D=w.D, xi=w.xi, tbar=w.tbar,
-                             seed=w.seed, synth_sigma=w.synth_sigma, synth_eta0=w.synth_eta0)
+                             seed=w.seed, synth_sigma=w.synth_sigma, synth_eta0=w.synth_eta0, flags=w.flags)
         scale = p_s / float(w.p)
         what = "fp32 mirror, M=%d workers, first %d of %d coordinates" % (w.M, p_s, w.p)
     else:
         o = oracle.OracleLaq(64, w.model, w.M, w.p, N=w.N, n_features=w.n_features, n_classes=w.n_classes,
                              n_hidden=w.n_hidden, alpha=w.alpha, lam=w.lam, b=w.b, D=w.D, xi=w.xi, tbar=w.tbar,
-                             bf16_ops=w.bf16_ops, theta0=w.theta0)
+                             bf16_ops=w.bf16_ops, theta0=w.theta0, seed=w.seed, flags=w.flags, batch=w.batch)
         for m in range(w.M):
             o.set_shard(m, w.X[m], w.y[m])
         scale = 1.0
@@ -249,7 +277,7 @@ def main():
         torch.cuda.synchronize()
 
     K, Wm = args.steps, args.warmup
-    ctx = laq.from_workload(w, trace_capacity=max(K, Wm))
+    ctx = laq.from_workload(w, trace_capacity=max(K, Wm), flags=w.flags, batch=w.batch)
     ctx.step(Wm)
     ctx.sync()
     s0 = ctx.get_state(big=False)
@@ -296,7 +324,7 @@ def main():
     theta0_host = torch.zeros(w.p, dtype=torch.float32).pin_memory().numpy() if w.theta0 is None else w.theta0
     barrier()
     t0 = time.perf_counter()
-    ctx2 = laq.from_workload(w, trace_capacity=1, theta0=theta0_host)     # theta0 and the shards cross PCIe here
+    ctx2 = laq.from_workload(w, trace_capacity=1, theta0=theta0_host, flags=w.flags, batch=w.batch)     # theta0 and the shards cross PCIe here
     tr_bytes = 0
     for _ in range(Ke):
         tr = ctx2.step(1, trace=True)                                     # per-step report read back to the host
@@ -322,7 +350,12 @@ def main():
             continue
         avg_ms = stage_ms[i] / iters_recorded  # per iteration (the gradient stage may be several launches)
         gbs = abytes[name] / (avg_ms * 1e-3) / 1e9 if avg_ms > 0 else 0.0
-        stages.append({"stage": name, "kernel": STAGE_KERNELS[name], "ms": avg_ms, "bytes": abytes[name],
+        if (w.flags & 1) and name == "radius":
+            continue                            # quantizer off: radius and norm share one sweep (the next slot)
+        kern = STAGE_KERNELS[name]
+        if w.flags & 1:
+            kern = {"quantize_kernel": "innovation_kernel", "aggregate_kernel": "aggregate_raw_kernel"}.get(kern, kern)
+        stages.append({"stage": name, "kernel": kern, "ms": avg_ms, "bytes": abytes[name],
                        "GB/s": gbs, "frac": gbs / peak, "share": stage_ms[i] / max(stage_ms.sum(), 1e-12)})
     dom = max(stages, key=lambda s: s["ms"])
     path_bytes = sum(s["bytes"] for s in stages)
@@ -355,7 +388,8 @@ def main():
             "warmup": Wm, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "name": w.name, "M": w.M, "p": w.p, "b": w.b, "D": w.D,
-                       "tbar": w.tbar, "alpha": w.alpha, "parallelism": "replicas x%d" % world,
+                       "tbar": w.tbar, "alpha": w.alpha, "flags": w.flags, "batch": w.batch,
+                       "parallelism": "replicas x%d" % world,
                        "l2": "no flush: the state swept every iteration (%.1f GB) exceeds the 126 MB L2"
                              % (ctx.workspace_bytes / 1e9) if ctx.workspace_bytes > 4e8 else
                              "no flush: working set is L2 resident by design of the workload"},

@@ -298,6 +298,7 @@ laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, siz
   P.seed_lo = (uint32_t)(c.seed & 0xffffffffull);
   P.seed_hi = (uint32_t)(c.seed >> 32);
   P.batch = c.batch;
+  P.zero = 0u;
   P.cz = (float)((double)c.synth_sigma / std::sqrt(21845.0));
   P.eta0 = c.synth_eta0;
   P.X = (const float* const*)(ws + pl.Xptr);

@@ -67,6 +67,7 @@ struct Params {
   // synthetic gradient stream
   uint32_t seed_lo, seed_hi;
   int batch;                 // 0: full local gradients; > 0: minibatch size per worker
+  uint32_t zero;             // always 0; opaque to the compiler (used to order a store after a load)
   float cz, eta0;
   // shards
   long long Ntot;

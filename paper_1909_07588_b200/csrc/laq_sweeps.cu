@@ -164,19 +164,20 @@ __device__ __forceinline__ void store_codes(uint32_t* row, uint32_t v, uint32_t 
                                             uint32_t y3, bool valid, long long cw) {
   // y_e = 0x4b000000 + code_e: the code sits in the low bits
   if (B == 3) {
-    // eight neighbouring groups (32 coordinates) fill three words: the 12-bit field of group v starts at bit
-    // 12 (v mod 8) of that 96-bit chunk and may straddle two of its words
+    // eight neighbouring groups (32 coordinates) fill three words.  Lane pairs first join their 12-bit fields into
+    // 24 bits A_0..A_3 (held by the even lanes of the octet); word j of the chunk is then cut out of A_j and A_j+1:
+    // W0 = A0 | A1 << 24, W1 = A1 >> 8 | A2 << 16, W2 = A2 >> 16 | A3 << 8.
     const uint32_t field = valid ? ((y0 & 7u) | ((y1 & 7u) << 3) | ((y2 & 7u) << 6) | ((y3 & 7u) << 9)) : 0u;
-    const uint32_t r = v & 7u, off = 12u * r, wi = off >> 5;
-    const unsigned long long t = (unsigned long long)field << (off & 31u);
-    const uint32_t lo = (uint32_t)t, hi = (uint32_t)(t >> 32);
-    const uint32_t octet = 0xffu << (threadIdx.x & 24u);
-    const uint32_t w0 = __reduce_or_sync(octet, wi == 0 ? lo : 0u);
-    const uint32_t w1 = __reduce_or_sync(octet, wi == 1 ? lo : (wi == 0 ? hi : 0u));
-    const uint32_t w2 = __reduce_or_sync(octet, wi == 2 ? lo : (wi == 1 ? hi : 0u));
-    const bool any_valid = __ballot_sync(octet, valid) != 0u;
+    const uint32_t lane = threadIdx.x & 31u, r = lane & 7u, base = lane & 24u;
+    const uint32_t pair = field | (__shfl_down_sync(0xffffffffu, field, 1) << 12);     // valid in even lanes
+    const uint32_t j = r < 3u ? r : 0u;
+    const uint32_t lo = __shfl_sync(0xffffffffu, pair, base + 2u * j);
+    const uint32_t hi = __shfl_sync(0xffffffffu, pair, base + 2u * j + 2u);
+    // (lo + hi 2^24) >> 8 j, 32 bits of it
+    const uint32_t word_bits = __funnelshift_r(lo | (hi << 24), hi >> 8, 8u * j);
+    const bool any_valid = __ballot_sync(0xffffffffu, valid) & (0xffu << base);
     const long long word = 3ll * (v >> 3) + r;
-    if (any_valid && r < 3u && word < cw) row[word] = r == 0 ? w0 : (r == 1 ? w1 : w2);
+    if (any_valid && r < 3u && word < cw) row[word] = word_bits;
   } else if (B == 16) {
     if (valid) reinterpret_cast<uint2*>(row)[v] = make_uint2(__byte_perm(y0, y1, 0x5410), __byte_perm(y2, y3, 0x5410));
   } else if (B == 8) {
@@ -688,23 +689,34 @@ __global__ void __launch_bounds__(256, LAQ_AGG_MIN_BLOCKS) aggregate_kernel(cons
 
 // Quantizer off: an uploader's innovation is g_m - Q_prev itself and Q_prev becomes g_m.
 template <bool SYNTH>
-__global__ void __launch_bounds__(256, 4) aggregate_raw_kernel(const Params P) {
+__global__ void __launch_bounds__(256, LAQ_AGG_MIN_BLOCKS) aggregate_raw_kernel(const Params P) {
   __shared__ int s_m[kMaxWorkers];
   __shared__ double sh[32];
   __shared__ bool is_last;
   if (*(volatile uint32_t*)&P.sc->err) return;
   const int n_up = (int)P.sc->n_up;
   const unsigned long long k = P.sc->k;
-  for (int u = threadIdx.x; u < n_up; u += blockDim.x) s_m[u] = P.up_m[u];
+  __shared__ Synth s_sy[SYNTH ? kMaxWorkers : 1];
+  for (int u = threadIdx.x; u < n_up; u += blockDim.x) {
+    s_m[u] = P.up_m[u];
+    if (SYNTH) s_sy[u].init(P, s_m[u], k + 1);
+  }
   __syncthreads();
   const uint32_t nv = (uint32_t)P.nv, v_full = (uint32_t)(P.p >> 2), stride = gridDim.x * blockDim.x;
   double dsum = 0.0, tsum = 0.0;
   for (uint32_t v = blockIdx.x * blockDim.x + threadIdx.x; v < nv; v += stride) {
     float4 a = reinterpret_cast<const float4*>(P.agg)[v];
     prefetch_l2(reinterpret_cast<const float4*>(P.theta) + v);
+#pragma unroll
+    for (int j = 0; j < kAggAhead; ++j)
+      if (j < n_up) {
+        const int m1 = s_m[j];
+        prefetch_l2(reinterpret_cast<const float4*>(P.qp + (long long)m1 * P.ps) + v);
+        if (!SYNTH) prefetch_l2(reinterpret_cast<const float4*>(P.g + (long long)m1 * P.ps) + v);
+      }
     for (int u = 0; u < n_up; ++u) {
-      if (u + 1 < n_up) {
-        const int m1 = s_m[u + 1];
+      if (u + kAggAhead < n_up) {
+        const int m1 = s_m[u + kAggAhead];
         prefetch_l2(reinterpret_cast<const float4*>(P.qp + (long long)m1 * P.ps) + v);
         if (!SYNTH) prefetch_l2(reinterpret_cast<const float4*>(P.g + (long long)m1 * P.ps) + v);
       }
@@ -713,13 +725,19 @@ __global__ void __launch_bounds__(256, 4) aggregate_raw_kernel(const Params P) {
       const float4 q = *qptr;
       float4 g;
       if (SYNTH) {
-        Synth sy;
-        sy.init(P, m, k + 1);
+        const Synth sy = s_sy[u];
         g = (v >= v_full) ? sy.at4_masked(v, P.p) : sy.at4(v);
       } else {
         g = __ldg(reinterpret_cast<const float4*>(P.g + (long long)m * P.ps) + v);
       }
-      *qptr = g;
+      {
+        // Q_prev := g exactly.  The stored value is made to depend on the loaded one (AND with a kernel parameter
+        // that is zero): a store issued while the load of the same address is still in flight was measured 3.6
+        // times slower per uploader than one that waits for it.
+        float4 t = g;
+        t.x = __uint_as_float(__float_as_uint(g.x) | (__float_as_uint(q.x) & P.zero));
+        *qptr = t;
+      }
       a.x = __fadd_rn(a.x, __fsub_rn(g.x, q.x));  // uploads are applied in ascending worker order
       a.y = __fadd_rn(a.y, __fsub_rn(g.y, q.y));
       a.z = __fadd_rn(a.z, __fsub_rn(g.z, q.z));
