@@ -273,13 +273,45 @@ __device__ void trigger_stage(const Params& P, int bpw) {
     }
     return;
   }
+  // Sum of the block partials of every worker, in a fixed order.  This block runs alone at the end of the sweep,
+  // so what counts is the number of dependent round trips to L2: with fewer workers than threads a worker's partials
+  // are cut into strips summed by neighbouring threads (all loads of a strip independent), then the strips in order.
+  __shared__ double s_strip[2][512];
+  __shared__ uint32_t s_Rb[kMaxWorkers];   // radius bits, bit 31 = skip
+  const int T = (int)blockDim.x;
+  int tpw = 1;
+  while (tpw < 16 && 2 * tpw * P.M <= T && 2 * tpw * P.M <= 512) tpw *= 2;
+  if (tpw > 1) {
+    const int len = (bpw + tpw - 1) / tpw;
+    if ((int)threadIdx.x < P.M * tpw) {
+      const int m = (int)threadIdx.x / tpw, j = (int)threadIdx.x % tpw;
+      const double* pq = P.part_q + (long long)m * kMaxSweepBlocksPerWorker * 2;
+      const int i1 = min(bpw, (j + 1) * len);
+      double a = 0.0, e = 0.0;
+#pragma unroll 16
+      for (int i = j * len; i < i1; ++i) {
+        a += __ldcg(pq + 2 * i);
+        e += __ldcg(pq + 2 * i + 1);
+      }
+      s_strip[0][threadIdx.x] = a;
+      s_strip[1][threadIdx.x] = e;
+    }
+    __syncthreads();
+  }
   for (int m = threadIdx.x; m < P.M; m += blockDim.x) {
     double n_dq = 0.0, n_eps = 0.0;
-    const double* pq = P.part_q + (long long)m * kMaxSweepBlocksPerWorker * 2;
-#pragma unroll 8
-    for (int i = 0; i < bpw; ++i) {  // fixed order
-      n_dq += __ldcg(pq + 2 * i);
-      n_eps += __ldcg(pq + 2 * i + 1);
+    if (tpw > 1) {
+      for (int j = 0; j < tpw; ++j) {
+        n_dq += s_strip[0][m * tpw + j];
+        n_eps += s_strip[1][m * tpw + j];
+      }
+    } else {
+      const double* pq = P.part_q + (long long)m * kMaxSweepBlocksPerWorker * 2;
+#pragma unroll 16
+      for (int i = 0; i < bpw; ++i) {
+        n_dq += __ldcg(pq + 2 * i);
+        n_eps += __ldcg(pq + 2 * i + 1);
+      }
     }
     double acc = 0.0;
     for (int d = 0; d < P.D; ++d) {
@@ -309,15 +341,16 @@ __device__ void trigger_stage(const Params& P, int bpw) {
       P.t_rhs[trow + m] = rhs;
     }
     P.Rbits[(par ^ 1) * P.M + m] = 0u;  // clear the other parity for the next iteration's max
+    s_Rb[m] = P.Rbits[par * P.M + m] | (skip ? 0x80000000u : 0u);   // finite, so bit 31 is free
   }
   __syncthreads();
-  if (threadIdx.x == 0) {
+  if (threadIdx.x == 0) {   // uploader list in ascending worker order, from shared memory (no global round trips)
     const float levels = (float)((1u << P.b) - 1u);
     const float two_tau = __fmul_rn(2.0f, __fdiv_rn(1.0f, levels));
     int n = 0;
     for (int m = 0; m < P.M; ++m) {
-      if (!P.skip[m]) {
-        const float R = __uint_as_float(P.Rbits[par * P.M + m]);
+      if (!(s_Rb[m] & 0x80000000u)) {
+        const float R = __uint_as_float(s_Rb[m]);
         P.up_m[n] = m;
         P.up_R[n] = R;
         P.up_s[n] = __fmul_rn(two_tau, R);
