@@ -71,7 +71,7 @@ __global__ void __launch_bounds__(kLrThreads) grad_logreg_kernel(const Params P,
   const int f_own = t % F, slice = t / F;
   float acc = 0.f;
   double loss = 0.0;
-  const RowWindow win = row_window(P, m);
+  RowWindow win = row_window(P, m);
   const long long ntiles = win.tiles(rows);
   for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
     long long r0;
@@ -120,6 +120,129 @@ __global__ void __launch_bounds__(kLrThreads) grad_logreg_kernel(const Params P,
   }
 }
 
+// Issue the copies of `count` consecutive floats global -> shared without waiting for them (the caller commits the
+// group and waits later); sources that are not 16-byte aligned are copied with plain loads.
+__device__ __forceinline__ void stage_rows_async(const float* __restrict__ src, float* dst, int count) {
+  if ((reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
+    const int n4 = count >> 2;
+    for (int i = threadIdx.x; i < n4; i += blockDim.x) __pipeline_memcpy_async(dst + 4 * i, src + 4 * i, 16);
+    for (int i = (n4 << 2) + threadIdx.x; i < count; i += blockDim.x) dst[i] = __ldg(src + i);
+  } else {
+    for (int i = threadIdx.x; i < count; i += blockDim.x) dst[i] = __ldg(src + i);
+  }
+}
+
+// The same for an even number of features.  Tiles of 128 rows in a two-deep ring of shared-memory buffers (the next
+// tile arrives while the current one is worked on); 8-byte reads (rows start 8-byte aligned); two threads per row in
+// the first phase (each half of the features, joined through shared memory), two features per thread in the second, so that a
+// residual read from shared memory feeds two multiply-adds.  About a third of the instructions of the kernel above.
+constexpr int kLr2Rows = 128;
+
+__global__ void __launch_bounds__(kLrThreads) grad_logreg_pair_kernel(const Params P, int gbpw) {
+  extern __shared__ __align__(16) float smem[];
+  const int F = P.F, F2 = F >> 1, m = blockIdx.y, t = threadIdx.x;
+  float* xs0 = smem;                         // [2][128][F]
+  float* ths = xs0 + 2 * kLr2Rows * F;       // [F]
+  float* rs = ths + ((F + 3) & ~3);          // [128]
+  float* red = rs + kLr2Rows;                // [2][kLrThreads]
+  __shared__ double shd[32];
+  __shared__ float zpart[kLr2Rows];
+  const float* __restrict__ X = P.X[m];
+  const int32_t* __restrict__ y = P.y[m];
+  for (int f = t; f < F; f += blockDim.x) ths[f] = P.theta[f];
+  const int S = kLrThreads / F2;             // row slices handled in parallel in the second phase
+  const bool active = t < S * F2;
+  const int j_own = t % F2, slice = t / F2;
+  const int row = t & (kLr2Rows - 1), half = t >> 7, fh = (F2 + 1) >> 1;   // first phase: half of the features of a row
+  const int f_lo = half * fh, f_hi = half ? F2 : fh;
+  float acc0 = 0.f, acc1 = 0.f;
+  double loss = 0.0;
+  RowWindow win = row_window(P, m);
+  const long long ntiles = win.tiles(kLr2Rows);
+  auto stage = [&](long long tile, float* xs) {
+    long long r0;
+    int nr;
+    win.tile(tile, kLr2Rows, r0, nr);
+    stage_rows_async(X + r0 * F, xs, nr * F);
+  };
+  int buf = 0;
+  if ((long long)blockIdx.x < ntiles) stage(blockIdx.x, xs0);
+  __pipeline_commit();
+  for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x, buf ^= 1) {
+    long long r0;
+    int nr;
+    win.tile(tile, kLr2Rows, r0, nr);
+    float* xs = xs0 + buf * kLr2Rows * F;
+    __syncthreads();                                  // everybody is done with the buffer refilled below
+    if (tile + gridDim.x < ntiles) stage(tile + gridDim.x, xs0 + (buf ^ 1) * kLr2Rows * F);
+    __pipeline_commit();
+    __pipeline_wait_prior(1);                         // this tile's copies (the older group) have landed
+    __syncthreads();
+    {
+      float z = 0.f;
+      if (row < nr) {
+        const float2* xr = reinterpret_cast<const float2*>(xs + row * F);
+        const float2* th2 = reinterpret_cast<const float2*>(ths);
+#pragma unroll 4
+        for (int f = f_lo; f < f_hi; ++f) {
+          const float2 x = xr[f], th = th2[f];
+          z = fmaf(x.x, th.x, z);
+          z = fmaf(x.y, th.y, z);
+        }
+      }
+      if (half) zpart[row] = z;                       // warps 4-7: second half of the features
+      __syncthreads();
+      if (half == 0 && row < nr) {                    // warps 0-3: join the halves, residual and loss
+        z = z + zpart[row];
+        const float yv = (float)y[r0 + row];
+        float sig, sp;
+        if (z >= 0.f) {
+          const float e = expf(-z);
+          sig = 1.0f / (1.0f + e);
+          sp = z + log1pf(e);
+        } else {
+          const float e = expf(z);
+          sig = e / (1.0f + e);
+          sp = log1pf(e);
+        }
+        rs[row] = sig - yv;
+        loss += (double)(sp - yv * z);
+      }
+    }
+    __syncthreads();
+    if (active) {
+      const float* px = xs + slice * F + 2 * j_own;
+      const int step = S * F;
+#pragma unroll 4
+      for (int r = slice; r < nr; r += S, px += step) {
+        const float2 x = *reinterpret_cast<const float2*>(px);
+        const float rv = rs[r];
+        acc0 = fmaf(rv, x.x, acc0);
+        acc1 = fmaf(rv, x.y, acc1);
+      }
+    }
+  }
+  __pipeline_wait_prior(0);
+  __syncthreads();
+  red[t] = active ? acc0 : 0.f;
+  red[kLrThreads + t] = active ? acc1 : 0.f;
+  __syncthreads();
+  if (t < F) {
+    const float* rp = red + (t & 1) * kLrThreads + (t >> 1);
+    float s = 0.f;
+    for (int sl = 0; sl < S; ++sl) s += rp[sl * F2];
+    P.gpart[((long long)m * gbpw + blockIdx.x) * P.ps + t] = s;
+  }
+  loss = warp_sum_d(loss);
+  if ((t & 31) == 0) shd[t >> 5] = loss;
+  __syncthreads();
+  if (t == 0) {
+    double l = 0.0;
+    for (int i = 0; i < kLrThreads / 32; ++i) l += shd[i];
+    P.lpart[(long long)m * gbpw + blockIdx.x] = l;
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // C-class softmax regression, F <= 1024
 // ------------------------------------------------------------------------------------------------
@@ -143,7 +266,7 @@ __global__ void __launch_bounds__(kSmThreads) grad_softmax_kernel(const Params P
 #pragma unroll
     for (int c = 0; c < C; ++c) acc[j][c] = 0.f;
   double loss = 0.0;
-  const RowWindow win = row_window(P, m);
+  RowWindow win = row_window(P, m);
   const long long ntiles = win.tiles(kSmRows);
   for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
     long long r0;
@@ -262,7 +385,7 @@ __global__ void __launch_bounds__(kS2Threads, 2) grad_softmax_tile_kernel(const 
 #pragma unroll
   for (int c = 0; c < C; ++c) acc01[c] = acc23[c] = 0ull;
   double loss = 0.0;
-  const RowWindow win = row_window(P, m);
+  RowWindow win = row_window(P, m);
   const long long ntiles = win.tiles(kS2Rows);
 
   // asynchronous staging of one tile: contiguous rows in global memory -> padded rows in shared memory
@@ -433,12 +556,13 @@ static int logreg_rows(int F) {
   return r > kLrMaxRows ? kLrMaxRows : r;
 }
 static size_t logreg_smem(int F) {
+  if ((F & 1) == 0) return sizeof(float) * (2 * (size_t)kLr2Rows * F + ((F + 3) & ~3) + kLr2Rows + 2 * kLrThreads);
   return sizeof(float) * ((size_t)logreg_rows(F) * F + ((F + 3) & ~3) + kLrMaxRows + kLrThreads);
 }
 static size_t softmax_smem(int F, int C) { return sizeof(float) * ((size_t)kSmRows * F + (size_t)kSmRows * C); }
 
 int grad_tiles_per_worker(int model, int F, long long n_max) {
-  const long long rows = (model == LAQ_MODEL_LOGREG_BIN) ? logreg_rows(F) : 8;
+  const long long rows = (model == LAQ_MODEL_LOGREG_BIN) ? ((F & 1) ? logreg_rows(F) : kLr2Rows) : 8;
   const long long t = (n_max + rows - 1) / rows;
   return (int)(t > 1024 ? 1024 : (t < 1 ? 1 : t));
 }
@@ -455,9 +579,13 @@ int launch_grad_logreg(const Params& P, const LaunchShape&, int gbpw, cudaStream
   static bool attr_done = false;
   if (!attr_done) {
     cudaFuncSetAttribute(grad_logreg_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    cudaFuncSetAttribute(grad_logreg_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     attr_done = true;
   }
-  grad_logreg_kernel<<<dim3(gbpw, P.M), kLrThreads, sm, st>>>(P, gbpw, logreg_rows(P.F));
+  if ((P.F & 1) == 0)
+    grad_logreg_pair_kernel<<<dim3(gbpw, P.M), kLrThreads, sm, st>>>(P, gbpw);
+  else
+    grad_logreg_kernel<<<dim3(gbpw, P.M), kLrThreads, sm, st>>>(P, gbpw, logreg_rows(P.F));
   return 1;
 }
 

@@ -96,18 +96,19 @@ __device__ __forceinline__ uint32_t fmix32(uint32_t x) {
 // (seed, m, k): rows [start, start + len_a) followed by rows [0, len_b).
 struct RowWindow {
   long long start, len_a, len_b;
-  __device__ __forceinline__ long long tiles(int rows) const {
-    return (len_a + rows - 1) / rows + (len_b + rows - 1) / rows;
+  long long tiles_a = 0;   // set by tiles(): tiles of the first piece (a 64-bit division, done once per kernel)
+  __device__ __forceinline__ long long tiles(int rows) {
+    tiles_a = (len_a + rows - 1) / rows;
+    return tiles_a + (len_b + rows - 1) / rows;
   }
-  // tile t of `rows` rows -> first row and number of rows (tiles never straddle the wrap)
+  // tile t of `rows` rows -> first row and number of rows (tiles never straddle the wrap); tiles(rows) comes first
   __device__ __forceinline__ void tile(long long t, int rows, long long& r0, int& nr) const {
-    const long long ta = (len_a + rows - 1) / rows;
     long long left;
-    if (t < ta) {
+    if (t < tiles_a) {
       r0 = start + t * rows;
       left = len_a - t * rows;
     } else {
-      t -= ta;
+      t -= tiles_a;
       r0 = t * rows;
       left = len_b - t * rows;
     }
