@@ -408,7 +408,7 @@ laq_status laq_step(laq_ctx* ctx, int32_t n_iters, const laq_trace* trace) {
     // run in one single-block kernel
     const bool small = small_iteration_applies(P);
     const bool linear = c.model == LAQ_MODEL_LOGREG_BIN || c.model == LAQ_MODEL_SOFTMAX;
-    const bool fuse_finalize = small && linear && ctx->gbpw <= 8;
+    const bool fuse_finalize = small && linear && ctx->gbpw <= 64;
     switch (c.model) {
       case LAQ_MODEL_LOGREG_BIN:
         ctx->launches += launch_grad_logreg(P, ctx->ls, ctx->gbpw, ctx->st);
