@@ -417,6 +417,8 @@ __global__ void __launch_bounds__(umma::kThreads) umma_hidden_kernel(const __gri
 //               A[c][j] = sum_r dZ[r][c] h[r][j]         (the W2 gradient)
 //               S[c][j] = sum_r dZ[r][c] [h[r][j] > 0]   (then db1[j] = sum_c W2[c][j] S[c][j])
 //           in a fixed order (no atomics).
+constexpr int kFusedStages = 2;   // two stages of ring per block, two blocks per SM
+
 __host__ __device__ inline size_t fused_extra_floats(int H) {
   return (size_t)H * 12 + (size_t)((H + 3) & ~3) + 128 * 33 + 128 * 12 + 2 * (size_t)12 * H + 16;
 }
@@ -429,7 +431,7 @@ struct FusedEpi {
   __device__ __forceinline__ void run(uint32_t tmem_base, int q, int lane) {
     const int H = P.H, C = P.C, F = P.F;
     const int tt = q * 32 + lane;            // 0..127: the tile row this thread owns
-    float* base = reinterpret_cast<float*>(umma::extra_smem(nt));
+    float* base = reinterpret_cast<float*>(umma::ring_smem());   // the ring is free once the accumulator is complete
     float* w2t = base;                       // [H][12]   W2 transposed (j-major), padded rows of 12
     float* b1s = w2t + (size_t)H * 12;       // [H]
     float* chunk = b1s + ((H + 3) & ~3);     // [128][33] one 32-column chunk of h
@@ -584,7 +586,7 @@ struct FusedEpi {
 };
 
 // grid: (tiles per worker, M); tile t of worker m covers the worker's rows 128 t .. 128 t + 127
-__global__ void __launch_bounds__(umma::kThreads) umma_hidden_fused_kernel(const __grid_constant__ CUtensorMap tmX,
+__global__ void __launch_bounds__(umma::kThreads, 2) umma_hidden_fused_kernel(const __grid_constant__ CUtensorMap tmX,
                                                                            const __grid_constant__ CUtensorMap tmW,
                                                                            const Params P, const MlpDev D, int nt) {
   const int m = blockIdx.y, tile = blockIdx.x;
@@ -603,7 +605,7 @@ __global__ void __launch_bounds__(umma::kThreads) umma_hidden_fused_kernel(const
     return;
   }
   FusedEpi epi{P, D, nt, m, tile, win};
-  umma::gemm_tn_tile(&tmX, &tmW, nt, tc, &P.sc->err, epi);
+  umma::gemm_tn_tile<kFusedStages>(&tmX, &tmW, nt, tc, &P.sc->err, epi);
 }
 
 struct Dw1Epi {
@@ -689,7 +691,7 @@ size_t forward_smem_tc(int H) {
 int fused_tiles_for(int F, int H, int C, const long long* N, int M) {
   if (!tc_shape_ok(F, H) || C > 12) return 0;
   const int nt1 = (H + 15) / 16 * 16;
-  if (umma::smem_bytes(nt1) + fused_extra_floats(H) * 4 > 226 * 1024) return 0;
+  if (fused_extra_floats(H) * 4 > kFusedStages * umma::stage_bytes(nt1)) return 0;   // the epilogue's scratch lives in the ring
   long long tiles = 0;
   for (int m = 0; m < M; ++m) {
     const long long t = (N[m] + umma::kTileM - 1) / umma::kTileM;
@@ -819,7 +821,7 @@ laq_status mlp_setup_tensor_path(MlpPlan& mp, const Params& P, cudaStream_t st) 
   hp->tc = true;
   const int ft = fused_tiles_for(P.F, P.H, P.C, hp->N_host.data(), M);
   if (ft > 0 && cudaFuncSetAttribute(umma_hidden_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)(umma::smem_bytes(hp->nt1) + fused_extra_floats(P.H) * 4)) == cudaSuccess) {
+                                     (int)umma::smem_bytes(hp->nt1, kFusedStages)) == cudaSuccess) {
     hp->fused_tiles = ft;
     hp->d.gb = ft;        // one partial slot per tile
     hp->d.window_tiles = P.batch > 0 ? 1 : 0;
@@ -848,7 +850,7 @@ int mlp_launch_gradients(MlpPlan& mp, const Params& P, const double* theta_sq, c
     mlp_pack_w1b_kernel<<<(F * H + 255) / 256, 256, 0, st>>>(P.theta, hp->d.W1b, F * H);
     if (hp->fused_tiles > 0) {
       umma_hidden_fused_kernel<<<dim3(hp->fused_tiles, P.M), umma::kThreads,
-                                 umma::smem_bytes(hp->nt1) + fused_extra_floats(H) * 4, st>>>(hp->tmX, hp->tmW, P, hp->d,
+                                 umma::smem_bytes(hp->nt1, kFusedStages), st>>>(hp->tmX, hp->tmW, P, hp->d,
                                                                                               hp->nt1);
       umma_dw1_kernel<<<dim3((F + hp->nt2 - 1) / hp->nt2, (H + umma::kTileM - 1) / umma::kTileM, P.M), umma::kThreads,
                         umma::smem_bytes(hp->nt2), st>>>(hp->tmD, hp->tmXT, P, hp->d, hp->nt2);

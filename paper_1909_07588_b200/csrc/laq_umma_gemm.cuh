@@ -22,7 +22,7 @@ namespace umma {
 
 constexpr int kTileM = 128;
 constexpr int kBlockK = 64;        // bf16 elements per stage along K: 128 bytes, one swizzle row
-constexpr int kStages = 4;
+constexpr int kStages = 4;          // default depth of the stage ring (gemm_tn_tile<STAGES>)
 constexpr int kThreads = 192;      // 6 warps
 constexpr uint32_t kWaitLimit = 1u << 22;
 
@@ -109,7 +109,7 @@ __device__ __forceinline__ void tmem_load_32(uint32_t taddr, uint32_t (&v)[32]) 
 }
 
 __host__ __device__ constexpr size_t stage_bytes(int nt) { return (size_t)(kTileM + nt) * kBlockK * 2; }
-__host__ __device__ constexpr size_t smem_bytes(int nt) { return kStages * stage_bytes(nt) + 1024 + 256; }
+__host__ __device__ constexpr size_t smem_bytes(int nt, int stages = kStages) { return stages * stage_bytes(nt) + 1024 + 256; }
 __host__ __device__ constexpr uint32_t tmem_cols(int nt) { return nt <= 32 ? 32u : nt <= 64 ? 64u : nt <= 128 ? 128u : 256u; }
 
 // Which part of the problem a CTA works on: tile origin in A rows (i0) and B rows (j0), and the K range
@@ -136,6 +136,15 @@ __device__ __forceinline__ unsigned char* extra_smem(int nt) {
   return umma_smem_raw + (aligned - base) + kStages * stage_bytes(nt);
 }
 
+// The stage ring itself.  Once the accumulator barrier has completed every tensor-core read of the ring is done and
+// no copy is in flight, so an epilogue may use the ring as its scratch: the block then needs no shared memory beyond
+// the ring, and two blocks fit on an SM (one computes while the other runs its epilogue).
+__device__ __forceinline__ unsigned char* ring_smem() {
+  extern __shared__ unsigned char umma_smem_raw[];
+  const uint32_t base = smem_u32(umma_smem_raw);
+  return umma_smem_raw + (((base + 1023u) & ~1023u) - base);
+}
+
 // Adapter: f(row_in_tile, col0, const float (&acc)[32]) is called by the thread that owns accumulator row
 // `row_in_tile` (0..127) for the 32-column chunks col0 = 0, 32, ... < NT.  The last chunk may reach past NT:
 // entries at columns >= NT are undefined and f must ignore them.
@@ -155,18 +164,18 @@ struct ChunkEpilogue {
   }
 };
 
-template <class Epi>
+template <int STAGES = kStages, class Epi>
 __device__ __forceinline__ void gemm_tn_tile(const CUtensorMap* tmA, const CUtensorMap* tmB, int nt, TileCoord tc,
                                              uint32_t* err_flag, Epi& epi) {
   extern __shared__ unsigned char umma_smem_raw[];
-  __shared__ uint64_t bars[2 * kStages + 1];
+  __shared__ uint64_t bars[2 * STAGES + 1];
   __shared__ uint32_t tmem_base_sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem0 = (smem_u32(umma_smem_raw) + 1023u) & ~1023u;   // stages are 1024-byte aligned
   const uint32_t a_bytes = kTileM * kBlockK * 2, st_bytes = (uint32_t)stage_bytes(nt);
-  const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[kStages]), accum = smem_u32(&bars[2 * kStages]);
+  const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]), accum = smem_u32(&bars[2 * STAGES]);
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < STAGES; ++s) {
       mbar_init(full0 + 8 * s, 1);
       mbar_init(empty0 + 8 * s, 1);
     }
@@ -187,8 +196,8 @@ __device__ __forceinline__ void gemm_tn_tile(const CUtensorMap* tmA, const CUten
   if (warp == 0) {
     if (lane == 0) {
       for (int kb = 0; kb < tc.nkb; ++kb) {
-        const int s = kb % kStages;
-        const uint32_t par = ((uint32_t)(kb / kStages) & 1u) ^ 1u;
+        const int s = kb % STAGES;
+        const uint32_t par = ((uint32_t)(kb / STAGES) & 1u) ^ 1u;
         if (!mbar_wait(empty0 + 8 * s, par, err_flag, 2u)) break;
         mbar_expect_tx(full0 + 8 * s, st_bytes);
         const uint32_t sa = smem0 + s * st_bytes;
@@ -201,8 +210,8 @@ __device__ __forceinline__ void gemm_tn_tile(const CUtensorMap* tmA, const CUten
       const uint32_t idesc = instr_desc_bf16(nt);
       bool ok = true;
       for (int kb = 0; kb < tc.nkb && ok; ++kb) {
-        const int s = kb % kStages;
-        ok = mbar_wait(full0 + 8 * s, (uint32_t)(kb / kStages) & 1u, err_flag, 4u);
+        const int s = kb % STAGES;
+        ok = mbar_wait(full0 + 8 * s, (uint32_t)(kb / STAGES) & 1u, err_flag, 4u);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t sa = smem0 + s * st_bytes;
