@@ -33,13 +33,15 @@ struct Synth {
     const uint32_t h0 = fmix32(v ^ key);
     uint32_t h1 = h0 * 0x9e3779b1u;
     h1 ^= h1 >> 15;
-    const int e0 = (int)__dp4a(h0, 0x00010001u, 0u), o0 = (int)__dp4a(h0, 0x01000100u, 0u);  // b0+b2, b1+b3
-    const int e1 = (int)__dp4a(h1, 0x00010001u, 0u), o1 = (int)__dp4a(h1, 0x01000100u, 0u);
+    // b0+b2 and b1+b3 of each word; the even sums land directly on the bit pattern of 1.5 * 2^23 (the dot
+    // product's addend), so that one integer add or subtract per value gives 1.5 * 2^23 + (a small integer)
+    const int e0 = (int)__dp4a(h0, 0x00010001u, 0x4b400000u), o0 = (int)__dp4a(h0, 0x01000100u, 0u);
+    const int e1 = (int)__dp4a(h1, 0x00010001u, 0x4b400000u), o1 = (int)__dp4a(h1, 0x01000100u, 0u);
     // exact int -> float through the mantissa of 1.5 * 2^23 (the -510 offset folds into the constant)
-    const float z0 = __int_as_float(0x4b400000 + e0 + o0) - (12582912.0f + 510.0f);
-    const float z1 = __int_as_float(0x4b400000 + e0 - o0) - 12582912.0f;
-    const float z2 = __int_as_float(0x4b400000 + e1 + o1) - (12582912.0f + 510.0f);
-    const float z3 = __int_as_float(0x4b400000 + e1 - o1) - 12582912.0f;
+    const float z0 = __int_as_float(e0 + o0) - (12582912.0f + 510.0f);
+    const float z1 = __int_as_float(e0 - o0) - 12582912.0f;
+    const float z2 = __int_as_float(e1 + o1) - (12582912.0f + 510.0f);
+    const float z3 = __int_as_float(e1 - o1) - 12582912.0f;
     float4 r;
     r.x = __fmul_rn(__fmaf_rn(drift, z2, z0), cz);
     r.y = __fmul_rn(__fmaf_rn(drift, z3, z1), cz);
@@ -86,8 +88,14 @@ __device__ __forceinline__ double block_sum(double v, double* sh /* >= 32 double
 #ifndef LAQ_SWEEP_UNROLL
 #define LAQ_SWEEP_UNROLL 2
 #endif
+#ifndef LAQ_QUANT_MAX_THREADS
+#define LAQ_QUANT_MAX_THREADS 512
+#endif
 #ifndef LAQ_QUANT_MIN_BLOCKS
 #define LAQ_QUANT_MIN_BLOCKS 2   // caps the quantize kernel at 64 registers (measured best)
+#endif
+#ifndef LAQ_QUANT_CHAINS
+#define LAQ_QUANT_CHAINS 1       // independent fp64 accumulation chains per sum and thread (more: registers spill)
 #endif
 constexpr int kUnroll = LAQ_SWEEP_UNROLL;  // 16-byte groups in flight per thread
 
@@ -253,8 +261,59 @@ __device__ __forceinline__ uint32_t quantize_one(float g, float q, float R, floa
   return __float_as_uint(fl);
 }
 
+// Four coordinates of Eq. (5)/(6) with the code taken from a cheap candidate wherever that provably is the code of
+// the exact evaluation, and from the exact evaluation otherwise.  Exact (reading of Eq. (5) used throughout):
+// x = RN(d + R), u = RN(x / s), code = floor(RN(u + 1/2)).  Candidate: u' = RN(d y + c) in one fused operation,
+// y = RN(1 / s), c = RN(R y).  With v = (d + R) / s <= 2 R / s =: L' (L' = (2^B - 1)(1 + O(2^-23))) and rho = 2^-24:
+//   |u' - v| <= 2 rho v + rho L' / 2 + O(rho^2),   |u - v| <= 2 rho v + O(rho^2),   so   |u' - u| < 1.125 * 2^(B-22).
+// Let f be the integer nearest to u' (one add of 2^23 in round-to-nearest) and w = u' - f.  When
+// |w| <= 1/2 - 2^(B-21), u + 1/2 lies in [f + 0.875 * 2^(B-22), f + 1 - 0.875 * 2^(B-22)], several ulps of 2^B away
+// from both integers, so floor(RN(u + 1/2)) = f.  Otherwise (for b = 8 about one coordinate in 4000) the whole group
+// is redone with the exact quotient.  Codes, dQ and eps are those of quantize_one<true>, bit for bit.
+// Acc = double: fp64 sums of exact products; Acc = float: the caller adds short runs of fp32 sums (see there).
+template <int B, typename Acc>
+__device__ __forceinline__ void quantize_group(const float4& g4, const float4& q4, float R, float s, float y, float c,
+                                               Acc& adq, Acc& aeps, uint32_t (&yy)[4]) {
+  static_assert(B <= 8, "the margin 2^(B-21) is only small for few levels");
+  constexpr float kSafe = 0.5f - (float)(1u << B) * 0x1p-21f;
+  const float g[4] = {g4.x, g4.y, g4.z, g4.w}, q[4] = {q4.x, q4.y, q4.z, q4.w};
+  float fl[4], f[4];
+  float worst = 0.f;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float u = __fmaf_rn(__fsub_rn(g[e], q[e]), y, c);
+    fl[e] = __fadd_rn(u, 8388608.0f);          // 2^23 + (integer nearest to u')
+    f[e] = __fsub_rn(fl[e], 8388608.0f);
+    worst = fmaxf(worst, fabsf(__fsub_rn(u, f[e])));
+  }
+  if (worst > kSafe) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float x = __fadd_rn(__fsub_rn(g[e], q[e]), R);
+      const float u = div_by_reciprocal(x, s, y);
+      fl[e] = __fadd_rd(__fadd_rn(u, 0.5f), 8388608.0f);
+      f[e] = __fsub_rn(fl[e], 8388608.0f);
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float dq = __fsub_rn(__fmul_rn(s, f[e]), R);   // Eq. (6): multiply, then subtract
+    const float er = __fsub_rn(g[e], __fadd_rn(q[e], dq));
+    if constexpr (sizeof(Acc) == 8) {
+      adq = fma((double)dq, (double)dq, adq);           // the product of two fp32 values is exact in fp64
+      aeps = fma((double)er, (double)er, aeps);
+    } else {
+      adq = __fmaf_rn(dq, dq, adq);
+      aeps = __fmaf_rn(er, er, aeps);
+    }
+    yy[e] = __float_as_uint(fl[e]);
+  }
+}
+
 // Skip rule (7a)+(7b), clocks, uploader list, counters: run by the last block of quantize_kernel.
-__device__ void trigger_stage(const Params& P, int bpw) {
+// scratch: kTriggerScratchBytes of shared memory, 8-byte aligned, free for this block to use.
+constexpr size_t kTriggerScratchBytes = 2 * 512 * sizeof(double) + kMaxWorkers * sizeof(uint32_t);
+__device__ void trigger_stage(const Params& P, int bpw, unsigned char* scratch) {
   DevScalars* sc = P.sc;
   const unsigned long long k = sc->k;
   const int par = (int)(k & 1ull);
@@ -276,8 +335,8 @@ __device__ void trigger_stage(const Params& P, int bpw) {
   // Sum of the block partials of every worker, in a fixed order.  This block runs alone at the end of the sweep,
   // so what counts is the number of dependent round trips to L2: with fewer workers than threads a worker's partials
   // are cut into strips summed by neighbouring threads (all loads of a strip independent), then the strips in order.
-  __shared__ double s_strip[2][512];
-  __shared__ uint32_t s_Rb[kMaxWorkers];   // radius bits, bit 31 = skip
+  double (*s_strip)[512] = reinterpret_cast<double (*)[512]>(scratch);                     // [2][512]
+  uint32_t* s_Rb = reinterpret_cast<uint32_t*>(scratch + 2 * 512 * sizeof(double));       // radius bits, bit 31 = skip
   const int T = (int)blockDim.x;
   int tpw = 1;
   while (tpw < 16 && 2 * tpw * P.M <= T && 2 * tpw * P.M <= 512) tpw *= 2;
@@ -366,17 +425,71 @@ __device__ void trigger_stage(const Params& P, int bpw) {
   }
 }
 
+// ---- asynchronous staging of a row through shared memory (quantize sweep over long rows) -----------------------
+// Every warp owns a ring of kRingStages tiles of kRingGroups 16-byte groups of its row of Q_prev.  One lane asks the
+// copy engine for a tile (cp.async.bulk, completion counted in bytes on the stage's mbarrier) kRingStages tiles ahead
+// of the one being worked on, so the loads in flight live in shared memory instead of in registers and no warp
+// waits on a load it has just issued.  A stage is refilled after __syncwarp(): every lane has then read its groups.
+#ifndef LAQ_RING_STAGES
+#define LAQ_RING_STAGES 2
+#endif
+#ifndef LAQ_RING_U
+#define LAQ_RING_U 8
+#endif
+constexpr int kRingStages = LAQ_RING_STAGES;
+constexpr int kRingU = LAQ_RING_U;                 // groups per lane and tile
+constexpr uint32_t kRingGroups = 32 * kRingU;      // 16-byte groups per tile (4 KB)
+constexpr int kRingMaxWarps = 16;                  // warps per block that can own a ring
+constexpr uint32_t kRingWaitLimit = 1u << 22;
+constexpr uint32_t kErrRingWait = 16u;             // bit of DevScalars::err: a wait on a staged tile ran out
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void ring_bar_init(uint32_t bar) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void ring_fetch(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ bool ring_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded: false once the limit is reached (the caller records it and stops using the ring).
+__device__ __forceinline__ bool ring_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t it = 0; it < kRingWaitLimit; ++it) {
+    if (ring_try_wait(bar, parity)) return true;
+    if (it > 64) __nanosleep(64);
+  }
+  return false;
+}
+
 // The per-worker sweep of quantize_kernel (R > 0).  FAST selects the reciprocal-based exact division.
 // Groups [0, nv_main) lie wholly inside the row and run without masks; the few groups after them are
 // handled by the first warp of the worker's first block with per-coordinate masks.  nv_main is even (a multiple
 // of 8 for b = 3), so the lane pairs of the 1-bit packing (the lane octets of the 3-bit packing) never straddle
 // the two parts.
-template <bool SYNTH, int B, bool FAST>
+// RING (rows generated in the kernel, FAST): the full tiles of the row come through the warp's shared-memory ring
+// (ring = the block's dynamic shared memory, bars = kRingStages mbarriers per warp); what is left of the main part
+// (less than one tile) goes through the plain loop below.
+template <bool SYNTH, int B, bool FAST, bool RING>
 __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned long long k, float R, float s,
-                                               double& sdq, double& seps) {
+                                               double& sdq, double& seps, unsigned char* ring = nullptr,
+                                               unsigned long long* bars = nullptr) {
   Synth sy;
   if (SYNTH) sy.init(P, m, k + 1);
-  const float y = __fdiv_rn(1.0f, s);
+  const float y = __fdiv_rn(1.0f, s), cy = __fmul_rn(R, y);
   const float4* __restrict__ q4 = reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps);
   const float4* __restrict__ g4 = SYNTH ? nullptr : reinterpret_cast<const float4*>(P.g + (long long)m * P.ps);
   uint32_t* row = P.codes + (long long)m * P.cw;
@@ -385,9 +498,86 @@ __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned 
                  stride = gridDim.x * blockDim.x;
   const uint32_t lane = threadIdx.x & 31;
   uint32_t v = blockIdx.x * blockDim.x + threadIdx.x;
-  double adq[4] = {0.0, 0.0, 0.0, 0.0}, aeps[4] = {0.0, 0.0, 0.0, 0.0};
+  constexpr int NC = LAQ_QUANT_CHAINS;
+  double adq[NC], aeps[NC];
+#pragma unroll
+  for (int c = 0; c < NC; ++c) adq[c] = aeps[c] = 0.0;
+  if constexpr (RING) {
+    const uint32_t w = threadIdx.x >> 5, wpb = blockDim.x >> 5;
+    const uint32_t gw = blockIdx.x * wpb + w, nw = gridDim.x * wpb;      // this warp among the worker's warps
+    const uint32_t n_tiles = nv_main / kRingGroups;
+    const uint32_t n_my = n_tiles > gw ? (n_tiles - gw + nw - 1) / nw : 0u;  // tiles gw, gw + nw, ...
+    const float4* stage0 = reinterpret_cast<const float4*>(ring) + (size_t)w * kRingStages * kRingGroups;
+    const uint32_t stage_a = smem_addr(stage0), bar_a = smem_addr(bars + w * kRingStages);
+    constexpr uint32_t kTileBytes = kRingGroups * 16;
+    if (lane == 0) {
+      for (int st = 0; st < kRingStages; ++st) ring_bar_init(bar_a + 8 * st);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      for (uint32_t i = 0; i < (uint32_t)kRingStages && i < n_my; ++i)
+        ring_fetch(stage_a + i * kTileBytes, q4 + (size_t)(gw + i * nw) * kRingGroups, kTileBytes, bar_a + 8 * i);
+    }
+    __syncwarp();
+    // per-lane state that advances by a constant per tile: first group of the tile for this lane, source of the
+    // tile kRingStages ahead, byte offset of the current stage
+    uint32_t v0 = gw * kRingGroups + lane;
+    const float4* src_ahead = q4 + (size_t)(gw + (uint32_t)kRingStages * nw) * kRingGroups;
+    const uint32_t step_groups = nw * kRingGroups;
+    uint32_t st = 0, parity = 0, done = 0;
+    for (; done < n_my; ++done) {
+      if (!__all_sync(0xffffffffu, ring_wait(bar_a + 8 * st, parity))) break;
+      const float4* tile = stage0 + st * kRingGroups + lane;
+      uint32_t* out = row + v0;
+      // the 4 kRingU coordinates of a lane in this tile are summed in fp32 (fused multiply-adds, 4 kRingU - 1
+      // roundings: relative error of the run below 4 kRingU * 2^-24) and the run is then added in fp64; with
+      // hundreds of thousands of runs per row the sums agree with the fp64 sums of exact products to ~1e-9
+      float rdq = 0.f, reps = 0.f;
+#pragma unroll
+      for (int j = 0; j < kRingU; ++j) {
+        const float4 q = tile[32 * j];
+        const float4 g = sy.at4(v0 + 32 * j);
+        uint32_t yy[4];
+        if constexpr (B <= 8) {
+          quantize_group<B>(g, q, R, s, y, cy, rdq, reps, yy);
+        } else {
+          yy[0] = quantize_one<true>(g.x, q.x, R, s, y, adq[0 % NC], aeps[0 % NC]);
+          yy[1] = quantize_one<true>(g.y, q.y, R, s, y, adq[1 % NC], aeps[1 % NC]);
+          yy[2] = quantize_one<true>(g.z, q.z, R, s, y, adq[2 % NC], aeps[2 % NC]);
+          yy[3] = quantize_one<true>(g.w, q.w, R, s, y, adq[3 % NC], aeps[3 % NC]);
+        }
+        if constexpr (B == 8) out[32 * j] = __byte_perm(__byte_perm(yy[0], yy[1], 0x0040), __byte_perm(yy[2], yy[3], 0x0040), 0x5410);
+        else store_codes<B>(row, v0 + 32 * j, yy[0], yy[1], yy[2], yy[3], true, P.cw);
+      }
+      if constexpr (B <= 8) {
+        adq[0] += (double)rdq;
+        aeps[0] += (double)reps;
+      }
+      __syncwarp();                                // every lane has read its groups: the stage may be refilled
+      if (lane == 0 && done + kRingStages < n_my) ring_fetch(stage_a + st * kTileBytes, src_ahead, kTileBytes, bar_a + 8 * st);
+      src_ahead += step_groups;
+      v0 += step_groups;
+      if (++st == (uint32_t)kRingStages) {
+        st = 0;
+        parity ^= 1u;
+      }
+    }
+    if (done < n_my) {
+      // a wait ran out: record it, and before leaving give the copies still in flight (at most kRingStages tiles,
+      // this one included) the same bounded time to land, so that none writes into shared memory of a later block
+      if (lane == 0) atomicOr(&P.sc->err, kErrRingWait);
+      const uint32_t issued = min(n_my, done + (uint32_t)kRingStages);
+      for (uint32_t i = done; i < issued; ++i) {
+        ring_wait(bar_a + 8 * st, parity);
+        if (++st == (uint32_t)kRingStages) {
+          st = 0;
+          parity ^= 1u;
+        }
+      }
+    }
+    v = n_tiles * kRingGroups + blockIdx.x * blockDim.x + threadIdx.x;   // what is left of the main part
+  }
   // hot loop: every group of every lane of the warp is valid, no predicates
-  for (; (unsigned long long)(v - lane + 31) + (kUnroll - 1) * (unsigned long long)stride < nv_main;
+  for (; !RING && (unsigned long long)(v - lane + 31) + (kUnroll - 1) * (unsigned long long)stride < nv_main;
        v += kUnroll * stride) {
     float4 q[kUnroll], g[kUnroll];
 #pragma unroll
@@ -397,15 +587,29 @@ __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned 
     }
 #pragma unroll
     for (int j = 0; j < kUnroll; ++j) {  // four independent accumulation chains per sum
-      const uint32_t y0 = quantize_one<FAST>(g[j].x, q[j].x, R, s, y, adq[0], aeps[0]);
-      const uint32_t y1 = quantize_one<FAST>(g[j].y, q[j].y, R, s, y, adq[1], aeps[1]);
-      const uint32_t y2 = quantize_one<FAST>(g[j].z, q[j].z, R, s, y, adq[2], aeps[2]);
-      const uint32_t y3 = quantize_one<FAST>(g[j].w, q[j].w, R, s, y, adq[3], aeps[3]);
-      store_codes<B>(row, v + j * stride, y0, y1, y2, y3, true, P.cw);
+      if constexpr (FAST && B <= 8) {
+        uint32_t yy[4];
+        quantize_group<B>(g[j], q[j], R, s, y, cy, adq[0], aeps[0], yy);
+        store_codes<B>(row, v + j * stride, yy[0], yy[1], yy[2], yy[3], true, P.cw);
+      } else {
+        const uint32_t y0 = quantize_one<FAST>(g[j].x, q[j].x, R, s, y, adq[0 % NC], aeps[0 % NC]);
+        const uint32_t y1 = quantize_one<FAST>(g[j].y, q[j].y, R, s, y, adq[1 % NC], aeps[1 % NC]);
+        const uint32_t y2 = quantize_one<FAST>(g[j].z, q[j].z, R, s, y, adq[2 % NC], aeps[2 % NC]);
+        const uint32_t y3 = quantize_one<FAST>(g[j].w, q[j].w, R, s, y, adq[3 % NC], aeps[3 % NC]);
+        store_codes<B>(row, v + j * stride, y0, y1, y2, y3, true, P.cw);
+      }
     }
   }
-  sdq += (adq[0] + adq[1]) + (adq[2] + adq[3]);
-  seps += (aeps[0] + aeps[1]) + (aeps[2] + aeps[3]);
+  if constexpr (NC == 4) {
+    sdq += (adq[0] + adq[1]) + (adq[2] + adq[3]);
+    seps += (aeps[0] + aeps[1]) + (aeps[2] + aeps[3]);
+  } else {
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+      sdq += adq[c];
+      seps += aeps[c];
+    }
+  }
   // remainder of the main part: all lanes of a warp run the same number of trips (the 1-bit packing
   // shuffles between lanes), invalid lanes compute on harmless operands and store nothing
   for (; v - lane < nv_main; v += stride) {
@@ -451,9 +655,12 @@ __device__ __forceinline__ void zero_codes(const Params& P, int m) {
 }
 
 template <bool SYNTH, int B>
-__global__ void __launch_bounds__(512, LAQ_QUANT_MIN_BLOCKS) quantize_kernel(const Params P) {
+__global__ void __launch_bounds__(LAQ_QUANT_MAX_THREADS, LAQ_QUANT_MIN_BLOCKS) quantize_kernel(const Params P) {
   __shared__ double sh[32];
   __shared__ bool is_last;
+  __shared__ __align__(8) unsigned long long ring_bars[SYNTH ? kRingMaxWarps * kRingStages : 1];
+  // dynamic shared memory: the trigger stage's scratch and, for SYNTH, kRingStages tiles per warp (the larger of both)
+  extern __shared__ __align__(128) unsigned char ring_smem[];
   const int m = blockIdx.y;
   const bool frozen = *(volatile uint32_t*)&P.sc->err != 0;
   const unsigned long long k = P.sc->k;
@@ -467,9 +674,9 @@ __global__ void __launch_bounds__(512, LAQ_QUANT_MIN_BLOCKS) quantize_kernel(con
     if (!(R > 0.f))
       zero_codes<B>(P, m);
     else if (s >= 0x1p-60f && s <= 0x1p60f)
-      quantize_sweep<SYNTH, B, true>(P, m, k, R, s, sdq, seps);
+      quantize_sweep<SYNTH, B, true, SYNTH>(P, m, k, R, s, sdq, seps, ring_smem, ring_bars);
     else
-      quantize_sweep<SYNTH, B, false>(P, m, k, R, s, sdq, seps);
+      quantize_sweep<SYNTH, B, false, false>(P, m, k, R, s, sdq, seps);
   }
   const double tdq = block_sum(sdq, sh);
   const double teps = block_sum(seps, sh);
@@ -486,7 +693,7 @@ __global__ void __launch_bounds__(512, LAQ_QUANT_MIN_BLOCKS) quantize_kernel(con
   __syncthreads();
   if (is_last && !frozen) {
     __threadfence();
-    trigger_stage(P, gridDim.x);
+    if (*(volatile uint32_t*)&P.sc->err == 0) trigger_stage(P, gridDim.x, ring_smem);   // no block gave up on a tile
   }
 }
 
@@ -501,6 +708,7 @@ __global__ void __launch_bounds__(512) innovation_kernel(const Params P) {
   __shared__ double sh[32];
   __shared__ uint32_t shm[32];
   __shared__ bool is_last;
+  __shared__ __align__(8) unsigned char trig_scratch[kTriggerScratchBytes];
   const int m = blockIdx.y;
   const bool frozen = *(volatile uint32_t*)&P.sc->err != 0;
   const unsigned long long k = P.sc->k;
@@ -561,7 +769,7 @@ __global__ void __launch_bounds__(512) innovation_kernel(const Params P) {
   __syncthreads();
   if (is_last && !frozen) {
     __threadfence();
-    trigger_stage(P, gridDim.x);
+    trigger_stage(P, gridDim.x, trig_scratch);
   }
 }
 
@@ -1018,15 +1226,26 @@ __global__ void __launch_bounds__(kSmallThreads) small_iteration_kernel(const Pa
   }
 }
 
+template <bool SYNTH, int B>
+void launch_quant_one(const Params& P, dim3 grid, int threads, size_t smem, cudaStream_t st) {
+  // more than the default 48 KB of dynamic shared memory has to be asked for (a failure shows up in the launch)
+  if (smem > 40 * 1024)
+    cudaFuncSetAttribute(quantize_kernel<SYNTH, B>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  quantize_kernel<SYNTH, B><<<grid, threads, smem, st>>>(P);
+}
+
 template <bool SYNTH>
 void launch_quant_b(const Params& P, dim3 grid, int threads, cudaStream_t st) {
+  // rows generated in the kernel: every warp stages its tiles of Q_prev through a ring in dynamic shared memory
+  const size_t ring = SYNTH ? (size_t)(threads / 32) * kRingStages * kRingGroups * 16 : 0;
+  const size_t smem = ring > kTriggerScratchBytes ? ring : kTriggerScratchBytes;
   switch (P.b) {
-    case 1: quantize_kernel<SYNTH, 1><<<grid, threads, 0, st>>>(P); break;
-    case 2: quantize_kernel<SYNTH, 2><<<grid, threads, 0, st>>>(P); break;
-    case 3: quantize_kernel<SYNTH, 3><<<grid, threads, 0, st>>>(P); break;
-    case 4: quantize_kernel<SYNTH, 4><<<grid, threads, 0, st>>>(P); break;
-    case 8: quantize_kernel<SYNTH, 8><<<grid, threads, 0, st>>>(P); break;
-    default: quantize_kernel<SYNTH, 16><<<grid, threads, 0, st>>>(P); break;
+    case 1: launch_quant_one<SYNTH, 1>(P, grid, threads, smem, st); break;
+    case 2: launch_quant_one<SYNTH, 2>(P, grid, threads, smem, st); break;
+    case 3: launch_quant_one<SYNTH, 3>(P, grid, threads, smem, st); break;
+    case 4: launch_quant_one<SYNTH, 4>(P, grid, threads, smem, st); break;
+    case 8: launch_quant_one<SYNTH, 8>(P, grid, threads, smem, st); break;
+    default: launch_quant_one<SYNTH, 16>(P, grid, threads, smem, st); break;
   }
 }
 
