@@ -24,8 +24,11 @@
  *   - Floating point: theta, gradients and quantizer state are fp32; each quantizer operation is one
  *     IEEE round-to-nearest operation in the order  d = g - Q_prev ; R = max|d| ; s = (2 tau) R ;
  *     t = (d + R)/s + 1/2 (IEEE division) ; q = floor t ; dQ = s q - R (multiply, then subtract) ;
- *     Q_new = Q_prev + dQ ; eps = g - Q_new, with no fused multiply-add; squared norms are fp64 sums of
- *     exact fp32 products; the skip rule is evaluated in fp64.
+ *     Q_new = Q_prev + dQ ; eps = g - Q_new, with no fused multiply-add (kernels may reach q by a cheaper
+ *     route where they can prove that it gives the same integer); codes, dQ, Q_new and eps are therefore
+ *     reproducible bit for bit.  Squared norms are fp64 sums of exact fp32 products, except that the sweep over
+ *     rows generated in the kernel (LAQ_MODEL_SYNTH) first sums runs of 32 products in fp32 (relative error of
+ *     a run below 2^-19; of a whole row typically 1e-9); the skip rule is evaluated in fp64.
  *   - Code stream of worker m (the paper's b p-bit part of the upload message): code i occupies bits
  *     [i b, (i+1) b) of the stream, bit j of the stream being bit (j mod 32) of 32-bit word floor(j / 32)
  *     (least significant first; for b = 3 a code may straddle two words).

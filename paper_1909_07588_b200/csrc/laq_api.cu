@@ -206,7 +206,8 @@ laq_status check_device_error(laq_ctx* ctx) {
   LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));
   if (err & 1u)
     return fail(ctx, LAQ_ENONFINITE, "a gradient or radius was not finite; the state is frozen at that iteration");
-  if (err & ~1u) return fail(ctx, LAQ_ECUDA, "a bounded wait in the tensor-core pipeline ran out; the state is frozen");
+  if (err & ~1u)
+    return fail(ctx, LAQ_ECUDA, "a bounded wait on an asynchronous copy or tensor-core stage ran out; the state is frozen");
   return LAQ_OK;
 }
 
