@@ -109,7 +109,7 @@ struct Plan {
 
 int default_gbpw(const laq_config& c) {
   // one wave of resident blocks (shared memory decides how many fit on an SM)
-  int g = (grad_blocks_per_sm(c.model, c.n_features) * kNumSMs) / c.M;
+  int g = (grad_blocks_per_sm(c.model, c.n_features, c.n_classes) * kNumSMs) / c.M;
   if (g > kGradBlocksCap) g = kGradBlocksCap;
   return g < 1 ? 1 : g;
 }
@@ -315,7 +315,7 @@ laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, siz
   if (c.model == LAQ_MODEL_LOGREG_BIN || c.model == LAQ_MODEL_SOFTMAX) {
     long long n_max = 1;
     for (int m = 0; m < c.M; ++m) n_max = ctx->N[m] > n_max ? ctx->N[m] : n_max;
-    const int tiles = grad_tiles_per_worker(c.model, c.n_features, n_max);
+    const int tiles = grad_tiles_per_worker(c.model, c.n_features, c.n_classes, n_max);
     if (ctx->gbpw > tiles) ctx->gbpw = tiles;
   }
 

@@ -361,10 +361,12 @@ constexpr int kS2Warps = 7;
 constexpr int kS2Rows = 8;
 constexpr int kS2Parts = 4 * kS2Warps;   // partial scores per (row, class)
 
-template <int C>
+// FT > 0 fixes the feature count at compile time (784, the 28 x 28 inputs of the paper's tests): every row and
+// class offset is then an immediate and the loops have known trip counts; FT = 0 reads it from the parameters.
+template <int C, int FT>
 __global__ void __launch_bounds__(kS2Threads, 2) grad_softmax_tile_kernel(const Params P, int gbpw) {
   extern __shared__ __align__(16) float smem[];
-  const int F = P.F, F4 = F >> 2, FP4 = F4 | 1, FP = FP4 << 2;      // padded row stride (floats)
+  const int F = FT > 0 ? FT : P.F, F4 = F >> 2, FP4 = F4 | 1, FP = FP4 << 2;      // padded row stride (floats)
   const int m = blockIdx.y, t = threadIdx.x, lane = t & 31, w = t >> 5;
   float* xs0 = smem;                                 // [2][8][FP]
   float* ths = xs0 + 2 * kS2Rows * FP;               // [C][F]      theta
@@ -545,10 +547,242 @@ __global__ void __launch_bounds__(256) grad_finalize_kernel(const Params P, int 
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// C-class softmax regression, wide path: feature count fixed at compile time (a multiple of 16), C <= 10.
+// One block of 256 threads per SM; tiles of 24 rows in two shared-memory stages.  The eighth warp asks the copy
+// engine for the next tile (one bulk copy per row into rows padded to an odd number of 16-byte units, completion
+// counted in bytes on the stage's mbarrier, bounded waits) while warps 0-6 work on the current one:
+//   scores     lane = (row group rg = lane mod 8, phase kp = lane / 8) owns rows rg, rg + 8, rg + 16 and, in each
+//              trip, the 16-byte feature group 4 (w + 7 trip) + kp: three 16-byte reads of x, C broadcast reads of
+//              theta, 6 C packed multiply-adds; the 28 partial scores per (row, class) go through shared memory;
+//   softmax    one thread per (row, class), a row's classes in neighbouring lanes: sum of the partials in a fixed
+//              order, maximum and sum of the row by shuffles (the same order in every lane of a row), residual, loss;
+//              the row's label is asked for before the score product;
+//   gradient   thread = four consecutive features: acc[4][C] += residual[r][c] x[r][f] over the tile's rows.
+// Every offset is an immediate and every loop has a known trip count.
+// ------------------------------------------------------------------------------------------------
+constexpr int kSwThreads = 256;
+constexpr int kSwWarps = 7;
+#ifndef LAQ_SW_RPL
+#define LAQ_SW_RPL 3
+#endif
+#ifndef LAQ_SW_STAGES
+#define LAQ_SW_STAGES 2
+#endif
+constexpr int kSwRpl = LAQ_SW_RPL;         // rows per lane in the score product
+constexpr int kSwRows = 8 * kSwRpl;        // rows per tile
+constexpr int kSwStages = LAQ_SW_STAGES;   // tiles in shared memory: one at work, the others on their way
+constexpr int kSwParts = 4 * kSwWarps;
+
+template <int C, int FT>
+struct SwShape {
+  static constexpr int F = FT, F4 = FT / 4, FP4 = F4 | 1, FP = FP4 * 4, QUADS = F4 / 4;
+  static constexpr int ITERS = (QUADS + kSwWarps - 1) / kSwWarps;
+  static constexpr int RC = kSwRows * C;
+  // floats: stages of samples, theta, partial scores, residual pairs
+  static constexpr size_t kFloats = kSwStages * (size_t)kSwRows * FP + (size_t)C * F + (size_t)kSwParts * RC + (size_t)kSwRows * 24;
+  static_assert(FT % 16 == 0 && F4 <= kSwThreads, "feature groups: a thread per group, four groups per trip");
+  static_assert(C >= 2 && C <= 10 && kSwRpl * C <= 32 && kSwThreads == 256, "a warp's lanes = its rows x classes");
+};
+
+template <int C, int FT>
+__global__ void __launch_bounds__(kSwThreads, 1) grad_softmax_wide_kernel(const Params P, int gbpw) {
+  using S = SwShape<C, FT>;
+  constexpr int F = S::F, F4 = S::F4, FP = S::FP, RC = S::RC;
+  extern __shared__ __align__(128) float smem[];
+  float* xs0 = smem;                                  // [stages][rows][FP]
+  float* ths = xs0 + kSwStages * kSwRows * FP;        // [C][F]
+  float* plog = ths + C * F;                          // [28][24][C]
+  float* res = plog + kSwParts * RC;                  // [rows][12][2] residuals, each stored twice (packed pairs)
+  __shared__ double shd[kSwThreads / 32];
+  __shared__ __align__(8) unsigned long long bars[kSwStages];
+  const int m = blockIdx.y, t = threadIdx.x, lane = t & 31, w = t >> 5;
+  const float* __restrict__ X = P.X[m];
+  const int32_t* __restrict__ y = P.y[m];
+  const uint32_t bar_a = smem_addr(bars), xs_a = smem_addr(xs0);
+  RowWindow win = row_window(P, m);
+  const long long ntiles = win.tiles(kSwRows);
+
+  // the producer warp asks for one tile: a copy per row, all counted on the stage's barrier
+  auto request = [&](long long tile, int s) {
+    long long r0;
+    int nr;
+    win.tile(tile, kSwRows, r0, nr);
+    if (lane == 0) ring_expect(bar_a + 8 * s, (uint32_t)nr * F * 4u);
+    __syncwarp();
+    if (lane < nr)
+      ring_copy(xs_a + (uint32_t)((s * kSwRows + lane) * FP) * 4u, X + (r0 + lane) * F, F * 4u, bar_a + 8 * s);
+  };
+
+  if (t == 0) {
+    for (int s = 0; s < kSwStages; ++s) ring_bar_init(bar_a + 8 * s);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  for (int i = t; i < C * F4; i += kSwThreads)
+    reinterpret_cast<float4*>(ths)[i] = __ldg(reinterpret_cast<const float4*>(P.theta) + i);
+  __syncthreads();
+  if (w == kSwWarps)   // the first tiles of this block, one per stage but the last
+    for (int s = 0; s < kSwStages - 1; ++s)
+      if ((long long)blockIdx.x + (long long)s * gridDim.x < ntiles) request(blockIdx.x + (long long)s * gridDim.x, s);
+
+  const bool owner = t < F4;                          // gradient phase: thread t owns features 4t .. 4t+3
+  unsigned long long acc01[C], acc23[C];              // packed pairs (features 4t, 4t+1) and (4t+2, 4t+3)
+#pragma unroll
+  for (int c = 0; c < C; ++c) acc01[c] = acc23[c] = 0ull;
+  double loss = 0.0;
+  const int rg = lane & 7, kp = lane >> 3;
+  // softmax phase: warp w owns rows kSwRpl w .. kSwRpl w + kSwRpl - 1, lane = (row within the warp, class)
+  constexpr uint32_t kRcMask = (kSwRpl * C >= 32) ? 0xffffffffu : ((1u << (kSwRpl * C)) - 1u);
+  const bool rc_lane = lane < kSwRpl * C;
+  const int row_rc = kSwRpl * w + lane / C, cls_rc = lane % C;
+  bool failed = false;
+  int i = 0, s = 0;
+  uint32_t parity = 0;
+  long long tile = blockIdx.x;
+  for (; tile < ntiles; tile += gridDim.x, ++i) {
+    long long r0;
+    int nr;
+    win.tile(tile, kSwRows, r0, nr);
+    const bool landed = ring_wait(bar_a + 8 * s, parity);
+    // also: everybody is done with the previous tile, whose stage the next request overwrites
+    if (!__syncthreads_and(landed ? 1 : 0)) {
+      failed = true;
+      break;
+    }
+    // the row's label, asked for now and used after the score product
+    const int yv = (rc_lane && row_rc < nr) ? __ldg(y + r0 + row_rc) : -1;
+    const long long ahead = tile + (long long)(kSwStages - 1) * gridDim.x;
+    if (w == kSwWarps && ahead < ntiles) request(ahead, s == 0 ? kSwStages - 1 : s - 1);
+    float* xs = xs0 + s * kSwRows * FP;
+    if (nr < kSwRows) {   // rows beyond the window's piece: zeros (block-uniform branch)
+      for (int j = t; j < (kSwRows - nr) * F4; j += kSwThreads) {
+        const int r = nr + j / F4, k = j - (j / F4) * F4;
+        *reinterpret_cast<float4*>(xs + r * FP + 4 * k) = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+      __syncthreads();
+    }
+    if (w < kSwWarps) {  // scores
+      unsigned long long z2[kSwRpl][C];
+#pragma unroll
+      for (int r = 0; r < kSwRpl; ++r)
+#pragma unroll
+        for (int c = 0; c < C; ++c) z2[r][c] = 0ull;
+      const float* xb = xs + rg * FP + 4 * kp;
+      const float* tb = ths + 4 * kp;
+#pragma unroll
+      for (int it = 0; it < S::ITERS; ++it) {
+        const int q = w + kSwWarps * it;
+        if (S::QUADS % kSwWarps == 0 || q < S::QUADS) {
+          ulonglong2 x[kSwRpl];
+#pragma unroll
+          for (int r = 0; r < kSwRpl; ++r) x[r] = *reinterpret_cast<const ulonglong2*>(xb + 16 * q + 8 * r * FP);
+#pragma unroll
+          for (int c = 0; c < C; ++c) {
+            const ulonglong2 th = *reinterpret_cast<const ulonglong2*>(tb + c * F + 16 * q);
+#pragma unroll
+            for (int r = 0; r < kSwRpl; ++r) z2[r][c] = ffma2(x[r].x, th.x, z2[r][c]);
+#pragma unroll
+            for (int r = 0; r < kSwRpl; ++r) z2[r][c] = ffma2(x[r].y, th.y, z2[r][c]);
+          }
+        }
+      }
+      float* pl = plog + ((4 * w + kp) * kSwRows + rg) * C;
+#pragma unroll
+      for (int r = 0; r < kSwRpl; ++r)
+#pragma unroll
+        for (int c = 0; c < C; ++c) {
+          float lo, hi;
+          unpack2(z2[r][c], lo, hi);
+          pl[8 * r * C + c] = lo + hi;
+        }
+    }
+    __syncthreads();
+    if (rc_lane) {  // one thread per (row, class); the classes of a row sit in neighbouring lanes of one warp
+      float z = 0.f;
+#pragma unroll
+      for (int pp = 0; pp < kSwParts; ++pp) z += plog[pp * RC + row_rc * C + cls_rc];   // fixed order
+      // every lane of a row reads the row's C values in the same order: identical maximum and sum in all of them
+      const int lane0 = lane - cls_rc;
+      float zmax = __shfl_sync(kRcMask, z, lane0);
+#pragma unroll
+      for (int c = 1; c < C; ++c) zmax = fmaxf(zmax, __shfl_sync(kRcMask, z, lane0 + c));
+      const float e = expf(z - zmax);
+      float sum = 0.f;
+#pragma unroll
+      for (int c = 0; c < C; ++c) sum += __shfl_sync(kRcMask, e, lane0 + c);
+      const float zy = __shfl_sync(kRcMask, z, lane0 + (yv >= 0 ? yv : 0));
+      const bool live = row_rc < nr;
+      const float inv = 1.0f / sum;
+      const float rv = live ? (e * inv - (cls_rc == yv ? 1.f : 0.f)) : 0.f;
+      res[(row_rc * 12 + cls_rc) * 2] = rv;
+      res[(row_rc * 12 + cls_rc) * 2 + 1] = rv;
+      if (live && cls_rc == 0) loss += (double)((zmax + logf(sum)) - zy);
+    }
+    __syncthreads();
+    if (owner) {  // gradient
+      const float* xc = xs + 4 * t;
+#pragma unroll 4
+      for (int r = 0; r < kSwRows; ++r) {             // rows beyond the piece hold zero residuals and zero samples
+        const ulonglong2 x = *reinterpret_cast<const ulonglong2*>(xc + r * FP);
+        const ulonglong2* rp = reinterpret_cast<const ulonglong2*>(res + r * 24);
+#pragma unroll
+        for (int c = 0; c < C; c += 2) {
+          const ulonglong2 rr = rp[c >> 1];           // (r_c, r_c), (r_c+1, r_c+1)
+          acc01[c] = ffma2(rr.x, x.x, acc01[c]);
+          acc23[c] = ffma2(rr.x, x.y, acc23[c]);
+          if (c + 1 < C) {
+            acc01[c + 1] = ffma2(rr.y, x.x, acc01[c + 1]);
+            acc23[c + 1] = ffma2(rr.y, x.y, acc23[c + 1]);
+          }
+        }
+      }
+    }
+    if (++s == kSwStages) {
+      s = 0;
+      parity ^= 1u;
+    }
+  }
+  if (failed) {
+    // record the failure and give the requests in flight (the tile waited for and up to kSwStages - 2 after it) the
+    // same bounded time once more, so that none lands in the shared memory of a later block
+    if (t == 0) atomicOr(&P.sc->err, kErrRingWait);
+    for (int j = 0; j < kSwStages - 1 && tile < ntiles; ++j, tile += gridDim.x) {
+      ring_wait(bar_a + 8 * s, parity);
+      if (++s == kSwStages) {
+        s = 0;
+        parity ^= 1u;
+      }
+    }
+  }
+  float* gp = P.gpart + ((long long)m * gbpw + blockIdx.x) * P.ps;
+  if (owner) {
+#pragma unroll
+    for (int c = 0; c < C; ++c) {
+      float4 v;
+      unpack2(acc01[c], v.x, v.y);
+      unpack2(acc23[c], v.z, v.w);
+      *reinterpret_cast<float4*>(gp + c * F + 4 * t) = v;
+    }
+  }
+  loss = warp_sum_d(loss);
+  __syncthreads();
+  if (lane == 0) shd[w] = loss;
+  __syncthreads();
+  if (t == 0) {
+    double l = 0.0;
+    for (int j = 0; j < kSwThreads / 32; ++j) l += shd[j];
+    P.lpart[(long long)m * gbpw + blockIdx.x] = l;
+  }
+}
+
+// shapes that take the wide path: the 28 x 28 inputs and ten classes of the paper's tests
+static bool softmax_wide_path(int F, int C) { return F == 784 && C == 10; }
+
 bool softmax_classes_supported(int C) { return C >= 2 && C <= 16; }
 
 // Row tiles of the largest shard: more gradient blocks per worker than this would only write zeros.
-int grad_tiles_per_worker(int model, int F, long long n_max);
+int grad_tiles_per_worker(int model, int F, int C, long long n_max);
 
 // rows per tile: a multiple of 4 (so every tile starts 16-byte aligned), at most 160 KB of samples
 static int logreg_rows(int F) {
@@ -561,15 +795,16 @@ static size_t logreg_smem(int F) {
 }
 static size_t softmax_smem(int F, int C) { return sizeof(float) * ((size_t)kSmRows * F + (size_t)kSmRows * C); }
 
-int grad_tiles_per_worker(int model, int F, long long n_max) {
-  const long long rows = (model == LAQ_MODEL_LOGREG_BIN) ? ((F & 1) ? logreg_rows(F) : kLr2Rows) : 8;
+int grad_tiles_per_worker(int model, int F, int C, long long n_max) {
+  const long long rows = (model == LAQ_MODEL_LOGREG_BIN) ? ((F & 1) ? logreg_rows(F) : kLr2Rows)
+                                                         : (softmax_wide_path(F, C) ? kSwRows : 8);
   const long long t = (n_max + rows - 1) / rows;
   return (int)(t > 1024 ? 1024 : (t < 1 ? 1 : t));
 }
 
 // Blocks of the gradient kernel that fit on one SM (shared memory bound): the grid is sized to one such wave.
-int grad_blocks_per_sm(int model, int F) {
-  if (model != LAQ_MODEL_LOGREG_BIN) return 2;
+int grad_blocks_per_sm(int model, int F, int C) {
+  if (model != LAQ_MODEL_LOGREG_BIN) return softmax_wide_path(F, C) ? 1 : 2;
   const int fit = (int)((227 * 1024) / (logreg_smem(F) + 1024));
   return fit < 1 ? 1 : (fit > 8 ? 8 : fit);
 }
@@ -598,12 +833,25 @@ static size_t softmax_tile_smem(int F, int C) {
 template <int C>
 static void launch_sm(const Params& P, int gbpw, cudaStream_t st) {
   constexpr int CT = (C <= 12 ? C : 2);   // the tile kernel is only instantiated for C <= 12
+  if (C == 10 && softmax_wide_path(P.F, C)) {
+    constexpr int CW = (C == 10 ? 10 : 2);
+    const size_t sm = SwShape<CW, 784>::kFloats * sizeof(float);
+    cudaFuncSetAttribute(grad_softmax_wide_kernel<CW, 784>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    grad_softmax_wide_kernel<CW, 784><<<dim3(gbpw, P.M), kSwThreads, sm, st>>>(P, gbpw);
+    return;
+  }
   if (softmax_tile_path(P.F, C) && softmax_tile_smem(P.F, C) <= 112 * 1024) {
     const size_t sm = softmax_tile_smem(P.F, C);
-    cudaFuncSetAttribute(grad_softmax_tile_kernel<CT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-    cudaFuncSetAttribute(grad_softmax_tile_kernel<CT>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                         cudaSharedmemCarveoutMaxShared);  // room for two blocks per SM
-    grad_softmax_tile_kernel<CT><<<dim3(gbpw, P.M), kS2Threads, sm, st>>>(P, gbpw);
+    auto launch = [&](auto kernel) {
+      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+      cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                           cudaSharedmemCarveoutMaxShared);  // room for two blocks per SM
+      kernel<<<dim3(gbpw, P.M), kS2Threads, sm, st>>>(P, gbpw);
+    };
+    if (C == 10 && P.F == 784)
+      launch(grad_softmax_tile_kernel<CT, (C == 10 ? 784 : 0)>);
+    else
+      launch(grad_softmax_tile_kernel<CT, 0>);
     return;
   }
   const size_t sm = softmax_smem(P.F, C);

@@ -418,6 +418,10 @@ __global__ void __launch_bounds__(umma::kThreads) umma_hidden_kernel(const __gri
 //               S[c][j] = sum_r dZ[r][c] [h[r][j] > 0]   (then db1[j] = sum_c W2[c][j] S[c][j])
 //           in a fixed order (no atomics).
 constexpr int kFusedStages = 2;   // two stages of ring per block, two blocks per SM
+#ifndef LAQ_DW1_STAGES
+#define LAQ_DW1_STAGES 4
+#endif
+constexpr int kDw1Stages = LAQ_DW1_STAGES;   // ring depth of the W1-gradient product (one block per SM)
 
 __host__ __device__ inline size_t fused_extra_floats(int H) {
   return (size_t)H * 12 + (size_t)((H + 3) & ~3) + 128 * 33 + 128 * 12 + 2 * (size_t)12 * H + 16;
@@ -658,7 +662,7 @@ __global__ void __launch_bounds__(umma::kThreads) umma_dw1_kernel(const __grid_c
                                          (float)((double)n / (double)P.Ntot * (double)P.lambda), P.H, P.F, tc.i0,
                                          tc.j0, nt},
                                   nt};
-  umma::gemm_tn_tile(&tmD, &tmXT, nt, tc, &P.sc->err, epi);
+  umma::gemm_tn_tile<kDw1Stages>(&tmD, &tmXT, nt, tc, &P.sc->err, epi);
 }
 
 struct HostPlan {
@@ -811,7 +815,7 @@ laq_status mlp_setup_tensor_path(MlpPlan& mp, const Params& P, cudaStream_t st) 
   if (cudaFuncSetAttribute(umma_hidden_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)umma::smem_bytes(hp->nt1)) != cudaSuccess ||
       cudaFuncSetAttribute(umma_dw1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)umma::smem_bytes(hp->nt2)) != cudaSuccess ||
+                           (int)umma::smem_bytes(hp->nt2, kDw1Stages)) != cudaSuccess ||
       cudaFuncSetAttribute(mlp_forward_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)forward_smem_tc(P.H)) != cudaSuccess) {
     cudaGetLastError();
@@ -853,7 +857,7 @@ int mlp_launch_gradients(MlpPlan& mp, const Params& P, const double* theta_sq, c
                                  umma::smem_bytes(hp->nt1, kFusedStages), st>>>(hp->tmX, hp->tmW, P, hp->d,
                                                                                               hp->nt1);
       umma_dw1_kernel<<<dim3((F + hp->nt2 - 1) / hp->nt2, (H + umma::kTileM - 1) / umma::kTileM, P.M), umma::kThreads,
-                        umma::smem_bytes(hp->nt2), st>>>(hp->tmD, hp->tmXT, P, hp->d, hp->nt2);
+                        umma::smem_bytes(hp->nt2, kDw1Stages), st>>>(hp->tmD, hp->tmXT, P, hp->d, hp->nt2);
       mlp_finalize_kernel<<<dim3((nsmall + 255) / 256, P.M), 256, 0, st>>>(P, hp->d, theta_sq);
       return 4;
     }
@@ -861,7 +865,7 @@ int mlp_launch_gradients(MlpPlan& mp, const Params& P, const double* theta_sq, c
                          umma::smem_bytes(hp->nt1), st>>>(hp->tmX, hp->tmW, P, hp->d, hp->nt1);
     mlp_forward_kernel<true><<<dim3(hp->d.gb, P.M), kThreads, forward_smem_tc(H), st>>>(P, hp->d);
     umma_dw1_kernel<<<dim3((F + hp->nt2 - 1) / hp->nt2, (H + umma::kTileM - 1) / umma::kTileM, P.M), umma::kThreads,
-                      umma::smem_bytes(hp->nt2), st>>>(hp->tmD, hp->tmXT, P, hp->d, hp->nt2);
+                      umma::smem_bytes(hp->nt2, kDw1Stages), st>>>(hp->tmD, hp->tmXT, P, hp->d, hp->nt2);
     mlp_finalize_kernel<<<dim3((nsmall + 255) / 256, P.M), 256, 0, st>>>(P, hp->d, theta_sq);
     return 5;
   }

@@ -91,6 +91,52 @@ __device__ __forceinline__ uint32_t fmix32(uint32_t x) {
   return x;
 }
 
+// ---- bulk asynchronous copies global -> shared, completion counted in bytes on an mbarrier ---------------------
+// Source, destination and size are multiples of 16 bytes.  Every wait is bounded: after kRingWaitLimit polls it
+// returns false; the caller records kErrRingWait in DevScalars::err, stops using the ring, and gives the copies
+// still in flight the same bounded time to land before it leaves.
+constexpr uint32_t kRingWaitLimit = 1u << 22;
+constexpr uint32_t kErrRingWait = 16u;             // bit of DevScalars::err: a wait on a staged tile ran out
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void ring_bar_init(uint32_t bar) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void ring_expect(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void ring_copy(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+// one copy that is the whole content of a stage
+__device__ __forceinline__ void ring_fetch(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  ring_expect(bar, bytes);
+  ring_copy(dst, src, bytes, bar);
+}
+__device__ __forceinline__ bool ring_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded: false once the limit is reached (the caller records it and stops using the ring).
+__device__ __forceinline__ bool ring_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t it = 0; it < kRingWaitLimit; ++it) {
+    if (ring_try_wait(bar, parity)) return true;
+    if (it > 64) __nanosleep(64);
+  }
+  return false;
+}
+
 // Rows of worker m that enter the local gradient of the iteration in progress: all N_m rows, or (minibatch
 // variant of Sec. 4) the cyclic window of B_m = min(batch, N_m) consecutive rows whose start is drawn from
 // (seed, m, k): rows [start, start + len_a) followed by rows [0, len_b).
@@ -163,8 +209,8 @@ int launch_grad_logreg(const Params& P, const LaunchShape& ls, int gbpw, cudaStr
 int launch_grad_softmax(const Params& P, const LaunchShape& ls, int gbpw, cudaStream_t st);
 int launch_grad_finalize(const Params& P, int gbpw, const double* theta_sq, cudaStream_t st);
 bool softmax_classes_supported(int C);
-int grad_tiles_per_worker(int model, int F, long long n_max);
-int grad_blocks_per_sm(int model, int F);
+int grad_tiles_per_worker(int model, int F, int C, long long n_max);
+int grad_blocks_per_sm(int model, int F, int C);
 
 // one-hidden-layer ReLU network (laq_grad_mlp.cu)
 struct MlpPlan {

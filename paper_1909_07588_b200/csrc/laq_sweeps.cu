@@ -440,40 +440,6 @@ constexpr int kRingStages = LAQ_RING_STAGES;
 constexpr int kRingU = LAQ_RING_U;                 // groups per lane and tile
 constexpr uint32_t kRingGroups = 32 * kRingU;      // 16-byte groups per tile (4 KB)
 constexpr int kRingMaxWarps = 16;                  // warps per block that can own a ring
-constexpr uint32_t kRingWaitLimit = 1u << 22;
-constexpr uint32_t kErrRingWait = 16u;             // bit of DevScalars::err: a wait on a staged tile ran out
-
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void ring_bar_init(uint32_t bar) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void ring_fetch(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
-}
-__device__ __forceinline__ bool ring_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n"
-      "}\n"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded: false once the limit is reached (the caller records it and stops using the ring).
-__device__ __forceinline__ bool ring_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t it = 0; it < kRingWaitLimit; ++it) {
-    if (ring_try_wait(bar, parity)) return true;
-    if (it > 64) __nanosleep(64);
-  }
-  return false;
-}
 
 // The per-worker sweep of quantize_kernel (R > 0).  FAST selects the reciprocal-based exact division.
 // Groups [0, nv_main) lie wholly inside the row and run without masks; the few groups after them are
