@@ -213,6 +213,22 @@ def test_synthetic_stream_bit_exact(b, M, p):
     ctx.close()
 
 
+@pytest.mark.parametrize("b,M,p", [(1, 5, 70001), (16, 5, 70001), (8, 4, 1), (8, 3, 100), (4, 6, 4095), (8, 6, 4100),
+                                   (3, 4, 8191), (2, 2, 300_001)])
+def test_synthetic_stream_short_rows_and_all_code_widths(b, M, p):
+    """Rows shorter than one staged tile (the plain loop and the masked tail do all the work), rows of a few tiles
+    with a ragged rest, and the code widths the other synthetic cases leave out."""
+    iters = 12
+    w = workloads.c4(M=M, p=p, b=b, iters=iters)
+    ctx = laq.from_workload(w, trace_capacity=iters)
+    mir = _mirror_for(w)
+    tr = ctx.step(iters, trace=True)
+    for j in range(iters):
+        _assert_trace_row(tr, j, mir.step())
+    _assert_state_bit_exact(ctx.get_state(codes=True), mir.state(), p, b)
+    ctx.close()
+
+
 def test_synthetic_full_size_sampled_workers():
     """The benchmark's launch configuration (M = 64, p = 25.6 M, b = 8): worker messages of the first
     iteration against the mirror for sampled workers, the aggregate invariant, and the clock rules."""
@@ -404,6 +420,22 @@ def test_c1_shape_softmax_reduced():
     w = workloads.c1(n_per=333, iters=40)
     first = _run_model_parity(w, w.iters)
     assert first is None or first > 3
+
+
+def test_c1_full_size_first_iterations():
+    """The benchmark's own shape and launch configuration (10 x 6000 rows, 784 features, 10 classes)."""
+    w = workloads.c1(iters=3)
+    _run_model_parity(w, 3)
+
+
+def test_c2_full_size_first_iterations():
+    w = workloads.c2(iters=4, theta0_scale=0.01)
+    _run_model_parity(w, 4)
+
+
+def test_c3_full_size_first_iterations():
+    w = workloads.c3(iters=2)
+    _run_model_parity(w, 2)
 
 
 def test_softmax_small_odd_shapes():
