@@ -24,16 +24,6 @@ __device__ __forceinline__ float warp_sum_f(float v) {
   return v;
 }
 
-// Packed fp32 pairs: sm_100 executes two fused multiply-adds per lane in one instruction.
-__device__ __forceinline__ unsigned long long ffma2(unsigned long long a, unsigned long long b, unsigned long long c) {
-  unsigned long long d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-
 // Copy `count` consecutive floats global -> shared; where alignment allows as asynchronous 16-byte copies, so
 // that every thread has all of its copies in flight at once.  Ends with the copies complete for this thread;
 // the caller's __syncthreads() makes them visible to the block.

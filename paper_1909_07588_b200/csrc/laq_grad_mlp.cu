@@ -459,9 +459,10 @@ struct FusedEpi {
     const bool valid = trow < n && win.contains(trow);
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
     // ---- pass 1
-    float z[12];
+    // scores as packed pairs of classes: z2[k] = (z[2k], z[2k+1]), one packed multiply-add per pair and hidden unit
+    unsigned long long z2[6];
 #pragma unroll
-    for (int c = 0; c < 12; ++c) z[c] = 0.f;
+    for (int c = 0; c < 6; ++c) z2[c] = 0ull;
     for (int c0 = 0; c0 < nt; c0 += 32) {
       uint32_t v[32];
       umma::tmem_load_32(taddr + (uint32_t)c0, v);
@@ -470,15 +471,19 @@ struct FusedEpi {
         const int j = c0 + i;
         if (j < H) {
           const float h = fmaxf(__uint_as_float(v[i]) + b1s[j], 0.f);
-          const float4 wa = *reinterpret_cast<const float4*>(w2t + j * 12);
-          const float4 wb = *reinterpret_cast<const float4*>(w2t + j * 12 + 4);
-          const float4 wc = *reinterpret_cast<const float4*>(w2t + j * 12 + 8);
-          z[0] = fmaf(h, wa.x, z[0]); z[1] = fmaf(h, wa.y, z[1]); z[2] = fmaf(h, wa.z, z[2]); z[3] = fmaf(h, wa.w, z[3]);
-          z[4] = fmaf(h, wb.x, z[4]); z[5] = fmaf(h, wb.y, z[5]); z[6] = fmaf(h, wb.z, z[6]); z[7] = fmaf(h, wb.w, z[7]);
-          z[8] = fmaf(h, wc.x, z[8]); z[9] = fmaf(h, wc.y, z[9]); z[10] = fmaf(h, wc.z, z[10]); z[11] = fmaf(h, wc.w, z[11]);
+          const unsigned long long hh = pack2(h, h);
+          const ulonglong2 wa = *reinterpret_cast<const ulonglong2*>(w2t + j * 12);
+          const ulonglong2 wb = *reinterpret_cast<const ulonglong2*>(w2t + j * 12 + 4);
+          const ulonglong2 wc = *reinterpret_cast<const ulonglong2*>(w2t + j * 12 + 8);
+          z2[0] = ffma2(hh, wa.x, z2[0]); z2[1] = ffma2(hh, wa.y, z2[1]);
+          z2[2] = ffma2(hh, wb.x, z2[2]); z2[3] = ffma2(hh, wb.y, z2[3]);
+          z2[4] = ffma2(hh, wc.x, z2[4]); z2[5] = ffma2(hh, wc.y, z2[5]);
         }
       }
     }
+    float z[12];
+#pragma unroll
+    for (int c = 0; c < 6; ++c) unpack2(z2[c], z[2 * c], z[2 * c + 1]);
     float dz[12];
     double loss = 0.0;
     {
@@ -507,6 +512,9 @@ struct FusedEpi {
       if (valid) loss = (double)((zmax + logf(sum)) - zy);
     }
     // ---- pass 2
+    unsigned long long dz2[6];
+#pragma unroll
+    for (int c = 0; c < 6; ++c) dz2[c] = pack2(dz[2 * c], dz[2 * c + 1]);
     const long long col = D.rowoffT[m] + trow;
     const bool in_segment = col < D.rowoffT[m + 1];        // rows of the padded segment (zeros beyond the shard)
     const int rq = tt >> 5, cl = tt & 31;                  // reduce phase: column cl, rows 32 rq .. 32 rq + 31
@@ -519,13 +527,16 @@ struct FusedEpi {
         float h = 0.f;
         if (j < H) {
           h = fmaxf(__uint_as_float(v[i]) + b1s[j], 0.f);
-          const float4 wa = *reinterpret_cast<const float4*>(w2t + j * 12);
-          const float4 wb = *reinterpret_cast<const float4*>(w2t + j * 12 + 4);
-          const float4 wc = *reinterpret_cast<const float4*>(w2t + j * 12 + 8);
-          float d = dz[0] * wa.x;
-          d = fmaf(dz[1], wa.y, d); d = fmaf(dz[2], wa.z, d); d = fmaf(dz[3], wa.w, d);
-          d = fmaf(dz[4], wb.x, d); d = fmaf(dz[5], wb.y, d); d = fmaf(dz[6], wb.z, d); d = fmaf(dz[7], wb.w, d);
-          d = fmaf(dz[8], wc.x, d); d = fmaf(dz[9], wc.y, d); d = fmaf(dz[10], wc.z, d); d = fmaf(dz[11], wc.w, d);
+          const ulonglong2 wa = *reinterpret_cast<const ulonglong2*>(w2t + j * 12);
+          const ulonglong2 wb = *reinterpret_cast<const ulonglong2*>(w2t + j * 12 + 4);
+          const ulonglong2 wc = *reinterpret_cast<const ulonglong2*>(w2t + j * 12 + 8);
+          // even and odd classes in the two halves of a packed sum, added at the end
+          unsigned long long d2 = ffma2(dz2[0], wa.x, 0ull);
+          d2 = ffma2(dz2[1], wa.y, d2); d2 = ffma2(dz2[2], wb.x, d2); d2 = ffma2(dz2[3], wb.y, d2);
+          d2 = ffma2(dz2[4], wc.x, d2); d2 = ffma2(dz2[5], wc.y, d2);
+          float d_even, d_odd;
+          unpack2(d2, d_even, d_odd);
+          const float d = d_even + d_odd;
           const float dh = h > 0.f ? d : 0.f;
           if (in_segment) D.dHT[(long long)j * D.ldT + col] = __float2bfloat16_rn(dh);
         }
@@ -533,21 +544,27 @@ struct FusedEpi {
       }
       umma::epilogue_sync();
       {  // column sums over this thread's 32 rows
-        float a[12], sgn[12];
+        unsigned long long a2[6], s2[6];    // packed pairs of classes
 #pragma unroll
-        for (int c = 0; c < 12; ++c) a[c] = sgn[c] = 0.f;
+        for (int c = 0; c < 6; ++c) a2[c] = s2[c] = 0ull;
+#pragma unroll 4
         for (int r = 32 * rq; r < 32 * rq + 32; ++r) {
           const float h = chunk[r * 33 + cl];
           const float pos = h > 0.f ? 1.f : 0.f;
-          const float4 da = *reinterpret_cast<const float4*>(dzs + r * 12);
-          const float4 db = *reinterpret_cast<const float4*>(dzs + r * 12 + 4);
-          const float4 dc = *reinterpret_cast<const float4*>(dzs + r * 12 + 8);
-          const float dv[12] = {da.x, da.y, da.z, da.w, db.x, db.y, db.z, db.w, dc.x, dc.y, dc.z, dc.w};
+          const unsigned long long hh = pack2(h, h), pp = pack2(pos, pos);
+          const ulonglong2 da = *reinterpret_cast<const ulonglong2*>(dzs + r * 12);
+          const ulonglong2 db = *reinterpret_cast<const ulonglong2*>(dzs + r * 12 + 4);
+          const ulonglong2 dc = *reinterpret_cast<const ulonglong2*>(dzs + r * 12 + 8);
+          a2[0] = ffma2(da.x, hh, a2[0]); a2[1] = ffma2(da.y, hh, a2[1]); a2[2] = ffma2(db.x, hh, a2[2]);
+          a2[3] = ffma2(db.y, hh, a2[3]); a2[4] = ffma2(dc.x, hh, a2[4]); a2[5] = ffma2(dc.y, hh, a2[5]);
+          s2[0] = ffma2(da.x, pp, s2[0]); s2[1] = ffma2(da.y, pp, s2[1]); s2[2] = ffma2(db.x, pp, s2[2]);
+          s2[3] = ffma2(db.y, pp, s2[3]); s2[4] = ffma2(dc.x, pp, s2[4]); s2[5] = ffma2(dc.y, pp, s2[5]);
+        }
+        float a[12], sgn[12];
 #pragma unroll
-          for (int c = 0; c < 12; ++c) {
-            a[c] = fmaf(dv[c], h, a[c]);
-            sgn[c] = fmaf(dv[c], pos, sgn[c]);
-          }
+        for (int c = 0; c < 6; ++c) {
+          unpack2(a2[c], a[2 * c], a[2 * c + 1]);
+          unpack2(s2[c], sgn[2 * c], sgn[2 * c + 1]);
         }
         umma::epilogue_sync();      // everybody has read the chunk: reuse it for the partial sums
 #pragma unroll

@@ -91,6 +91,21 @@ __device__ __forceinline__ uint32_t fmix32(uint32_t x) {
   return x;
 }
 
+// Packed fp32 pairs: sm_100 executes two fused multiply-adds per lane in one instruction.
+__device__ __forceinline__ unsigned long long ffma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+  unsigned long long v;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+  return v;
+}
+
 // ---- bulk asynchronous copies global -> shared, completion counted in bytes on an mbarrier ---------------------
 // Source, destination and size are multiples of 16 bytes.  Every wait is bounded: after kRingWaitLimit polls it
 // returns false; the caller records kErrRingWait in DevScalars::err, stops using the ring, and gives the copies
