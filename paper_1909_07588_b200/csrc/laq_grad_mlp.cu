@@ -417,53 +417,67 @@ __global__ void __launch_bounds__(umma::kThreads) umma_hidden_kernel(const __gri
 //               A[c][j] = sum_r dZ[r][c] h[r][j]         (the W2 gradient)
 //               S[c][j] = sum_r dZ[r][c] [h[r][j] > 0]   (then db1[j] = sum_c W2[c][j] S[c][j])
 //           in a fixed order (no atomics).
+// Eight epilogue warps: two sets of four, each set taking every other 32-column chunk in both passes.
 constexpr int kFusedStages = 2;   // two stages of ring per block, two blocks per SM
 #ifndef LAQ_DW1_STAGES
 #define LAQ_DW1_STAGES 4
 #endif
 constexpr int kDw1Stages = LAQ_DW1_STAGES;   // ring depth of the W1-gradient product (one block per SM)
 
+constexpr int kFusedEpiWarps = 8;                      // two sets of four epilogue warps
+constexpr int kFusedThreads = 64 + 32 * kFusedEpiWarps;
+
 __host__ __device__ inline size_t fused_extra_floats(int H) {
-  return (size_t)H * 12 + (size_t)((H + 3) & ~3) + 128 * 33 + 128 * 12 + 2 * (size_t)12 * H + 16;
+  return (size_t)H * 12 + (size_t)((H + 3) & ~3) + 2 * 128 * 33 + 128 * 12 + 2 * (size_t)12 * H + 16;
 }
 
+// Both sets of epilogue warps own all 128 rows (thread = row) and share the 32-column chunks of the accumulator
+// between them: set 0 takes chunks 0, 2, 4, ..., set 1 chunks 1, 3, 5, ...  The scores are the sum of the two sets'
+// partial scores (set 0's first); every later step is per column, so the sets only meet at three block-wide points.
 struct FusedEpi {
   const Params& P;
   const MlpDev& D;
   int nt, m, tile;          // worker and tile index within the worker
   RowWindow win;            // rows of the worker that enter this iteration's gradient
-  __device__ __forceinline__ void run(uint32_t tmem_base, int q, int lane) {
+  static __device__ __forceinline__ void sync_all() { umma::named_sync<1, 32 * kFusedEpiWarps>(); }
+  static __device__ __forceinline__ void sync_set(int set) {
+    if (set == 0) umma::named_sync<2, 128>(); else umma::named_sync<3, 128>();
+  }
+  __device__ __forceinline__ void run(uint32_t tmem_base, int q, int lane, int set) {
     const int H = P.H, C = P.C, F = P.F;
     const int tt = q * 32 + lane;            // 0..127: the tile row this thread owns
+    const int et = set * 128 + tt;           // 0..255 among the epilogue threads
     float* base = reinterpret_cast<float*>(umma::ring_smem());   // the ring is free once the accumulator is complete
     float* w2t = base;                       // [H][12]   W2 transposed (j-major), padded rows of 12
     float* b1s = w2t + (size_t)H * 12;       // [H]
-    float* chunk = b1s + ((H + 3) & ~3);     // [128][33] one 32-column chunk of h
-    float* dzs = chunk + 128 * 33;           // [128][12]
+    float* chunks = b1s + ((H + 3) & ~3);    // [2][128][33] one 32-column chunk of h per set
+    float* dzs = chunks + 2 * 128 * 33;      // [128][12]
     float* accA = dzs + 128 * 12;            // [12][H]
     float* accS = accA + (size_t)12 * H;     // [12][H]
     double* lossw = reinterpret_cast<double*>(accS + (size_t)12 * H);      // [4] (8-byte aligned: all sizes even)
+    float* chunk = chunks + set * 128 * 33;  // this set's chunk buffer
     float* red = chunk;                      // [4][2 C][32] partial column sums, reuses the chunk buffer
+    float* zpart = chunks;                   // [2][128][12] partial scores of the two sets, before the chunks are used
     const float* __restrict__ theta = P.theta;
     const float* __restrict__ b1 = theta + (long long)H * F;
     const float* __restrict__ W2 = b1 + H;
     const float* __restrict__ b2 = W2 + (long long)C * H;
-    for (int i = tt; i < H * 12; i += 128) {
+    for (int i = et; i < H * 12; i += 256) {
       const int j = i / 12, c = i - 12 * j;
       w2t[i] = (c < C) ? __ldg(W2 + (size_t)c * H + j) : 0.f;
     }
-    for (int i = tt; i < H; i += 128) b1s[i] = __ldg(b1 + i);
-    umma::epilogue_sync();
+    for (int i = et; i < H; i += 256) b1s[i] = __ldg(b1 + i);
     const long long n = P.N[m];
     const long long trow = (long long)tile * umma::kTileM + tt;   // row within the worker's shard
     const bool valid = trow < n && win.contains(trow);
+    const int yv = valid ? __ldg(P.y[m] + trow) : -1;             // asked for now, used after the first pass
+    sync_all();
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-    // ---- pass 1
-    // scores as packed pairs of classes: z2[k] = (z[2k], z[2k+1]), one packed multiply-add per pair and hidden unit
+    // ---- pass 1: partial scores over this set's chunks, as packed pairs of classes z2[k] = (z[2k], z[2k+1])
     unsigned long long z2[6];
 #pragma unroll
     for (int c = 0; c < 6; ++c) z2[c] = 0ull;
-    for (int c0 = 0; c0 < nt; c0 += 32) {
+    for (int c0 = 32 * set; c0 < nt; c0 += 64) {
       uint32_t v[32];
       umma::tmem_load_32(taddr + (uint32_t)c0, v);
 #pragma unroll
@@ -481,12 +495,19 @@ struct FusedEpi {
         }
       }
     }
-    float z[12];
-#pragma unroll
-    for (int c = 0; c < 6; ++c) unpack2(z2[c], z[2 * c], z[2 * c + 1]);
+    {
+      ulonglong2* zp = reinterpret_cast<ulonglong2*>(zpart + (set * 128 + tt) * 12);
+      zp[0] = make_ulonglong2(z2[0], z2[1]);
+      zp[1] = make_ulonglong2(z2[2], z2[3]);
+      zp[2] = make_ulonglong2(z2[4], z2[5]);
+    }
+    sync_all();
     float dz[12];
     double loss = 0.0;
-    {
+    {  // both sets do the softmax of the row (the same arithmetic), set 0 keeps the loss and publishes dZ
+      float z[12];
+#pragma unroll
+      for (int c = 0; c < 12; ++c) z[c] = zpart[tt * 12 + c] + zpart[(128 + tt) * 12 + c];
       float zmax = -3.0e38f;
 #pragma unroll
       for (int c = 0; c < 12; ++c)
@@ -500,17 +521,17 @@ struct FusedEpi {
         e[c] = (c < C) ? expf(z[c] - zmax) : 0.f;
         sum += e[c];
       }
-      const int yv = valid ? P.y[m][trow] : -1;
       const float inv = 1.0f / sum;
       float zy = 0.f;
 #pragma unroll
       for (int c = 0; c < 12; ++c) {
         if (c == yv) zy = z[c];
         dz[c] = (valid && c < C) ? (e[c] * inv - (c == yv ? 1.f : 0.f)) : 0.f;
-        dzs[tt * 12 + c] = dz[c];
+        if (set == 0) dzs[tt * 12 + c] = dz[c];
       }
-      if (valid) loss = (double)((zmax + logf(sum)) - zy);
+      if (valid && set == 0) loss = (double)((zmax + logf(sum)) - zy);
     }
+    sync_all();   // dZ is published; nobody reads the partial scores any more (the chunk buffers take their place)
     // ---- pass 2
     unsigned long long dz2[6];
 #pragma unroll
@@ -518,7 +539,7 @@ struct FusedEpi {
     const long long col = D.rowoffT[m] + trow;
     const bool in_segment = col < D.rowoffT[m + 1];        // rows of the padded segment (zeros beyond the shard)
     const int rq = tt >> 5, cl = tt & 31;                  // reduce phase: column cl, rows 32 rq .. 32 rq + 31
-    for (int c0 = 0; c0 < nt; c0 += 32) {
+    for (int c0 = 32 * set; c0 < nt; c0 += 64) {
       uint32_t v[32];
       umma::tmem_load_32(taddr + (uint32_t)c0, v);
 #pragma unroll
@@ -542,7 +563,7 @@ struct FusedEpi {
         }
         chunk[tt * 33 + i] = h;
       }
-      umma::epilogue_sync();
+      sync_set(set);
       {  // column sums over this thread's 32 rows
         unsigned long long a2[6], s2[6];    // packed pairs of classes
 #pragma unroll
@@ -566,14 +587,14 @@ struct FusedEpi {
           unpack2(a2[c], a[2 * c], a[2 * c + 1]);
           unpack2(s2[c], sgn[2 * c], sgn[2 * c + 1]);
         }
-        umma::epilogue_sync();      // everybody has read the chunk: reuse it for the partial sums
+        sync_set(set);              // the set has read the chunk: reuse it for the partial sums
 #pragma unroll
         for (int c = 0; c < 12; ++c) {
           red[(rq * 24 + c) * 32 + cl] = a[c];
           red[(rq * 24 + 12 + c) * 32 + cl] = sgn[c];
         }
       }
-      umma::epilogue_sync();
+      sync_set(set);
       for (int i = tt; i < 24 * 32; i += 128) {   // fixed order over the four row quarters
         const int k = i >> 5, cc = i & 31, j = c0 + cc;
         if (j < H) {
@@ -582,32 +603,32 @@ struct FusedEpi {
           if (k < 12) accA[k * H + j] = sum4; else accS[(k - 12) * H + j] = sum4;
         }
       }
-      umma::epilogue_sync();
+      sync_set(set);
     }
     // ---- the tile's partials: [db1 (H) | dW2 (C H) | db2 (C)] and the loss
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, o);
+    if (lane == 0 && set == 0) lossw[q] = loss;
+    sync_all();
     const int gb = D.gb;
     float* sp = D.spart + ((long long)m * gb + tile) * (H + C * H + C);
-    for (int j = tt; j < H; j += 128) {
+    for (int j = et; j < H; j += 256) {
       float s = 0.f;
       for (int c = 0; c < C; ++c) s = fmaf(w2t[j * 12 + c], accS[c * H + j], s);
       sp[j] = s;
       for (int c = 0; c < C; ++c) sp[H + c * H + j] = accA[c * H + j];
     }
-    if (tt < C) {
+    if (set == 1 && tt < C) {
       float s = 0.f;
       for (int r = 0; r < 128; ++r) s += dzs[r * 12 + tt];
       sp[H + C * H + tt] = s;
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, o);
-    if (lane == 0) lossw[q] = loss;
-    umma::epilogue_sync();
-    if (tt == 0) D.lpart[(long long)m * gb + tile] = ((lossw[0] + lossw[1]) + lossw[2]) + lossw[3];
+    if (et == 0) D.lpart[(long long)m * gb + tile] = ((lossw[0] + lossw[1]) + lossw[2]) + lossw[3];
   }
 };
 
 // grid: (tiles per worker, M); tile t of worker m covers the worker's rows 128 t .. 128 t + 127
-__global__ void __launch_bounds__(umma::kThreads, 2) umma_hidden_fused_kernel(const __grid_constant__ CUtensorMap tmX,
+__global__ void __launch_bounds__(kFusedThreads, 2) umma_hidden_fused_kernel(const __grid_constant__ CUtensorMap tmX,
                                                                            const __grid_constant__ CUtensorMap tmW,
                                                                            const Params P, const MlpDev D, int nt) {
   const int m = blockIdx.y, tile = blockIdx.x;
@@ -626,7 +647,7 @@ __global__ void __launch_bounds__(umma::kThreads, 2) umma_hidden_fused_kernel(co
     return;
   }
   FusedEpi epi{P, D, nt, m, tile, win};
-  umma::gemm_tn_tile<kFusedStages>(&tmX, &tmW, nt, tc, &P.sc->err, epi);
+  umma::gemm_tn_tile<kFusedStages, kFusedEpiWarps>(&tmX, &tmW, nt, tc, &P.sc->err, epi);
 }
 
 struct Dw1Epi {
@@ -870,7 +891,7 @@ int mlp_launch_gradients(MlpPlan& mp, const Params& P, const double* theta_sq, c
   if (hp->tc) {
     mlp_pack_w1b_kernel<<<(F * H + 255) / 256, 256, 0, st>>>(P.theta, hp->d.W1b, F * H);
     if (hp->fused_tiles > 0) {
-      umma_hidden_fused_kernel<<<dim3(hp->fused_tiles, P.M), umma::kThreads,
+      umma_hidden_fused_kernel<<<dim3(hp->fused_tiles, P.M), kFusedThreads,
                                  umma::smem_bytes(hp->nt1, kFusedStages), st>>>(hp->tmX, hp->tmW, P, hp->d,
                                                                                               hp->nt1);
       umma_dw1_kernel<<<dim3((F + hp->nt2 - 1) / hp->nt2, (H + umma::kTileM - 1) / umma::kTileM, P.M), umma::kThreads,

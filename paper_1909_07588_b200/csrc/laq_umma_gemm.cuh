@@ -123,10 +123,17 @@ struct TileCoord {
   }
 };
 
-// Epi::run(tmem_base, q, lane) is executed by the four epilogue warps once the accumulator is complete; warp
+// Epi::run(tmem_base, q, lane, set) is executed by the epilogue warps once the accumulator is complete; warp
 // quarter q (0..3) may read TMEM lanes 32 q .. 32 q + 31, i.e. accumulator rows 32 q + lane.  The epilogue warps
-// are threads 64..191 of the block; they may synchronise among themselves with named barrier 1 (128 threads).
+// are threads 64.. of the block: four of them (EPI_WARPS = 4, set = 0), or eight (EPI_WARPS = 8: two sets of four,
+// set = 0 or 1, both sets see all rows and may share the columns between them).  They may synchronise among
+// themselves with named barrier 1 over 32 EPI_WARPS threads.
 __device__ __forceinline__ void epilogue_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// Named barrier ID (1..15) over COUNT threads (a multiple of 32); every participating warp names the same count.
+template <int ID, int COUNT>
+__device__ __forceinline__ void named_sync() {
+  asm volatile("bar.sync %0, %1;" ::"n"(ID), "n"(COUNT) : "memory");
+}
 
 // Shared memory that follows the stage ring (for an epilogue's own buffers); pass the extra bytes at launch.
 __device__ __forceinline__ unsigned char* extra_smem(int nt) {
@@ -152,7 +159,7 @@ template <class F>
 struct ChunkEpilogue {
   F f;
   int nt;
-  __device__ __forceinline__ void run(uint32_t tmem_base, int q, int lane) {
+  __device__ __forceinline__ void run(uint32_t tmem_base, int q, int lane, int /*set*/) {
     for (int c0 = 0; c0 < nt; c0 += 32) {
       uint32_t v[32];
       tmem_load_32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
@@ -164,7 +171,7 @@ struct ChunkEpilogue {
   }
 };
 
-template <int STAGES = kStages, class Epi>
+template <int STAGES = kStages, int EPI_WARPS = 4, class Epi>
 __device__ __forceinline__ void gemm_tn_tile(const CUtensorMap* tmA, const CUtensorMap* tmB, int nt, TileCoord tc,
                                              uint32_t* err_flag, Epi& epi) {
   extern __shared__ unsigned char umma_smem_raw[];
@@ -227,12 +234,15 @@ __device__ __forceinline__ void gemm_tn_tile(const CUtensorMap* tmA, const CUten
     const int q = warp & 3;                         // the TMEM lane quarter this warp may read
     const bool ok = __all_sync(0xffffffffu, mbar_wait(accum, 0u, err_flag, 8u));
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    // all four epilogue warps take the same branch (the verdicts are combined), so an epilogue may use
-    // its named barrier
-    __shared__ int epi_ok[4];
-    if (lane == 0) epi_ok[q] = (ok && tc.nkb > 0) ? 1 : 0;
-    epilogue_sync();
-    if (epi_ok[0] & epi_ok[1] & epi_ok[2] & epi_ok[3]) epi.run(tmem_base, q, lane);
+    // all epilogue warps take the same branch (the verdicts are combined), so an epilogue may use
+    // its named barriers
+    __shared__ int epi_ok[EPI_WARPS];
+    if (lane == 0) epi_ok[warp - 2] = (ok && tc.nkb > 0) ? 1 : 0;
+    named_sync<1, 32 * EPI_WARPS>();
+    int all_ok = 1;
+#pragma unroll
+    for (int e = 0; e < EPI_WARPS; ++e) all_ok &= epi_ok[e];
+    if (all_ok) epi.run(tmem_base, q, lane, (warp - 2) >> 2);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
