@@ -169,7 +169,10 @@ laq_status laq_set_gradients(laq_ctx* ctx, const float* g, int32_t on_device);
 
 /* Run n_iters iterations of Algorithm 2 (for EXTERNAL: n_iters must be 1).  With trace == NULL the
  * call only enqueues work on the stream and returns.  With a trace (n_iters <= trace_capacity) it
- * synchronises once at the end, fills the HOST arrays and reports device-detected errors. */
+ * synchronises once at the end, fills the HOST arrays and reports device-detected errors.
+ * Calls of four or more iterations replay the iteration's kernels as CUDA graphs (captured once per context on
+ * a stream of the library's own, launched into the context's stream; plain launches if capture is not possible,
+ * while per-stage timing is on, or after laq_tune(ctx, "graphs", 0)). */
 laq_status laq_step(laq_ctx* ctx, int32_t n_iters, const laq_trace* trace);
 
 /* Wait for the stream and report device-detected errors. */
@@ -190,8 +193,9 @@ laq_status laq_set_state(laq_ctx* ctx, const laq_state* in);
 int64_t laq_kernel_launches(const laq_ctx* ctx);
 
 /* Launch-shape override for measurement sweeps: key "sweep_threads", "sweep_blocks_per_sm",
- * "agg_threads", "agg_blocks_per_sm", "grad_blocks_per_worker".  Values outside the documented
- * limits return LAQ_EINVAL and change nothing. */
+ * "agg_threads", "agg_blocks_per_sm", "grad_blocks_per_worker", and "graphs" (0: laq_step uses plain launches
+ * only; 1, the default: graph replay).  Values outside the documented limits return LAQ_EINVAL and change
+ * nothing. */
 laq_status laq_tune(laq_ctx* ctx, const char* key, int32_t value);
 
 /* Per-kernel device timing for measurement.  While enabled, laq_step brackets every stage of an iteration

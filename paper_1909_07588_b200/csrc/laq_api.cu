@@ -35,6 +35,11 @@ struct laq_ctx {
   int ev_used = 0;                    // iterations recorded and not yet read
   double stage_ms[4] = {0, 0, 0, 0};
   int64_t stage_launches[4] = {0, 0, 0, 0};
+  // the kernels of one iteration (and of kGraphIters iterations) as executable graphs, replayed by laq_step
+  bool graphs_enabled = true, graphs_failed = false;
+  cudaStream_t cap_stream = nullptr;   // capture happens here, never on the caller's stream
+  cudaGraphExec_t graph_one = nullptr, graph_many = nullptr;
+  int64_t launches_per_iter = 0;
 };
 
 namespace {
@@ -219,6 +224,109 @@ double host_sum_sq(const float* v, long long n) {
 
 }  // namespace
 
+namespace {
+
+constexpr int kGraphIters = 8;       // iterations per replay of the larger graph
+constexpr int kGraphMinIters = 4;    // shorter calls go out as plain launches
+
+// The kernels of one iteration on stream st; ev (5 events) brackets the four stages when profiling.
+void enqueue_iteration(laq_ctx* ctx, cudaStream_t st, cudaEvent_t* ev) {
+  const laq_config& c = ctx->cfg;
+  const Params& P = ctx->P;
+  if (ev) cudaEventRecord(ev[0], st);
+  const int64_t l0 = ctx->launches;
+  // small problems: steps 2-5 (and, when cheap, the combination of the gradient kernels' block partials)
+  // run in one single-block kernel
+  const bool small = small_iteration_applies(P);
+  const bool linear = c.model == LAQ_MODEL_LOGREG_BIN || c.model == LAQ_MODEL_SOFTMAX;
+  const bool fuse_finalize = small && linear && ctx->gbpw <= 64;
+  switch (c.model) {
+    case LAQ_MODEL_LOGREG_BIN:
+      ctx->launches += launch_grad_logreg(P, ctx->ls, ctx->gbpw, st);
+      if (!fuse_finalize) ctx->launches += launch_grad_finalize(P, ctx->gbpw, &P.sc->theta_sq, st);
+      break;
+    case LAQ_MODEL_SOFTMAX:
+      ctx->launches += launch_grad_softmax(P, ctx->ls, ctx->gbpw, st);
+      if (!fuse_finalize) ctx->launches += launch_grad_finalize(P, ctx->gbpw, &P.sc->theta_sq, st);
+      break;
+    case LAQ_MODEL_MLP2:
+      ctx->launches += mlp_launch_gradients(ctx->mlp, P, &P.sc->theta_sq, st);
+      break;
+    default: break;
+  }
+  if (ev) {
+    cudaEventRecord(ev[1], st);
+    ctx->stage_launches[0] += ctx->launches - l0;
+  }
+  if (small) {
+    if (ev) {
+      cudaEventRecord(ev[2], st);
+      cudaEventRecord(ev[3], st);
+    }
+    ctx->launches += launch_small_iteration(P, fuse_finalize ? ctx->gbpw : 0, st);
+  } else {
+    if (c.flags & LAQ_FLAG_QUANT_OFF) {
+      // no quantizer: one sweep gives the radius, the norm and the skip decisions (the radius slot stays empty)
+      if (ev) cudaEventRecord(ev[2], st);
+      ctx->launches += launch_innovation_trigger(P, ctx->ls, st);
+    } else {
+      ctx->launches += launch_radius(P, ctx->ls, st);
+      if (ev) cudaEventRecord(ev[2], st);
+      ctx->launches += launch_quantize_trigger(P, ctx->ls, st);
+    }
+    if (ev) cudaEventRecord(ev[3], st);
+    ctx->launches += launch_aggregate(P, ctx->ls, st);
+  }
+  if (ev) {
+    cudaEventRecord(ev[4], st);
+    for (int s = 1; s < 4; ++s) ctx->stage_launches[s] += 1;
+  }
+}
+
+bool graphs_usable(const laq_ctx* ctx) {
+  return ctx->graphs_enabled && !ctx->graphs_failed && !ctx->profiling && ctx->cfg.model != LAQ_MODEL_EXTERNAL;
+}
+
+void drop_graphs(laq_ctx* ctx) {
+  if (ctx->graph_one) cudaGraphExecDestroy(ctx->graph_one);
+  if (ctx->graph_many) cudaGraphExecDestroy(ctx->graph_many);
+  ctx->graph_one = ctx->graph_many = nullptr;
+}
+
+// Captures n iterations on the library's own capture stream (the caller's stream may be the legacy default
+// stream, which cannot capture) and instantiates them; null on any failure.
+cudaGraphExec_t capture_iterations(laq_ctx* ctx, int n) {
+  cudaGraph_t graph = nullptr;
+  cudaGraphExec_t exec = nullptr;
+  if (cudaStreamBeginCapture(ctx->cap_stream, cudaStreamCaptureModeRelaxed) != cudaSuccess) return nullptr;
+  const int64_t l0 = ctx->launches;
+  for (int i = 0; i < n; ++i) enqueue_iteration(ctx, ctx->cap_stream, nullptr);
+  ctx->launches_per_iter = (ctx->launches - l0) / n;
+  ctx->launches = l0;                                  // nothing ran: the replays are counted when they are launched
+  const cudaError_t e = cudaStreamEndCapture(ctx->cap_stream, &graph);
+  if (e == cudaSuccess && graph) {
+    if (cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) exec = nullptr;
+    cudaGraphDestroy(graph);
+  }
+  return exec;
+}
+
+void build_graphs(laq_ctx* ctx) {
+  if (!ctx->cap_stream && cudaStreamCreateWithFlags(&ctx->cap_stream, cudaStreamNonBlocking) != cudaSuccess) {
+    ctx->graphs_failed = true;
+    return;
+  }
+  ctx->graph_one = capture_iterations(ctx, 1);
+  ctx->graph_many = ctx->graph_one ? capture_iterations(ctx, kGraphIters) : nullptr;
+  if (!ctx->graph_one || !ctx->graph_many) {
+    drop_graphs(ctx);
+    ctx->graphs_failed = true;    // plain launches from now on
+    cudaGetLastError();
+  }
+}
+
+}  // namespace
+
 extern "C" {
 
 size_t laq_workspace_bytes(const laq_config* cfg) {
@@ -397,60 +505,33 @@ laq_status laq_step(laq_ctx* ctx, int32_t n_iters, const laq_trace* trace) {
   }
   if (trace && n_iters > c.trace_capacity) return fail(ctx, LAQ_EINVAL, "n_iters exceeds trace_capacity");
   LAQ_CUDA(ctx, cudaMemsetAsync(&P.sc->trace_pos, trace ? 0 : 0xff, 4, ctx->st));  // 0xffffffff = tracing off
-  for (int it = 0; it < n_iters; ++it) {
+  int it = 0;
+  if (graphs_usable(ctx) && n_iters >= kGraphMinIters) {
+    // the first iteration of a context goes out as plain launches (it also sets the kernels' attributes); the
+    // graphs are then captured once and replayed: fewer host calls and shorter gaps between dependent kernels
+    if (!ctx->graph_one) {
+      enqueue_iteration(ctx, ctx->st, nullptr);
+      it = 1;
+      build_graphs(ctx);
+    }
+    if (ctx->graph_one) {
+      for (; it + kGraphIters <= n_iters; it += kGraphIters) {
+        LAQ_CUDA(ctx, cudaGraphLaunch(ctx->graph_many, ctx->st));
+        ctx->launches += ctx->launches_per_iter * kGraphIters;
+      }
+      for (; it < n_iters; ++it) {
+        LAQ_CUDA(ctx, cudaGraphLaunch(ctx->graph_one, ctx->st));
+        ctx->launches += ctx->launches_per_iter;
+      }
+    }
+  }
+  for (; it < n_iters; ++it) {
     cudaEvent_t* ev = nullptr;
     if (ctx->profiling && ctx->ev_used < kProfIters) {
       ev = &ctx->ev[(size_t)ctx->ev_used * 5];
       ctx->ev_used += 1;
-      cudaEventRecord(ev[0], ctx->st);
     }
-    const int64_t l0 = ctx->launches;
-    // small problems: steps 2-5 (and, when cheap, the combination of the gradient kernels' block partials)
-    // run in one single-block kernel
-    const bool small = small_iteration_applies(P);
-    const bool linear = c.model == LAQ_MODEL_LOGREG_BIN || c.model == LAQ_MODEL_SOFTMAX;
-    const bool fuse_finalize = small && linear && ctx->gbpw <= 64;
-    switch (c.model) {
-      case LAQ_MODEL_LOGREG_BIN:
-        ctx->launches += launch_grad_logreg(P, ctx->ls, ctx->gbpw, ctx->st);
-        if (!fuse_finalize) ctx->launches += launch_grad_finalize(P, ctx->gbpw, &P.sc->theta_sq, ctx->st);
-        break;
-      case LAQ_MODEL_SOFTMAX:
-        ctx->launches += launch_grad_softmax(P, ctx->ls, ctx->gbpw, ctx->st);
-        if (!fuse_finalize) ctx->launches += launch_grad_finalize(P, ctx->gbpw, &P.sc->theta_sq, ctx->st);
-        break;
-      case LAQ_MODEL_MLP2:
-        ctx->launches += mlp_launch_gradients(ctx->mlp, P, &P.sc->theta_sq, ctx->st);
-        break;
-      default: break;
-    }
-    if (ev) {
-      cudaEventRecord(ev[1], ctx->st);
-      ctx->stage_launches[0] += ctx->launches - l0;
-    }
-    if (small) {
-      if (ev) {
-        cudaEventRecord(ev[2], ctx->st);
-        cudaEventRecord(ev[3], ctx->st);
-      }
-      ctx->launches += launch_small_iteration(P, fuse_finalize ? ctx->gbpw : 0, ctx->st);
-    } else {
-      if (c.flags & LAQ_FLAG_QUANT_OFF) {
-        // no quantizer: one sweep gives the radius, the norm and the skip decisions (the radius slot stays empty)
-        if (ev) cudaEventRecord(ev[2], ctx->st);
-        ctx->launches += launch_innovation_trigger(P, ctx->ls, ctx->st);
-      } else {
-        ctx->launches += launch_radius(P, ctx->ls, ctx->st);
-        if (ev) cudaEventRecord(ev[2], ctx->st);
-        ctx->launches += launch_quantize_trigger(P, ctx->ls, ctx->st);
-      }
-      if (ev) cudaEventRecord(ev[3], ctx->st);
-      ctx->launches += launch_aggregate(P, ctx->ls, ctx->st);
-    }
-    if (ev) {
-      cudaEventRecord(ev[4], ctx->st);
-      for (int s = 1; s < 4; ++s) ctx->stage_launches[s] += 1;
-    }
+    enqueue_iteration(ctx, ctx->st, ev);
   }
   LAQ_CUDA(ctx, cudaGetLastError());
   if (c.model == LAQ_MODEL_EXTERNAL && n_iters == 1) ctx->ext_g_set = false;
@@ -599,7 +680,9 @@ laq_status laq_tune(laq_ctx* ctx, const char* key, int32_t value) {
   else if (k == "agg_threads" && pow2_threads(value) && value <= 256) ctx->ls.agg_threads = value;
   else if (k == "agg_blocks_per_sm" && value >= 1 && value <= 32) ctx->ls.agg_blocks_per_sm = value;
   else if (k == "grad_blocks_per_worker" && value >= 1 && value <= ctx->gbpw_cap) ctx->gbpw = value;
+  else if (k == "graphs" && (value == 0 || value == 1)) ctx->graphs_enabled = value != 0;
   else return fail(ctx, LAQ_EINVAL, "unknown tuning key or value outside its limits");
+  drop_graphs(ctx);     // captured launch shapes are stale
   return LAQ_OK;
 }
 
@@ -640,6 +723,8 @@ void laq_destroy(laq_ctx* ctx) {
   if (!ctx) return;
   if (ctx->ws) cudaStreamSynchronize(ctx->st);
   mlp_teardown(ctx->mlp);
+  drop_graphs(ctx);
+  if (ctx->cap_stream) cudaStreamDestroy(ctx->cap_stream);
   for (auto& e : ctx->ev) cudaEventDestroy(e);
   delete ctx;
 }

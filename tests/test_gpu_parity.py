@@ -490,6 +490,32 @@ def test_state_round_trip_resumes_bit_identically():
     b_.close()
 
 
+@pytest.mark.parametrize("make", [lambda: workloads.c4(M=5, p=43210, b=4), lambda: workloads.c0(),
+                                  lambda: workloads.c1(n_per=240, iters=30), lambda: workloads.c3(n_per=300, iters=30)],
+                         ids=["synthetic", "logreg", "softmax", "network"])
+def test_graph_replay_equals_plain_launches(make):
+    """laq_step replays long calls as CUDA graphs (eight iterations per replay, single ones for the rest): same
+    kernels, same order, so traces, states and the launch count equal those of plain launches bit for bit."""
+    w = make()
+    n = 27                                   # 1 plain + 3 x 8 + 2 single replays
+    runs = []
+    for graphs in (1, 0):
+        c = laq.from_workload(w, trace_capacity=n)
+        c.tune("graphs", graphs)
+        c.step(2)                            # short calls stay plain launches in both runs
+        tr = c.step(n, trace=True)
+        tr2 = c.step(9, trace=True)          # a second long call reuses the captured graphs
+        runs.append((tr, tr2, c.get_state(codes=True), c.kernel_launches()))
+        c.close()
+    (ta, ta2, sa, la), (tb, tb2, sb, lb) = runs
+    for key in ta:
+        np.testing.assert_array_equal(ta[key], tb[key])
+        np.testing.assert_array_equal(ta2[key], tb2[key])
+    for key in ("theta", "agg", "qprev", "n_eps_hat", "clock", "ring", "counters", "codes"):
+        np.testing.assert_array_equal(sa[key], sb[key])
+    assert la == lb and la > 0
+
+
 def test_runs_are_reproducible_bit_for_bit():
     w = workloads.c4(M=7, p=54321, b=2)
     outs = []
