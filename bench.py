@@ -357,6 +357,15 @@ def main():
             kern = {"quantize_kernel": "innovation_kernel", "aggregate_kernel": "aggregate_raw_kernel"}.get(kern, kern)
         stages.append({"stage": name, "kernel": kern, "ms": avg_ms, "bytes": abytes[name],
                        "GB/s": gbs, "frac": gbs / peak, "share": stage_ms[i] / max(stage_ms.sum(), 1e-12)})
+    if w.model != 3 and w.M * ((w.p + 15) // 16 * 16) <= 8192:
+        # small problems run steps 2-5 in one single-block kernel: its time sits in the last slot, the radius and
+        # quantize slots are empty; it moves the bytes of all three sweeps
+        last = stages[-1]
+        last.update({"stage": "steps_2_to_5_single_block", "kernel": "small_iteration_kernel",
+                     "bytes": abytes["radius"] + abytes["quantize_norms_trigger"] + abytes["aggregate_theta_step"]})
+        last["GB/s"] = last["bytes"] / (last["ms"] * 1e-3) / 1e9 if last["ms"] > 0 else 0.0
+        last["frac"] = last["GB/s"] / peak
+        stages = [st for st in stages if st["stage"] not in ("radius", "quantize_norms_trigger")]
     dom = max(stages, key=lambda s: s["ms"])
     path_bytes = sum(s["bytes"] for s in stages)
     path_ms = sum(s["ms"] for s in stages)
@@ -378,12 +387,6 @@ def main():
         roofline.update({"bound": "tensor", "kernel": "umma_hidden_fused_kernel + umma_dw1_kernel (whole gradient stage)",
                          "achieved": tf, "peak": tpeak, "unit": "TFLOP/s", "frac": tf / tpeak, "traffic": None,
                          "peak_source": tsrc, "flops_per_launch": flops, "ms_per_launch": g_stage["ms"]})
-    if w.model != 3 and w.M * ((w.p + 15) // 16 * 16) <= 8192:
-        # small problems run steps 2-5 in one single-block kernel: the radius and quantize slots are empty
-        stages = [st for st in stages if st["stage"] not in ("radius", "quantize_norms_trigger")]
-        stages[-1]["stage"] = "steps_2_to_5_single_block"
-        stages[-1]["kernel"] = "small_iteration_kernel"
-        roofline["stages"] = stages
     line = {"metric": METRIC, "value": replicas_throughput(world, K, ms), "unit": "iters/s", "n_gpus": world, "steps": K,
             "warmup": Wm, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
