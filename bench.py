@@ -180,8 +180,10 @@ def traffic_for(stage, w):
     try:
         with open(path) as f:
             rec = json.load(f)
-        src = os.path.join(ROOT, "paper_1909_07588_b200", "csrc", rec["source"])
-        if hashlib.sha256(open(src, "rb").read()).hexdigest() != rec["source_sha256"]:
+        h = hashlib.sha256()
+        for name in rec["sources"]:
+            h.update(open(os.path.join(ROOT, "paper_1909_07588_b200", "csrc", name), "rb").read())
+        if h.hexdigest() != rec["sources_sha256"]:
             return None
         per_coord = rec["bytes_per_worker_coordinate"]["c4_b%d" % w.b][stage]
         return None if per_coord is None or w.model != 3 else per_coord * float(w.M) * w.p
