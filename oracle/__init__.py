@@ -7,5 +7,5 @@ from .binding import (  # noqa: F401
     MODEL_LOGREG_BIN, MODEL_SOFTMAX, MODEL_MLP2, MODEL_SYNTH, MODEL_GIVEN,
     FLAG_QUANT_OFF, FLAG_TRIGGER_OFF,
     build, lib, quantize, decode, pack_codes, unpack_codes, trigger, batch_offset,
-    grad_logreg_bin, grad_softmax, grad_mlp2, synth_gradient, round_bf16, OracleLaq,
+    grad_logreg_bin, grad_softmax, grad_mlp2, synth_gradient, round_bf16, lyapunov, OracleLaq,
 )

@@ -218,6 +218,25 @@ def synth_gradient(seed, m, M, p, k, sigma, eta0):
     return g
 
 
+def lyapunov(losses, dtheta2s, xi, alpha, f_star):
+    """Lyapunov function of Sec. 3, written out term by term:
+        V(theta^k) = f(theta^k) - f(theta*) + sum_{d=1}^{D} sum_{j=d}^{D} (xi_j / alpha) ||theta^{k+1-d} - theta^{k-d}||^2.
+    losses[k-1] = f(theta^k), dtheta2s[k-1] = ||theta^{k+1} - theta^k||^2 for k = 1..n; differences that lie before
+    the first iteration do not exist and count as zero."""
+    D, n = len(xi), len(losses)
+    out = []
+    for k in range(1, n + 1):
+        v = float(losses[k - 1]) - float(f_star)
+        for d in range(1, D + 1):
+            it = k - d                      # ||theta^{k+1-d} - theta^{k-d}||^2 is the step of iteration k - d
+            if it < 1:
+                continue
+            for j in range(d, D + 1):
+                v += float(xi[j - 1]) / float(alpha) * float(dtheta2s[it - 1])
+        out.append(v)
+    return np.array(out)
+
+
 def round_bf16(x):
     return lib().laqo_round_bf16(float(x))
 

@@ -333,3 +333,52 @@ def test_minibatch_as_large_as_the_shard_is_the_full_gradient():
         sa, sb = a.step(), b.step()
         np.testing.assert_array_equal(sa["skip"], sb["skip"])
         np.testing.assert_allclose(b.state(big=False)["theta"], a.state(big=False)["theta"], rtol=1e-11, atol=1e-13)
+
+
+# ------------------------------------------------------------------------------------------------
+# Lyapunov function of Sec. 3
+# ------------------------------------------------------------------------------------------------
+def test_lyapunov_hand_numbers():
+    """D = 2, xi = (0.25, 0.5), alpha = 0.5: c_1 = (0.25 + 0.5) / 0.5 = 1.5, c_2 = 0.5 / 0.5 = 1.
+    f = (10, 7, 5, 4), steps ||theta^{k+1} - theta^k||^2 = (4, 2, 1, .), f* = 3:
+      V^1 = 7                         (no earlier step exists)
+      V^2 = 4 + 1.5 * 4           = 10
+      V^3 = 2 + 1.5 * 2 + 1 * 4   = 9
+      V^4 = 1 + 1.5 * 1 + 1 * 2   = 4.5"""
+    v = oracle.lyapunov([10.0, 7.0, 5.0, 4.0], [4.0, 2.0, 1.0, 99.0], [0.25, 0.5], 0.5, 3.0)
+    np.testing.assert_allclose(v, [7.0, 10.0, 9.0, 4.5], rtol=0, atol=1e-15)
+    # all weights zero: the Lyapunov function is the loss residual
+    v0 = oracle.lyapunov([10.0, 7.0, 5.0], [4.0, 2.0, 1.0], [0.0, 0.0, 0.0], 0.5, 3.0)
+    np.testing.assert_allclose(v0, [7.0, 4.0, 2.0], rtol=0, atol=0)
+
+
+def test_lyapunov_function_decays_linearly_under_the_lemma_parameters():
+    """Theorem 1 on a tiny least-squares problem with xi_d = 1/(16 D), alpha = 1/(8 L): V >= f - f* >= 0, and V
+    shrinks by a constant factor per iteration on average (it need not be monotone: Lemma 1 has the
+    quantization errors on its right-hand side)."""
+    rng = np.random.default_rng(11)
+    M, p, D = 3, 4, 5
+    A = rng.standard_normal((M, 6, p))
+    bvec = rng.standard_normal((M, 6))
+    H = sum(a.T @ a for a in A)
+    theta_star = np.linalg.solve(H, sum(a.T @ bb for a, bb in zip(A, bvec)))
+    f = lambda th: 0.5 * sum(np.sum((a @ th - bb) ** 2) for a, bb in zip(A, bvec))
+    L = np.linalg.eigvalsh(H).max()
+    alpha, xi = 1.0 / (8 * L), np.full(D, 1.0 / (16 * D))
+    o = oracle.OracleLaq(64, oracle.MODEL_GIVEN, M, p, alpha=alpha, b=4, D=D, xi=xi, tbar=20)
+    theta = np.zeros(p)
+    losses, d2s = [], []
+    for k in range(700):
+        losses.append(f(theta))
+        st = o.step_given(np.stack([a.T @ (a @ theta - bb) for a, bb in zip(A, bvec)]))
+        d2s.append(st["dtheta2"])
+        theta = o.state()["theta"]
+    v = oracle.lyapunov(losses, d2s, xi, alpha, f(theta_star))
+    res = np.array(losses) - f(theta_star)
+    assert np.all(v >= res - 1e-15) and np.all(res > -1e-12)
+    ks = np.arange(20, 500)
+    ok = v[ks] > 1e-24
+    sigma = np.exp(np.polyfit(ks[ok], np.log(v[ks][ok]), 1)[0])
+    assert 0.0 < sigma < 0.99
+    assert v[600] < 1e-10 * v[0]
+    assert np.all(v[100:] < v[50])
