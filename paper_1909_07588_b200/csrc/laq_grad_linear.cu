@@ -128,9 +128,13 @@ __device__ __forceinline__ void stage_rows_async(const float* __restrict__ src, 
 // residual read from shared memory feeds two multiply-adds.  About a third of the instructions of the kernel above.
 constexpr int kLr2Rows = 128;
 
+// FT > 0 fixes the feature count at compile time (54 and 22, the shapes of the paper's two logistic-regression
+// tests): offsets become immediates, the score loop is straight-line code and its half of theta sits in registers.
+// FT = 0 reads the count from the parameters.  The arithmetic and its order are the same in both forms.
+template <int FT>
 __global__ void __launch_bounds__(kLrThreads) grad_logreg_pair_kernel(const Params P, int gbpw) {
   extern __shared__ __align__(16) float smem[];
-  const int F = P.F, F2 = F >> 1, m = blockIdx.y, t = threadIdx.x;
+  const int F = FT > 0 ? FT : P.F, F2 = F >> 1, m = blockIdx.y, t = threadIdx.x;
   float* xs0 = smem;                         // [2][128][F]
   float* ths = xs0 + 2 * kLr2Rows * F;       // [F]
   float* rs = ths + ((F + 3) & ~3);          // [128]
@@ -139,12 +143,20 @@ __global__ void __launch_bounds__(kLrThreads) grad_logreg_pair_kernel(const Para
   __shared__ float zpart[kLr2Rows];
   const float* __restrict__ X = P.X[m];
   const int32_t* __restrict__ y = P.y[m];
-  for (int f = t; f < F; f += blockDim.x) ths[f] = P.theta[f];
   const int S = kLrThreads / F2;             // row slices handled in parallel in the second phase
   const bool active = t < S * F2;
   const int j_own = t % F2, slice = t / F2;
   const int row = t & (kLr2Rows - 1), half = t >> 7, fh = (F2 + 1) >> 1;   // first phase: half of the features of a row
   const int f_lo = half * fh, f_hi = half ? F2 : fh;
+  constexpr int kHalfPairs = FT > 0 ? (FT / 2 + 1) / 2 : 1;
+  float2 thr[kHalfPairs];                    // FT > 0: this thread's half of theta, as pairs
+  if constexpr (FT > 0) {
+#pragma unroll
+    for (int i = 0; i < kHalfPairs; ++i)
+      thr[i] = f_lo + i < f_hi ? __ldg(reinterpret_cast<const float2*>(P.theta) + f_lo + i) : make_float2(0.f, 0.f);
+  } else {
+    for (int f = t; f < F; f += blockDim.x) ths[f] = P.theta[f];
+  }
   float acc0 = 0.f, acc1 = 0.f;
   double loss = 0.0;
   RowWindow win = row_window(P, m);
@@ -164,6 +176,8 @@ __global__ void __launch_bounds__(kLrThreads) grad_logreg_pair_kernel(const Para
     win.tile(tile, kLr2Rows, r0, nr);
     float* xs = xs0 + buf * kLr2Rows * F;
     __syncthreads();                                  // everybody is done with the buffer refilled below
+    // the row's label, asked for now and used after the scores
+    const int y_row = (half == 0 && row < nr) ? __ldg(y + r0 + row) : 0;
     if (tile + gridDim.x < ntiles) stage(tile + gridDim.x, xs0 + (buf ^ 1) * kLr2Rows * F);
     __pipeline_commit();
     __pipeline_wait_prior(1);                         // this tile's copies (the older group) have landed
@@ -172,19 +186,30 @@ __global__ void __launch_bounds__(kLrThreads) grad_logreg_pair_kernel(const Para
       float z = 0.f;
       if (row < nr) {
         const float2* xr = reinterpret_cast<const float2*>(xs + row * F);
-        const float2* th2 = reinterpret_cast<const float2*>(ths);
+        if constexpr (FT > 0) {
+          const float2* xh = xr + f_lo;
+#pragma unroll
+          for (int i = 0; i < kHalfPairs; ++i)
+            if (i + 1 < kHalfPairs || f_lo + i < f_hi) {   // only the last pair of the second half can be missing
+              const float2 x = xh[i];
+              z = fmaf(x.x, thr[i].x, z);
+              z = fmaf(x.y, thr[i].y, z);
+            }
+        } else {
+          const float2* th2 = reinterpret_cast<const float2*>(ths);
 #pragma unroll 4
-        for (int f = f_lo; f < f_hi; ++f) {
-          const float2 x = xr[f], th = th2[f];
-          z = fmaf(x.x, th.x, z);
-          z = fmaf(x.y, th.y, z);
+          for (int f = f_lo; f < f_hi; ++f) {
+            const float2 x = xr[f], th = th2[f];
+            z = fmaf(x.x, th.x, z);
+            z = fmaf(x.y, th.y, z);
+          }
         }
       }
       if (half) zpart[row] = z;                       // warps 4-7: second half of the features
       __syncthreads();
       if (half == 0 && row < nr) {                    // warps 0-3: join the halves, residual and loss
         z = z + zpart[row];
-        const float yv = (float)y[r0 + row];
+        const float yv = (float)y_row;
         float sig, sp;
         if (z >= 0.f) {
           const float e = expf(-z);
@@ -804,11 +829,15 @@ int launch_grad_logreg(const Params& P, const LaunchShape&, int gbpw, cudaStream
   static bool attr_done = false;
   if (!attr_done) {
     cudaFuncSetAttribute(grad_logreg_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    cudaFuncSetAttribute(grad_logreg_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    cudaFuncSetAttribute(grad_logreg_pair_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    cudaFuncSetAttribute(grad_logreg_pair_kernel<22>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    cudaFuncSetAttribute(grad_logreg_pair_kernel<54>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     attr_done = true;
   }
   if ((P.F & 1) == 0)
-    grad_logreg_pair_kernel<<<dim3(gbpw, P.M), kLrThreads, sm, st>>>(P, gbpw);
+    if (P.F == 54) grad_logreg_pair_kernel<54><<<dim3(gbpw, P.M), kLrThreads, sm, st>>>(P, gbpw);
+    else if (P.F == 22) grad_logreg_pair_kernel<22><<<dim3(gbpw, P.M), kLrThreads, sm, st>>>(P, gbpw);
+    else grad_logreg_pair_kernel<0><<<dim3(gbpw, P.M), kLrThreads, sm, st>>>(P, gbpw);
   else
     grad_logreg_kernel<<<dim3(gbpw, P.M), kLrThreads, sm, st>>>(P, gbpw, logreg_rows(P.F));
   return 1;
