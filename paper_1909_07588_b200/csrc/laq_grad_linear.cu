@@ -826,20 +826,17 @@ int grad_blocks_per_sm(int model, int F, int C) {
 
 int launch_grad_logreg(const Params& P, const LaunchShape&, int gbpw, cudaStream_t st) {
   const size_t sm = logreg_smem(P.F);
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaFuncSetAttribute(grad_logreg_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    cudaFuncSetAttribute(grad_logreg_pair_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    cudaFuncSetAttribute(grad_logreg_pair_kernel<22>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    cudaFuncSetAttribute(grad_logreg_pair_kernel<54>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    attr_done = true;
-  }
-  if ((P.F & 1) == 0)
-    if (P.F == 54) grad_logreg_pair_kernel<54><<<dim3(gbpw, P.M), kLrThreads, sm, st>>>(P, gbpw);
-    else if (P.F == 22) grad_logreg_pair_kernel<22><<<dim3(gbpw, P.M), kLrThreads, sm, st>>>(P, gbpw);
-    else grad_logreg_pair_kernel<0><<<dim3(gbpw, P.M), kLrThreads, sm, st>>>(P, gbpw);
-  else
-    grad_logreg_kernel<<<dim3(gbpw, P.M), kLrThreads, sm, st>>>(P, gbpw, logreg_rows(P.F));
+  const dim3 grid(gbpw, P.M);
+  // more than the default 48 KB of dynamic shared memory is asked for per kernel and per device; the call is cheap
+  // and idempotent, so it goes with every launch rather than behind a process-wide flag
+  auto launch = [&](auto kernel, auto... extra) {
+    if (sm > 40 * 1024) cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    kernel<<<grid, kLrThreads, sm, st>>>(P, gbpw, extra...);
+  };
+  if (P.F & 1) launch(grad_logreg_kernel, logreg_rows(P.F));
+  else if (P.F == 54) launch(grad_logreg_pair_kernel<54>);
+  else if (P.F == 22) launch(grad_logreg_pair_kernel<22>);
+  else launch(grad_logreg_pair_kernel<0>);
   return 1;
 }
 
