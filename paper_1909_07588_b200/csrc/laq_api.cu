@@ -40,6 +40,7 @@ struct laq_ctx {
   cudaStream_t cap_stream = nullptr;   // capture happens here, never on the caller's stream
   cudaGraphExec_t graph_one = nullptr, graph_many = nullptr;
   int64_t launches_per_iter = 0;
+  std::vector<char> trace_host;        // short per-iteration reports land here in one copy
 };
 
 namespace {
@@ -48,6 +49,7 @@ constexpr size_t kAlign = 256;
 constexpr int kMaxAggBlocks = kNumSMs * 32;
 constexpr int kGradBlocksCap = 64;
 constexpr int kProfIters = 512;
+constexpr size_t kTraceSpanMax = 64 * 1024;   // reports up to this size come back in one copy
 
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
@@ -537,6 +539,28 @@ laq_status laq_step(laq_ctx* ctx, int32_t n_iters, const laq_trace* trace) {
   if (c.model == LAQ_MODEL_EXTERNAL && n_iters == 1) ctx->ext_g_set = false;
   if (!trace) return LAQ_OK;
   const size_t n = (size_t)n_iters, M = (size_t)c.M;
+  // The eight report arrays lie one after the other in the workspace.  Short reports come back as ONE copy of that
+  // span into a host buffer of the context and are handed out from there: a call that steps one iteration and reads
+  // its report pays for one transfer instead of eight.  Long reports are copied array by array, rows used only.
+  const char* span0 = (const char*)P.t_skip;
+  const size_t span = (size_t)((const char*)P.t_up + (size_t)c.trace_capacity * 4 - span0);
+  if (span <= kTraceSpanMax) {
+    if (ctx->trace_host.size() < span) ctx->trace_host.resize(span);
+    LAQ_CUDA(ctx, cudaMemcpyAsync(ctx->trace_host.data(), span0, span, cudaMemcpyDeviceToHost, ctx->st));
+    const laq_status status = check_device_error(ctx);     // synchronises
+    auto hand = [&](void* dst, const void* src, size_t bytes) {
+      if (dst && bytes) std::memcpy(dst, ctx->trace_host.data() + ((const char*)src - span0), bytes);
+    };
+    hand(trace->skip, P.t_skip, n * M);
+    hand(trace->R, P.t_R, n * M * 4);
+    hand(trace->n_dq, P.t_ndq, n * M * 8);
+    hand(trace->n_eps, P.t_neps, n * M * 8);
+    hand(trace->rhs, P.t_rhs, n * M * 8);
+    hand(trace->dtheta2, P.t_d2, n * 8);
+    hand(trace->loss, P.t_loss, n * 8);
+    hand(trace->uploads, P.t_up, n * 4);
+    return status;
+  }
   auto pull = [&](void* dst, const void* src, size_t bytes) -> cudaError_t {
     if (!dst || !bytes) return cudaSuccess;
     return cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, ctx->st);
