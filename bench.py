@@ -346,7 +346,7 @@ def main():
     peak, peak_src = hbm_peak()
     abytes = algorithmic_bytes(w, u)
     stages = []
-    iters_recorded = int(stage_n[1])          # the library brackets at most 512 iterations per call
+    iters_recorded = int(stage_n[3])          # one aggregate launch per iteration; at most 512 iterations are bracketed
     for i, name in enumerate(STAGES):
         if stage_n[i] == 0 or iters_recorded == 0:
             continue

@@ -242,14 +242,16 @@ void enqueue_iteration(laq_ctx* ctx, cudaStream_t st, cudaEvent_t* ev) {
   const bool small = small_iteration_applies(P);
   const bool linear = c.model == LAQ_MODEL_LOGREG_BIN || c.model == LAQ_MODEL_SOFTMAX;
   const bool fuse_finalize = small && linear && ctx->gbpw <= 64;
+  // mid-size linear models: the kernel that combines the gradient partials also takes the quantizer's radius
+  const bool fuse_radius = linear && !small && !(c.flags & LAQ_FLAG_QUANT_OFF);
   switch (c.model) {
     case LAQ_MODEL_LOGREG_BIN:
       ctx->launches += launch_grad_logreg(P, ctx->ls, ctx->gbpw, st);
-      if (!fuse_finalize) ctx->launches += launch_grad_finalize(P, ctx->gbpw, &P.sc->theta_sq, st);
+      if (!fuse_finalize) ctx->launches += launch_grad_finalize(P, ctx->gbpw, &P.sc->theta_sq, fuse_radius, st);
       break;
     case LAQ_MODEL_SOFTMAX:
       ctx->launches += launch_grad_softmax(P, ctx->ls, ctx->gbpw, st);
-      if (!fuse_finalize) ctx->launches += launch_grad_finalize(P, ctx->gbpw, &P.sc->theta_sq, st);
+      if (!fuse_finalize) ctx->launches += launch_grad_finalize(P, ctx->gbpw, &P.sc->theta_sq, fuse_radius, st);
       break;
     case LAQ_MODEL_MLP2:
       ctx->launches += mlp_launch_gradients(ctx->mlp, P, &P.sc->theta_sq, st);
@@ -272,7 +274,7 @@ void enqueue_iteration(laq_ctx* ctx, cudaStream_t st, cudaEvent_t* ev) {
       if (ev) cudaEventRecord(ev[2], st);
       ctx->launches += launch_innovation_trigger(P, ctx->ls, st);
     } else {
-      ctx->launches += launch_radius(P, ctx->ls, st);
+      if (!fuse_radius) ctx->launches += launch_radius(P, ctx->ls, st);
       if (ev) cudaEventRecord(ev[2], st);
       ctx->launches += launch_quantize_trigger(P, ctx->ls, st);
     }
@@ -281,7 +283,7 @@ void enqueue_iteration(laq_ctx* ctx, cudaStream_t st, cudaEvent_t* ev) {
   }
   if (ev) {
     cudaEventRecord(ev[4], st);
-    for (int s = 1; s < 4; ++s) ctx->stage_launches[s] += 1;
+    for (int s = 1; s < 4; ++s) ctx->stage_launches[s] += (s == 1 && (small || fuse_radius || (c.flags & LAQ_FLAG_QUANT_OFF))) ? 0 : 1;
   }
 }
 

@@ -4,7 +4,7 @@
 // as a skinny contraction that reads every sample once: a block stages a tile of consecutive rows
 // (contiguous in memory) in shared memory, computes the residuals (sigma(z) - y, or softmax - onehot)
 // and accumulates residual^T x in registers across its tiles.  Block partials are combined in a
-// fixed order by grad_finalize_kernel, which also adds the regulariser share.
+// fixed order by grad_finalize_kernel, which also adds the regulariser share (and takes the quantizer's radius).
 #include <cuda_pipeline.h>
 
 #include "laq_internal.cuh"
@@ -543,17 +543,28 @@ __global__ void __launch_bounds__(kS2Threads, 2) grad_softmax_tile_kernel(const 
 // Combine the block partials of worker blockIdx.y in block order, scale by 1/N and add the
 // worker's share (N_m/N) lambda theta of the regulariser; block 0 of each worker also writes the
 // worker's loss term.  theta_sq = ||theta^k||^2 comes from the previous theta step.
+// RADIUS: the kernel also takes the largest |g_m - Q_prev| of its coordinates (as unsigned bit patterns, which order
+// like the floats and put inf and nan on top) into the worker's radius word of this iteration, so that the separate
+// radius sweep is not launched: the gradient is in a register here anyway.
+template <bool RADIUS>
 __global__ void __launch_bounds__(256) grad_finalize_kernel(const Params P, int gbpw, const double* theta_sq) {
   const int m = blockIdx.y;
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const double inv_N = 1.0 / (double)P.Ntot;
   const double share = (double)P.N[m] / (double)P.Ntot;
+  uint32_t mx = 0;
   if (i < P.p) {
     const float* gp = P.gpart + (long long)m * gbpw * P.ps + i;
     double s = 0.0;
     for (int blk = 0; blk < gbpw; ++blk) s += (double)gp[(long long)blk * P.ps];
     const double g = s * (inv_N * batch_scale(P, m)) + share * (double)P.lambda * (double)P.theta[i];
-    P.g[(long long)m * P.ps + i] = (float)g;
+    const float gf = (float)g;
+    P.g[(long long)m * P.ps + i] = gf;
+    if (RADIUS) mx = __float_as_uint(__fsub_rn(gf, P.qp[(long long)m * P.ps + i])) & 0x7fffffffu;
+  }
+  if (RADIUS) {
+    mx = __reduce_max_sync(0xffffffffu, mx);
+    if ((threadIdx.x & 31) == 0 && mx != 0u) atomicMax(&P.Rbits[(P.sc->k & 1ull) * P.M + m], mx);   // order independent
   }
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     double l = 0.0;
@@ -887,9 +898,12 @@ int launch_grad_softmax(const Params& P, const LaunchShape&, int gbpw, cudaStrea
   return 1;
 }
 
-int launch_grad_finalize(const Params& P, int gbpw, const double* theta_sq, cudaStream_t st) {
+int launch_grad_finalize(const Params& P, int gbpw, const double* theta_sq, bool with_radius, cudaStream_t st) {
   dim3 grid((unsigned)((P.p + 255) / 256), P.M);
-  grad_finalize_kernel<<<grid, 256, 0, st>>>(P, gbpw, theta_sq);
+  if (with_radius)
+    grad_finalize_kernel<true><<<grid, 256, 0, st>>>(P, gbpw, theta_sq);
+  else
+    grad_finalize_kernel<false><<<grid, 256, 0, st>>>(P, gbpw, theta_sq);
   return 1;
 }
 

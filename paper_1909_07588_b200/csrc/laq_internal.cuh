@@ -222,7 +222,7 @@ int launch_quantize_trigger(const Params& P, const LaunchShape& ls, cudaStream_t
 int launch_aggregate(const Params& P, const LaunchShape& ls, cudaStream_t st);
 int launch_grad_logreg(const Params& P, const LaunchShape& ls, int gbpw, cudaStream_t st);
 int launch_grad_softmax(const Params& P, const LaunchShape& ls, int gbpw, cudaStream_t st);
-int launch_grad_finalize(const Params& P, int gbpw, const double* theta_sq, cudaStream_t st);
+int launch_grad_finalize(const Params& P, int gbpw, const double* theta_sq, bool with_radius, cudaStream_t st);
 bool softmax_classes_supported(int C);
 int grad_tiles_per_worker(int model, int F, int C, long long n_max);
 int grad_blocks_per_sm(int model, int F, int C);
