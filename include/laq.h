@@ -18,17 +18,19 @@
  *   - All device work is enqueued on the stream given to laq_init.
  *   - No function throws, aborts or traps the device.  Every fallible function returns a laq_status;
  *     laq_last_error() gives a text for the most recent failure on that context.
- *   - Conditions detected on the device (a non-finite gradient or radius) freeze the state at the
- *     iteration where they occurred and are reported by the next call that synchronises
- *     (laq_step with a trace, laq_get_state, laq_sync) as LAQ_ENONFINITE.
+ *   - Conditions detected on the device freeze the state at the iteration where they occurred and are
+ *     reported by the next call that synchronises (laq_step with a trace, laq_get_state, laq_get_worker,
+ *     laq_sync): a non-finite gradient or radius as LAQ_ENONFINITE, a bounded wait that ran out as
+ *     LAQ_ETIMEOUT.  No kernel waits without a limit, and none traps.  laq_set_state clears the condition.
  *   - Floating point: theta, gradients and quantizer state are fp32; each quantizer operation is one
  *     IEEE round-to-nearest operation in the order  d = g - Q_prev ; R = max|d| ; s = (2 tau) R ;
  *     t = (d + R)/s + 1/2 (IEEE division) ; q = floor t ; dQ = s q - R (multiply, then subtract) ;
  *     Q_new = Q_prev + dQ ; eps = g - Q_new, with no fused multiply-add (kernels may reach q by a cheaper
  *     route where they can prove that it gives the same integer); codes, dQ, Q_new and eps are therefore
  *     reproducible bit for bit.  Squared norms are fp64 sums of exact fp32 products, except that the sweep over
- *     rows generated in the kernel (LAQ_MODEL_SYNTH) first sums runs of 32 products in fp32 (relative error of
- *     a run below 2^-19; of a whole row typically 1e-9); the skip rule is evaluated in fp64.
+ *     rows generated in the kernel (LAQ_MODEL_SYNTH) and over rows of 2^20 or more coordinates read from memory
+ *     first sums runs of 32 products in fp32 (relative error of a run below 2^-19; of a whole row typically
+ *     1e-9); the skip rule is evaluated in fp64.
  *   - Code stream of worker m (the paper's b p-bit part of the upload message): code i occupies bits
  *     [i b, (i+1) b) of the stream, bit j of the stream being bit (j mod 32) of 32-bit word floor(j / 32)
  *     (least significant first; for b = 3 a code may straddle two words).
@@ -54,7 +56,9 @@ typedef enum {
   LAQ_EWORKSPACE = 2,  /* workspace pointer null, misaligned (256 B) or too small */
   LAQ_ECUDA = 3,       /* a CUDA runtime call failed */
   LAQ_ENONFINITE = 4,  /* a gradient or radius was inf/nan; state frozen at that iteration */
-  LAQ_ESTATE = 5       /* call not valid in the context's current state (e.g. shards missing) */
+  LAQ_ESTATE = 5,      /* call not valid in the context's current state (e.g. shards missing) */
+  LAQ_ETIMEOUT = 6     /* a bounded wait inside a kernel (on an asynchronous copy or a tensor-core stage) ran out;
+                          the kernel gave up, the state is frozen at that iteration, the CUDA context stays usable */
 } laq_status;
 
 /* Which f_m the workers hold (supplement, "Simulation details"; global loss f = (1/N) sum_m f_m,
@@ -81,8 +85,11 @@ enum {
   LAQ_FLAG_QUANT_OFF = 1u,  /* no quantizer: an upload carries the innovation g_m - Q_m(theta_hat^{k-1}) itself,
                                32 bits per coordinate, eps = 0 in (7a): the lazily aggregated gradient baseline
                                (LAG) of Sec. 4.  R is still reported; no codes are written (they stay zero) */
-  LAQ_FLAG_TRIGGER_OFF = 2u /* every worker uploads every iteration: Algorithm 1 (QGD); with LAQ_FLAG_QUANT_OFF
+  LAQ_FLAG_TRIGGER_OFF = 2u,/* every worker uploads every iteration: Algorithm 1 (QGD); with LAQ_FLAG_QUANT_OFF
                                as well: gradient descent, Eq. (2) */
+  LAQ_FLAG_STORE_G = 4u     /* LAQ_MODEL_SYNTH only: step 1 writes the M x p gradients of the iteration to the
+                               workspace (as a gradient kernel does, Algorithm 2's worker step) and steps 2-5 read
+                               them from memory instead of regenerating them; same values, same results */
 };
 
 typedef struct {
@@ -97,8 +104,11 @@ typedef struct {
   float lambda;             /* l2 regulariser */
   int32_t b;                /* bits per coordinate: 1, 2, 3, 4, 8 or 16 */
   int32_t D;                /* number of stored parameter differences, 1..64; the paper requires D <= t_bar */
-  const float* xi;          /* HOST, length D: weights xi_1..xi_D of (7a), xi[0] pairs with the newest difference */
-  int32_t tbar;             /* staleness bound of (7b) */
+  const float* xi;          /* HOST, length D: weights xi_1..xi_D of (7a), finite and >= 0; xi[0] pairs with the
+                               newest difference */
+  int32_t tbar;             /* staleness bound of (7b), -1 .. 2^31 - 3 (with -1 the clock test always fails:
+                               nobody ever skips).  The paper asks for D <= t_bar; smaller values are accepted,
+                               the rule (7a) then looks further back than a copy can be stale */
   int32_t clock_mode;       /* 0: Algorithm 2 as printed, skip allowed while t_m <= t_bar;
                                1: strict, skip needs t_m + 2 <= t_bar (t_bar = 1 never skips) */
   uint32_t flags;           /* LAQ_FLAG_* */
@@ -138,7 +148,7 @@ typedef struct {
   int32_t* clock;     /* (S) [M]        t_m */
   double* ring;       /* (S) [D]        stored squared differences, newest first */
   int64_t* counters;  /* (S) [3]        iterations done, uploads so far, bits so far (uploads x (32 + b p)) */
-  float* g;           /*     [M][p]     last local gradients (not for SYNTH) */
+  float* g;           /*     [M][p]     last local gradients (SYNTH: only with LAQ_FLAG_STORE_G) */
   uint32_t* codes;    /*     [M][W]     last code streams, W = ceil(p b / 32) words per worker */
   float* R;           /*     [M]        last radii */
   double* n_dq;       /*     [M]        last ||dQ_m||^2 */
@@ -178,7 +188,8 @@ laq_status laq_step(laq_ctx* ctx, int32_t n_iters, const laq_trace* trace);
 /* Wait for the stream and report device-detected errors. */
 laq_status laq_sync(laq_ctx* ctx);
 
-/* Copy state to HOST buffers (synchronises).  Returns LAQ_ENONFINITE if the state is frozen. */
+/* Copy state to HOST buffers (synchronises).  The buffers are filled even when the state is frozen; the call
+ * then returns LAQ_ENONFINITE or LAQ_ETIMEOUT. */
 laq_status laq_get_state(laq_ctx* ctx, const laq_state* out);
 
 /* One worker's rows after the last iteration (synchronises): qprev [p] = Q_m(theta_hat_m), g [p] = its
@@ -195,8 +206,17 @@ int64_t laq_kernel_launches(const laq_ctx* ctx);
 /* Launch-shape override for measurement sweeps: key "sweep_threads", "sweep_blocks_per_sm",
  * "agg_threads", "agg_blocks_per_sm", "grad_blocks_per_worker", and "graphs" (0: laq_step uses plain launches
  * only; 1, the default: graph replay).  Values outside the documented limits return LAQ_EINVAL and change
- * nothing. */
+ * nothing.
+ * Key "starve_copies" (0 or 1, default 0) exists for testing the LAQ_ETIMEOUT path without disturbing the device:
+ * while it is 1, one warp of the quantize sweep over generated rows (LAQ_MODEL_SYNTH), and the loader of one block
+ * of the network's tensor-core kernels (LAQ_MODEL_MLP2), issue none of their asynchronous copies and poll with a
+ * short limit, so their consumers' waits run out with nothing in flight. */
 laq_status laq_tune(laq_ctx* ctx, const char* key, int32_t value);
+
+/* Read-only facts about the launch plan, for tests and reports: key "sweep_blocks_per_worker", "sweep_threads",
+ * "sweep_tile_groups" (16-byte groups per staged tile of the quantize sweep over generated or stored rows),
+ * "aggregate_blocks", "grad_blocks_per_worker".  Unknown keys return LAQ_EINVAL. */
+laq_status laq_query(const laq_ctx* ctx, const char* key, int64_t* value /* HOST */);
 
 /* Per-kernel device timing for measurement.  While enabled, laq_step brackets every stage of an iteration
  * with CUDA events on the context's stream (up to 512 iterations per call are recorded).
@@ -224,7 +244,9 @@ laq_status laq_kernel_times(laq_ctx* ctx, double* ms, int64_t* launches);
  * previous call's values (the call clears what must start at zero): calls whose kernels overlap on the same
  * GPU race with each other, so keep them on one stream or otherwise serialised.  The first call on each
  * device looks up the scratch's device address (and loads the module); make that call during start-up,
- * before any stream capture.  A non-finite input yields a non-finite *d_R, zero norms and untouched codes. */
+ * before any stream capture.  The device that holds the buffers must be the current device of the calling thread
+ * (checked: LAQ_EINVAL otherwise).  The looked-up address is cached per device and does not survive a
+ * cudaDeviceReset.  A non-finite input yields a non-finite *d_R, zero norms and untouched codes. */
 laq_status laq_quantize_worker_static(const float* d_g, const float* d_qprev, int64_t p, int32_t b,
                                       uint32_t* d_codes, float* d_R, double* d_norms, void* cuda_stream,
                                       char* errbuf, size_t errbuf_len);

@@ -85,6 +85,8 @@ float round_bf16(float x) {
 // Operation order (each one IEEE operation in T):
 //   d = g - qp ; R = max |d| ; tau = 1/(2^b-1) ; s = (2 tau) R ; t = (d + R)/s + 1/2 ;
 //   q = clamp(floor(t), 0, 2^b-1) ; dq = s q - R ; qnew = qp + dq ; eps = g - qnew.
+// Eq. (5) is 0/0 (or x/0) when the grid step s is zero: R = 0, or R so small that 2 tau R underflows in T.
+// Then q = 0, and Eq. (6) is applied as printed (for R = 0 it gives dq = 0).
 // ---------------------------------------------------------------------------------------------
 template <typename T>
 void quantize(const T* g, const T* qp, i64 p, int b, T* R_out, int32_t* q, T* dq, T* qnew, T* eps,
@@ -103,16 +105,15 @@ void quantize(const T* g, const T* qp, i64 p, int b, T* R_out, int32_t* q, T* dq
   double sdq = 0.0, seps = 0.0;
   for (i64 i = 0; i < p; ++i) {
     int32_t qi = 0;
-    T dqi = 0;
-    if (R > (T)0) {
+    if (s > (T)0) {
       T d = g[i] - qp[i];
       T t = (d + R) / s + (T)0.5;
       T f = std::floor(t);
       if (f < (T)0) f = 0;
       if (f > levels) f = levels;
       qi = (int32_t)f;
-      dqi = s * (T)qi - R;  // Eq. (6): multiply, then subtract
     }
+    T dqi = s * (T)qi - R;  // Eq. (6): multiply, then subtract
     T qn = qp[i] + dqi;
     T e = g[i] - qn;
     if (q) q[i] = qi;
@@ -133,7 +134,7 @@ void decode(T R, const int32_t* q, const T* qp, i64 p, int b, T* qnew, T* dq) {
   const T tau = (T)1 / levels;
   const T s = ((T)2 * tau) * R;
   for (i64 i = 0; i < p; ++i) {
-    T d = (R > (T)0) ? (s * (T)q[i] - R) : (T)0;
+    T d = s * (T)q[i] - R;
     if (dq) dq[i] = d;
     qnew[i] = qp[i] + d;
   }

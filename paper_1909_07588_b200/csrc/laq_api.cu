@@ -73,10 +73,14 @@ const char* check_config(const laq_config* c) {
   if (!valid_b(c->b)) return "b must be 1, 2, 3, 4, 8 or 16";
   if (c->D < 1 || c->D > kMaxD) return "D must be in 1..64";
   if (!c->xi) return "xi is null";
+  for (int d = 0; d < c->D; ++d)
+    if (!std::isfinite(c->xi[d]) || c->xi[d] < 0.f) return "every xi_d must be finite and >= 0";
+  if (c->tbar < -1 || c->tbar > 0x7fffffff - 2) return "tbar must be in -1..2^31-3";
   if (!(c->alpha > 0.f) || !std::isfinite(c->alpha)) return "alpha must be positive and finite";
   if (c->clock_mode != 0 && c->clock_mode != 1) return "clock_mode must be 0 or 1";
   if (c->trace_capacity < 0) return "trace_capacity must be >= 0";
-  if (c->flags & ~(uint32_t)(LAQ_FLAG_TRIGGER_OFF | LAQ_FLAG_QUANT_OFF)) return "unknown flag";
+  if (c->flags & ~(uint32_t)(LAQ_FLAG_TRIGGER_OFF | LAQ_FLAG_QUANT_OFF | LAQ_FLAG_STORE_G)) return "unknown flag";
+  if ((c->flags & LAQ_FLAG_STORE_G) && c->model != LAQ_MODEL_SYNTH) return "LAQ_FLAG_STORE_G needs LAQ_MODEL_SYNTH";
   if (c->batch < 0) return "batch must be >= 0";
   if (c->batch > 0 && (c->model == LAQ_MODEL_SYNTH || c->model == LAQ_MODEL_EXTERNAL))
     return "batch > 0 needs a model with samples";
@@ -139,7 +143,7 @@ Plan make_plan(const laq_config& c) {
   pl.theta = take(pl.ps * 4);
   pl.agg = take(pl.ps * 4);
   pl.qp = take(M * pl.ps * 4);
-  pl.g = (c.model == LAQ_MODEL_SYNTH) ? off : take(M * pl.ps * 4);
+  pl.g = (c.model == LAQ_MODEL_SYNTH && !(c.flags & LAQ_FLAG_STORE_G)) ? off : take(M * pl.ps * 4);
   pl.codes = take(M * pl.cw * 4);
   pl.Rbits = take(2 * M * 4);
   pl.norms = take(3 * M * 8);
@@ -206,22 +210,21 @@ bool needs_shards(const laq_ctx* c) {
   return c->cfg.model == LAQ_MODEL_LOGREG_BIN || c->cfg.model == LAQ_MODEL_SOFTMAX || c->cfg.model == LAQ_MODEL_MLP2;
 }
 
+// What the device error word says (bit 0: non-finite gradient or radius; any other bit: a bounded wait ran out).
+laq_status status_of_error_word(laq_ctx* ctx, uint32_t err) {
+  if (err & 1u)
+    return fail(ctx, LAQ_ENONFINITE, "a gradient or radius was not finite; the state is frozen at that iteration");
+  if (err & ~1u)
+    return fail(ctx, LAQ_ETIMEOUT, "a bounded wait on an asynchronous copy or tensor-core stage ran out; the state is frozen at that iteration");
+  return LAQ_OK;
+}
+
 // Reads the device error word after a synchronisation.
 laq_status check_device_error(laq_ctx* ctx) {
   uint32_t err = 0;
   LAQ_CUDA(ctx, cudaMemcpyAsync(&err, &ctx->P.sc->err, 4, cudaMemcpyDeviceToHost, ctx->st));
   LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));
-  if (err & 1u)
-    return fail(ctx, LAQ_ENONFINITE, "a gradient or radius was not finite; the state is frozen at that iteration");
-  if (err & ~1u)
-    return fail(ctx, LAQ_ECUDA, "a bounded wait on an asynchronous copy or tensor-core stage ran out; the state is frozen");
-  return LAQ_OK;
-}
-
-double host_sum_sq(const float* v, long long n) {
-  double s = 0.0;
-  for (long long i = 0; i < n; ++i) s += (double)v[i] * (double)v[i];
-  return s;
+  return status_of_error_word(ctx, err);
 }
 
 }  // namespace
@@ -255,6 +258,9 @@ void enqueue_iteration(laq_ctx* ctx, cudaStream_t st, cudaEvent_t* ev) {
       break;
     case LAQ_MODEL_MLP2:
       ctx->launches += mlp_launch_gradients(ctx->mlp, P, &P.sc->theta_sq, st);
+      break;
+    case LAQ_MODEL_SYNTH:
+      if (c.flags & LAQ_FLAG_STORE_G) ctx->launches += launch_synth_fill(P, st);
       break;
     default: break;
   }
@@ -383,7 +389,7 @@ laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, siz
   P.theta = (float*)(ws + pl.theta);
   P.agg = (float*)(ws + pl.agg);
   P.qp = (float*)(ws + pl.qp);
-  P.g = (c.model == LAQ_MODEL_SYNTH) ? nullptr : (float*)(ws + pl.g);
+  P.g = (c.model == LAQ_MODEL_SYNTH && !(c.flags & LAQ_FLAG_STORE_G)) ? nullptr : (float*)(ws + pl.g);
   P.codes = (uint32_t*)(ws + pl.codes);
   P.Rbits = (uint32_t*)(ws + pl.Rbits);
   P.norms = (double*)(ws + pl.norms);
@@ -412,6 +418,7 @@ laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, siz
   P.seed_hi = (uint32_t)(c.seed >> 32);
   P.batch = c.batch;
   P.zero = 0u;
+  P.starve = 0u;
   P.cz = (float)((double)c.synth_sigma / std::sqrt(21845.0));
   P.eta0 = c.synth_eta0;
   P.X = (const float* const*)(ws + pl.Xptr);
@@ -455,8 +462,7 @@ laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, siz
   LAQ_CUDA(ctx, cudaMemcpyAsync(P.xi, ctx->xi.data(), 4 * (size_t)c.D, cudaMemcpyHostToDevice, ctx->st));
   if (theta0) {
     LAQ_CUDA(ctx, cudaMemcpyAsync(P.theta, theta0, 4 * (size_t)c.p, cudaMemcpyHostToDevice, ctx->st));
-    const double tsq = host_sum_sq(theta0, c.p);
-    LAQ_CUDA(ctx, cudaMemcpyAsync(&P.sc->theta_sq, &tsq, 8, cudaMemcpyHostToDevice, ctx->st));
+    ctx->launches += launch_theta_sq(P, ctx->st);        // ||theta^0||^2 for the regulariser term of the loss
   }
   LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));  // the host vectors above go out of scope
   return LAQ_OK;
@@ -632,9 +638,7 @@ laq_status laq_get_state(laq_ctx* ctx, const laq_state* out) {
     out->counters[1] = (int64_t)sc.uploads;
     out->counters[2] = (int64_t)sc.bits;
   }
-  if (sc.err & 1u)
-    return fail(ctx, LAQ_ENONFINITE, "a gradient or radius was not finite; the state is frozen at that iteration");
-  return LAQ_OK;
+  return status_of_error_word(ctx, sc.err);
 }
 
 laq_status laq_get_worker(laq_ctx* ctx, int32_t m, float* qprev, float* g, uint32_t* codes, float* R) {
@@ -655,7 +659,7 @@ laq_status laq_get_worker(laq_ctx* ctx, int32_t m, float* qprev, float* g, uint3
       LAQ_CUDA(ctx, cudaMemcpyAsync(R, P.Rbits + ((sc.k - 1) & 1ull) * P.M + m, 4, cudaMemcpyDeviceToHost, ctx->st));
   }
   LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));
-  return LAQ_OK;
+  return status_of_error_word(ctx, sc.err);
 }
 
 laq_status laq_set_state(laq_ctx* ctx, const laq_state* in) {
@@ -671,7 +675,6 @@ laq_status laq_set_state(laq_ctx* ctx, const laq_state* in) {
     return cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, ctx->st);
   };
   LAQ_CUDA(ctx, push(P.theta, in->theta, p * 4));
-  if (in->theta) sc.theta_sq = host_sum_sq(in->theta, (long long)p);
   LAQ_CUDA(ctx, push(P.agg, in->agg, p * 4));
   if (in->qprev)
     LAQ_CUDA(ctx, cudaMemcpy2DAsync(P.qp, (size_t)P.ps * 4, in->qprev, p * 4, p * 4, M, cudaMemcpyHostToDevice, ctx->st));
@@ -691,6 +694,7 @@ laq_status laq_set_state(laq_ctx* ctx, const laq_state* in) {
   sc.cnt_quant = sc.cnt_agg = 0;
   LAQ_CUDA(ctx, cudaMemsetAsync(P.Rbits, 0, 2 * M * 4, ctx->st));
   LAQ_CUDA(ctx, cudaMemcpyAsync(P.sc, &sc, sizeof(sc), cudaMemcpyHostToDevice, ctx->st));
+  if (in->theta) ctx->launches += launch_theta_sq(P, ctx->st);   // after the scalars: it overwrites theta_sq
   LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));
   return LAQ_OK;
 }
@@ -707,8 +711,21 @@ laq_status laq_tune(laq_ctx* ctx, const char* key, int32_t value) {
   else if (k == "agg_blocks_per_sm" && value >= 1 && value <= 32) ctx->ls.agg_blocks_per_sm = value;
   else if (k == "grad_blocks_per_worker" && value >= 1 && value <= ctx->gbpw_cap) ctx->gbpw = value;
   else if (k == "graphs" && (value == 0 || value == 1)) ctx->graphs_enabled = value != 0;
+  else if (k == "starve_copies" && (value == 0 || value == 1)) ctx->P.starve = (uint32_t)value;
   else return fail(ctx, LAQ_EINVAL, "unknown tuning key or value outside its limits");
   drop_graphs(ctx);     // captured launch shapes are stale
+  return LAQ_OK;
+}
+
+laq_status laq_query(const laq_ctx* ctx, const char* key, int64_t* value) {
+  if (!ctx || !ctx->ws || !key || !value) return LAQ_EINVAL;
+  const std::string k(key);
+  if (k == "sweep_blocks_per_worker") *value = sweep_blocks_per_worker(ctx->P, ctx->ls);
+  else if (k == "sweep_threads") *value = ctx->ls.sweep_threads;
+  else if (k == "sweep_tile_groups") *value = sweep_tile_groups();
+  else if (k == "aggregate_blocks") *value = aggregate_blocks(ctx->P, ctx->ls);
+  else if (k == "grad_blocks_per_worker") *value = ctx->gbpw;
+  else return LAQ_EINVAL;
   return LAQ_OK;
 }
 

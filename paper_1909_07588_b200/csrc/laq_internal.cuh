@@ -68,6 +68,7 @@ struct Params {
   uint32_t seed_lo, seed_hi;
   int batch;                 // 0: full local gradients; > 0: minibatch size per worker
   uint32_t zero;             // always 0; opaque to the compiler (used to order a store after a load)
+  uint32_t starve;           // test hook (laq_tune "starve_copies"): one loader issues no copies, see laq.h
   float cz, eta0;
   // shards
   long long Ntot;
@@ -111,6 +112,7 @@ __device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
 // returns false; the caller records kErrRingWait in DevScalars::err, stops using the ring, and gives the copies
 // still in flight the same bounded time to land before it leaves.
 constexpr uint32_t kRingWaitLimit = 1u << 22;
+constexpr uint32_t kStarvedWaitLimit = 1u << 10;   // polls of a consumer whose loader was told to issue nothing
 constexpr uint32_t kErrRingWait = 16u;             // bit of DevScalars::err: a wait on a staged tile ran out
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -144,8 +146,8 @@ __device__ __forceinline__ bool ring_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded: false once the limit is reached (the caller records it and stops using the ring).
-__device__ __forceinline__ bool ring_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t it = 0; it < kRingWaitLimit; ++it) {
+__device__ __forceinline__ bool ring_wait(uint32_t bar, uint32_t parity, uint32_t limit = kRingWaitLimit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (ring_try_wait(bar, parity)) return true;
     if (it > 64) __nanosleep(64);
   }
@@ -214,6 +216,8 @@ struct LaunchShape {
 };
 
 // kernels' host-side launchers (each returns the number of kernels it launched)
+bool generated_in_sweeps(const Params& P);
+int launch_synth_fill(const Params& P, cudaStream_t st);
 int launch_radius(const Params& P, const LaunchShape& ls, cudaStream_t st);
 bool small_iteration_applies(const Params& P);
 int launch_small_iteration(const Params& P, int gbpw_finalize, cudaStream_t st);
@@ -242,6 +246,8 @@ int mlp_convert_shard(MlpPlan& mp, const Params& P, int m, const float* X, long 
 int mlp_launch_gradients(MlpPlan& mp, const Params& P, const double* theta_sq, cudaStream_t st);
 void mlp_teardown(MlpPlan& mp);
 int sweep_blocks_per_worker(const Params& P, const LaunchShape& ls);
+int sweep_tile_groups();
+int launch_theta_sq(const Params& P, cudaStream_t st);
 int aggregate_blocks(const Params& P, const LaunchShape& ls);
 
 }  // namespace laq

@@ -18,6 +18,8 @@
 // device asks the runtime for the real address (cudaGetSymbolAddress with that device current),
 // checks the result, caches it, and passes it to the kernels.  That first call also loads the
 // module onto the device, so make it once during start-up, before any stream capture begins.
+// The cached address belongs to the device's primary context: a host that destroys that context
+// (cudaDeviceReset) must not call this entry point on the device again in the same process.
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -92,7 +94,7 @@ __global__ void __launch_bounds__(kThreads) static_quantize_kernel(const float* 
   __shared__ bool is_last;
   const uint32_t rb = sc->r_bits;
   const float R = __uint_as_float(rb);
-  const bool finite = rb < 0x7f800000u, live = finite && R > 0.f;
+  const bool finite = rb < 0x7f800000u, live = finite && R > 0.f;   // R = 0: all codes 0, both norms 0
   const float levels = (float)((1u << B) - 1u);
   const float s = __fmul_rn(__fmul_rn(2.0f, __fdiv_rn(1.0f, levels)), R);
   double sdq = 0.0, seps = 0.0;
@@ -105,8 +107,8 @@ __global__ void __launch_bounds__(kThreads) static_quantize_kernel(const float* 
       if (live && i < p) {
         const float gi = __ldg(g + i), qi = __ldg(q + i);
         const float d = __fsub_rn(gi, qi);
-        const float t = __fadd_rn(__fdiv_rn(__fadd_rn(d, R), s), 0.5f);
-        const float f = fminf(fmaxf(floorf(t), 0.f), levels);
+        // a grid step that underflowed to zero makes Eq. (5) x / 0: code 0, as for R = 0
+        const float f = s > 0.f ? fminf(fmaxf(floorf(__fadd_rn(__fdiv_rn(__fadd_rn(d, R), s), 0.5f)), 0.f), levels) : 0.f;
         const float dq = __fsub_rn(__fmul_rn(s, f), R);
         const float e_ = __fsub_rn(gi, __fadd_rn(qi, dq));
         sdq = fma((double)dq, (double)dq, sdq);
@@ -160,6 +162,15 @@ extern "C" laq_status laq_quantize_worker_static(const float* d_g, const float* 
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
     return set_err(errbuf, errbuf_len, LAQ_ECUDA, "no current CUDA device (or device ordinal >= 64)");
+  // the scratch used is the current device's: inputs that live on another GPU would make the kernels run there
+  // against this device's scratch address
+  cudaPointerAttributes attr;
+  if (cudaPointerGetAttributes(&attr, d_g) != cudaSuccess) {
+    cudaGetLastError();
+    return set_err(errbuf, errbuf_len, LAQ_EINVAL, "d_g is not a pointer the CUDA runtime knows");
+  }
+  if ((attr.type == cudaMemoryTypeDevice || attr.type == cudaMemoryTypeManaged) && attr.device != dev)
+    return set_err(errbuf, errbuf_len, LAQ_EINVAL, "the buffers live on another GPU than the current device: make their device current for the call");
   StaticScratch* sc = nullptr;
   {
     std::lock_guard<std::mutex> lock(g_mutex);

@@ -99,6 +99,32 @@ __device__ __forceinline__ double block_sum(double v, double* sh /* >= 32 double
 #endif
 constexpr int kUnroll = LAQ_SWEEP_UNROLL;  // 16-byte groups in flight per thread
 
+// ||theta||^2 of the iterate in memory (set by the caller: theta^0, or a restored state) into DevScalars::theta_sq,
+// which the kernels otherwise keep up to date themselves.  One block, fp64, fixed order.
+__global__ void __launch_bounds__(1024) theta_sq_kernel(const Params P) {
+  __shared__ double sh[32];
+  double t = 0.0;
+  for (long long i = threadIdx.x; i < P.p; i += blockDim.x) t = fma((double)P.theta[i], (double)P.theta[i], t);
+  t = block_sum(t, sh);
+  if (threadIdx.x == 0) P.sc->theta_sq = t;
+}
+
+// ------------------------------------------------------------------------------------------------
+// LAQ_FLAG_STORE_G with LAQ_MODEL_SYNTH: the workers' gradients of the iteration are written to memory first
+// (this kernel is then step 1 of the iteration) and the sweeps read them from there, as they do downstream of
+// a real gradient kernel.  Padding coordinates are written as zeros.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) synth_fill_kernel(const Params P) {
+  if (*(volatile uint32_t*)&P.sc->err) return;
+  const int m = blockIdx.y;
+  Synth sy;
+  sy.init(P, m, P.sc->k + 1);
+  float4* __restrict__ g4 = reinterpret_cast<float4*>(P.g + (long long)m * P.ps);
+  const uint32_t nv = (uint32_t)P.nv, v_full = (uint32_t)(P.p >> 2), stride = gridDim.x * blockDim.x;
+  for (uint32_t v = blockIdx.x * blockDim.x + threadIdx.x; v < nv; v += stride)
+    g4[v] = v < v_full ? sy.at4(v) : sy.at4_masked(v, P.p);
+}
+
 // ------------------------------------------------------------------------------------------------
 // radius
 // ------------------------------------------------------------------------------------------------
@@ -243,16 +269,26 @@ __device__ __forceinline__ float div_by_reciprocal(float x, float s, float y) {
 }
 
 // One coordinate of Eq. (5)/(6).  Returns 2^23 + code as a float bit pattern (code in the low bits);
-// updates the two fp64 sums.  No clamp: |d| <= R bounds floor(t) by 2^b - 1 (t <= 2^b - 1/2 + rounding).
+// updates the two fp64 sums.
+// FAST (2^-60 <= s <= 2^60): no clamp, |d| <= R bounds floor(t) by 2^b - 1 (t <= 2^b - 1/2 + rounding).
+// Otherwise the grid step s = 2 tau R may be subnormal or zero although R > 0: the quotient then loses bits (or
+// is x / 0) and floor(t) can leave [0, 2^b - 1], so the code is clamped to that range as Eq. (5) defines it, and
+// s = 0 gives code 0 (the 0/0 reading used for R = 0).  Eq. (6) is applied as printed in every case.
 template <bool FAST>
-__device__ __forceinline__ uint32_t quantize_one(float g, float q, float R, float s, float y, double& sdq,
-                                                 double& seps) {
+__device__ __forceinline__ uint32_t quantize_one(float g, float q, float R, float s, float y, float levels,
+                                                 double& sdq, double& seps) {
   const float d = __fsub_rn(g, q);
   const float x = __fadd_rn(d, R);
-  const float u = FAST ? div_by_reciprocal(x, s, y) : __fdiv_rn(x, s);
-  const float t = __fadd_rn(u, 0.5f);
-  const float fl = __fadd_rd(t, 8388608.0f);        // 2^23 + floor(t): rounding down at unit spacing
-  const float f = __fsub_rn(fl, 8388608.0f);        // floor(t), exact
+  float fl, f;
+  if (FAST) {
+    const float t = __fadd_rn(div_by_reciprocal(x, s, y), 0.5f);
+    fl = __fadd_rd(t, 8388608.0f);                  // 2^23 + floor(t): rounding down at unit spacing
+    f = __fsub_rn(fl, 8388608.0f);                  // floor(t), exact
+  } else {
+    f = 0.f;
+    if (s > 0.f) f = fminf(fmaxf(floorf(__fadd_rn(__fdiv_rn(x, s), 0.5f)), 0.f), levels);
+    fl = __fadd_rn(f, 8388608.0f);
+  }
   const float dq = __fsub_rn(__fmul_rn(s, f), R);   // Eq. (6): multiply, then subtract
   const float qn = __fadd_rn(q, dq);
   const float e = __fsub_rn(g, qn);
@@ -426,10 +462,12 @@ __device__ void trigger_stage(const Params& P, int bpw, unsigned char* scratch) 
 }
 
 // ---- asynchronous staging of a row through shared memory (quantize sweep over long rows) -----------------------
-// Every warp owns a ring of kRingStages tiles of kRingGroups 16-byte groups of its row of Q_prev.  One lane asks the
-// copy engine for a tile (cp.async.bulk, completion counted in bytes on the stage's mbarrier) kRingStages tiles ahead
-// of the one being worked on, so the loads in flight live in shared memory instead of in registers and no warp
-// waits on a load it has just issued.  A stage is refilled after __syncwarp(): every lane has then read its groups.
+// Every warp owns a ring of kRingStages stages; a stage holds one tile of kRingGroups 16-byte groups of the warp's
+// row of Q_prev and, when the gradients are read from memory, the same tile of g behind it.  One lane asks the
+// copy engine for a stage's tiles (cp.async.bulk, completion counted in bytes on the stage's mbarrier) kRingStages
+// tiles ahead of the one being worked on, so the loads in flight live in shared memory instead of in registers and
+// no warp waits on a load it has just issued.  A stage is refilled after __syncwarp(): every lane has then read
+// its groups.
 #ifndef LAQ_RING_STAGES
 #define LAQ_RING_STAGES 2
 #endif
@@ -439,16 +477,23 @@ __device__ void trigger_stage(const Params& P, int bpw, unsigned char* scratch) 
 constexpr int kRingStages = LAQ_RING_STAGES;
 constexpr int kRingU = LAQ_RING_U;                 // groups per lane and tile
 constexpr uint32_t kRingGroups = 32 * kRingU;      // 16-byte groups per tile (4 KB)
+constexpr uint32_t kRingTileBytes = kRingGroups * 16;
 constexpr int kRingMaxWarps = 16;                  // warps per block that can own a ring
+// rows read from memory take the ring from this many coordinates on (shorter rows: the plain loop), in blocks of
+// up to 8 warps (two tiles per stage: more warps would not fit the shared memory of an SM)
+constexpr long long kRingMinStoredP = 1ll << 20;
+__host__ __device__ constexpr bool stored_rows_take_ring(long long p, int threads) {
+  return p >= kRingMinStoredP && threads <= 256;
+}
 
 // The per-worker sweep of quantize_kernel (R > 0).  FAST selects the reciprocal-based exact division.
 // Groups [0, nv_main) lie wholly inside the row and run without masks; the few groups after them are
 // handled by the first warp of the worker's first block with per-coordinate masks.  nv_main is even (a multiple
 // of 8 for b = 3), so the lane pairs of the 1-bit packing (the lane octets of the 3-bit packing) never straddle
 // the two parts.
-// RING (rows generated in the kernel, FAST): the full tiles of the row come through the warp's shared-memory ring
-// (ring = the block's dynamic shared memory, bars = kRingStages mbarriers per warp); what is left of the main part
-// (less than one tile) goes through the plain loop below.
+// RING (FAST; rows generated in the kernel, or long rows read from memory): the full tiles of the row come through
+// the warp's shared-memory ring (ring = the block's dynamic shared memory, bars = kRingStages mbarriers per warp);
+// what is left of the main part (less than one tile) goes through the plain loop below.
 template <bool SYNTH, int B, bool FAST, bool RING>
 __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned long long k, float R, float s,
                                                double& sdq, double& seps, unsigned char* ring = nullptr,
@@ -456,6 +501,7 @@ __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned 
   Synth sy;
   if (SYNTH) sy.init(P, m, k + 1);
   const float y = __fdiv_rn(1.0f, s), cy = __fmul_rn(R, y);
+  const float levels = (float)((1u << B) - 1u);
   const float4* __restrict__ q4 = reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps);
   const float4* __restrict__ g4 = SYNTH ? nullptr : reinterpret_cast<const float4*>(P.g + (long long)m * P.ps);
   uint32_t* row = P.codes + (long long)m * P.cw;
@@ -469,30 +515,41 @@ __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned 
 #pragma unroll
   for (int c = 0; c < NC; ++c) adq[c] = aeps[c] = 0.0;
   if constexpr (RING) {
+    constexpr uint32_t NS = SYNTH ? 1u : 2u;                              // tiles per stage: Q_prev (and g)
+    constexpr uint32_t kStageBytes = NS * kRingTileBytes;
     const uint32_t w = threadIdx.x >> 5, wpb = blockDim.x >> 5;
     const uint32_t gw = blockIdx.x * wpb + w, nw = gridDim.x * wpb;      // this warp among the worker's warps
     const uint32_t n_tiles = nv_main / kRingGroups;
     const uint32_t n_my = n_tiles > gw ? (n_tiles - gw + nw - 1) / nw : 0u;  // tiles gw, gw + nw, ...
-    const float4* stage0 = reinterpret_cast<const float4*>(ring) + (size_t)w * kRingStages * kRingGroups;
+    const float4* stage0 = reinterpret_cast<const float4*>(ring) + (size_t)w * kRingStages * NS * kRingGroups;
     const uint32_t stage_a = smem_addr(stage0), bar_a = smem_addr(bars + w * kRingStages);
-    constexpr uint32_t kTileBytes = kRingGroups * 16;
+    // test hook: this one warp issues no copies and polls with a short limit, so its waits run out with
+    // nothing in flight (see laq_tune "starve_copies")
+    const bool starved = P.starve != 0u && m == 0 && gw == 0;
+    const uint32_t wait_limit = starved ? kStarvedWaitLimit : kRingWaitLimit;
+    auto fetch = [&](uint32_t stage, size_t first_group) {
+      const uint32_t dst = stage_a + stage * kStageBytes, bar = bar_a + 8 * stage;
+      ring_expect(bar, kStageBytes);
+      ring_copy(dst, q4 + first_group, kRingTileBytes, bar);
+      if constexpr (!SYNTH) ring_copy(dst + kRingTileBytes, g4 + first_group, kRingTileBytes, bar);
+    };
     if (lane == 0) {
       for (int st = 0; st < kRingStages; ++st) ring_bar_init(bar_a + 8 * st);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      for (uint32_t i = 0; i < (uint32_t)kRingStages && i < n_my; ++i)
-        ring_fetch(stage_a + i * kTileBytes, q4 + (size_t)(gw + i * nw) * kRingGroups, kTileBytes, bar_a + 8 * i);
+      if (!starved)
+        for (uint32_t i = 0; i < (uint32_t)kRingStages && i < n_my; ++i) fetch(i, (size_t)(gw + i * nw) * kRingGroups);
     }
     __syncwarp();
-    // per-lane state that advances by a constant per tile: first group of the tile for this lane, source of the
-    // tile kRingStages ahead, byte offset of the current stage
+    // per-lane state that advances by a constant per tile: first group of the tile for this lane, first group of
+    // the tile kRingStages ahead, the current stage
     uint32_t v0 = gw * kRingGroups + lane;
-    const float4* src_ahead = q4 + (size_t)(gw + (uint32_t)kRingStages * nw) * kRingGroups;
+    size_t ahead = (size_t)(gw + (uint32_t)kRingStages * nw) * kRingGroups;
     const uint32_t step_groups = nw * kRingGroups;
     uint32_t st = 0, parity = 0, done = 0;
     for (; done < n_my; ++done) {
-      if (!__all_sync(0xffffffffu, ring_wait(bar_a + 8 * st, parity))) break;
-      const float4* tile = stage0 + st * kRingGroups + lane;
+      if (!__all_sync(0xffffffffu, ring_wait(bar_a + 8 * st, parity, wait_limit))) break;
+      const float4* tile = stage0 + st * (NS * kRingGroups) + lane;
       uint32_t* out = row + v0;
       // the 4 kRingU coordinates of a lane in this tile are summed in fp32 (fused multiply-adds, 4 kRingU - 1
       // roundings: relative error of the run below 4 kRingU * 2^-24) and the run is then added in fp64; with
@@ -501,15 +558,17 @@ __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned 
 #pragma unroll
       for (int j = 0; j < kRingU; ++j) {
         const float4 q = tile[32 * j];
-        const float4 g = sy.at4(v0 + 32 * j);
+        float4 g;
+        if constexpr (SYNTH) g = sy.at4(v0 + 32 * j);
+        else g = tile[kRingGroups + 32 * j];
         uint32_t yy[4];
         if constexpr (B <= 8) {
           quantize_group<B>(g, q, R, s, y, cy, rdq, reps, yy);
         } else {
-          yy[0] = quantize_one<true>(g.x, q.x, R, s, y, adq[0 % NC], aeps[0 % NC]);
-          yy[1] = quantize_one<true>(g.y, q.y, R, s, y, adq[1 % NC], aeps[1 % NC]);
-          yy[2] = quantize_one<true>(g.z, q.z, R, s, y, adq[2 % NC], aeps[2 % NC]);
-          yy[3] = quantize_one<true>(g.w, q.w, R, s, y, adq[3 % NC], aeps[3 % NC]);
+          yy[0] = quantize_one<true>(g.x, q.x, R, s, y, levels, adq[0 % NC], aeps[0 % NC]);
+          yy[1] = quantize_one<true>(g.y, q.y, R, s, y, levels, adq[1 % NC], aeps[1 % NC]);
+          yy[2] = quantize_one<true>(g.z, q.z, R, s, y, levels, adq[2 % NC], aeps[2 % NC]);
+          yy[3] = quantize_one<true>(g.w, q.w, R, s, y, levels, adq[3 % NC], aeps[3 % NC]);
         }
         if constexpr (B == 8) out[32 * j] = __byte_perm(__byte_perm(yy[0], yy[1], 0x0040), __byte_perm(yy[2], yy[3], 0x0040), 0x5410);
         else store_codes<B>(row, v0 + 32 * j, yy[0], yy[1], yy[2], yy[3], true, P.cw);
@@ -519,8 +578,8 @@ __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned 
         aeps[0] += (double)reps;
       }
       __syncwarp();                                // every lane has read its groups: the stage may be refilled
-      if (lane == 0 && done + kRingStages < n_my) ring_fetch(stage_a + st * kTileBytes, src_ahead, kTileBytes, bar_a + 8 * st);
-      src_ahead += step_groups;
+      if (lane == 0 && done + kRingStages < n_my) fetch(st, ahead);
+      ahead += step_groups;
       v0 += step_groups;
       if (++st == (uint32_t)kRingStages) {
         st = 0;
@@ -528,12 +587,12 @@ __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned 
       }
     }
     if (done < n_my) {
-      // a wait ran out: record it, and before leaving give the copies still in flight (at most kRingStages tiles,
+      // a wait ran out: record it, and before leaving give the copies still in flight (at most kRingStages stages,
       // this one included) the same bounded time to land, so that none writes into shared memory of a later block
       if (lane == 0) atomicOr(&P.sc->err, kErrRingWait);
       const uint32_t issued = min(n_my, done + (uint32_t)kRingStages);
       for (uint32_t i = done; i < issued; ++i) {
-        ring_wait(bar_a + 8 * st, parity);
+        ring_wait(bar_a + 8 * st, parity, wait_limit);
         if (++st == (uint32_t)kRingStages) {
           st = 0;
           parity ^= 1u;
@@ -558,10 +617,10 @@ __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned 
         quantize_group<B>(g[j], q[j], R, s, y, cy, adq[0], aeps[0], yy);
         store_codes<B>(row, v + j * stride, yy[0], yy[1], yy[2], yy[3], true, P.cw);
       } else {
-        const uint32_t y0 = quantize_one<FAST>(g[j].x, q[j].x, R, s, y, adq[0 % NC], aeps[0 % NC]);
-        const uint32_t y1 = quantize_one<FAST>(g[j].y, q[j].y, R, s, y, adq[1 % NC], aeps[1 % NC]);
-        const uint32_t y2 = quantize_one<FAST>(g[j].z, q[j].z, R, s, y, adq[2 % NC], aeps[2 % NC]);
-        const uint32_t y3 = quantize_one<FAST>(g[j].w, q[j].w, R, s, y, adq[3 % NC], aeps[3 % NC]);
+        const uint32_t y0 = quantize_one<FAST>(g[j].x, q[j].x, R, s, y, levels, adq[0 % NC], aeps[0 % NC]);
+        const uint32_t y1 = quantize_one<FAST>(g[j].y, q[j].y, R, s, y, levels, adq[1 % NC], aeps[1 % NC]);
+        const uint32_t y2 = quantize_one<FAST>(g[j].z, q[j].z, R, s, y, levels, adq[2 % NC], aeps[2 % NC]);
+        const uint32_t y3 = quantize_one<FAST>(g[j].w, q[j].w, R, s, y, levels, adq[3 % NC], aeps[3 % NC]);
         store_codes<B>(row, v + j * stride, y0, y1, y2, y3, true, P.cw);
       }
     }
@@ -586,10 +645,10 @@ __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned 
       g = SYNTH ? sy.at4(v) : __ldg(g4 + v);
     }
     double a = 0.0, c = 0.0;
-    const uint32_t y0 = quantize_one<FAST>(g.x, q.x, R, s, y, a, c);
-    const uint32_t y1 = quantize_one<FAST>(g.y, q.y, R, s, y, a, c);
-    const uint32_t y2 = quantize_one<FAST>(g.z, q.z, R, s, y, a, c);
-    const uint32_t y3 = quantize_one<FAST>(g.w, q.w, R, s, y, a, c);
+    const uint32_t y0 = quantize_one<FAST>(g.x, q.x, R, s, y, levels, a, c);
+    const uint32_t y1 = quantize_one<FAST>(g.y, q.y, R, s, y, levels, a, c);
+    const uint32_t y2 = quantize_one<FAST>(g.z, q.z, R, s, y, levels, a, c);
+    const uint32_t y3 = quantize_one<FAST>(g.w, q.w, R, s, y, levels, a, c);
     if (ok) {
       sdq += a;
       seps += c;
@@ -606,7 +665,7 @@ __device__ __forceinline__ void quantize_sweep(const Params& P, int m, unsigned 
       const float gg[4] = {g.x, g.y, g.z, g.w}, qq[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
       for (int e = 0; e < 4; ++e)
-        if (4ll * v + e < p) yy[e] = quantize_one<FAST>(gg[e], qq[e], R, s, y, sdq, seps);
+        if (4ll * v + e < p) yy[e] = quantize_one<FAST>(gg[e], qq[e], R, s, y, levels, sdq, seps);
     }
     store_codes<B>(row, v, yy[0], yy[1], yy[2], yy[3], ok, P.cw);
   }
@@ -624,8 +683,8 @@ template <bool SYNTH, int B>
 __global__ void __launch_bounds__(LAQ_QUANT_MAX_THREADS, LAQ_QUANT_MIN_BLOCKS) quantize_kernel(const Params P) {
   __shared__ double sh[32];
   __shared__ bool is_last;
-  __shared__ __align__(8) unsigned long long ring_bars[SYNTH ? kRingMaxWarps * kRingStages : 1];
-  // dynamic shared memory: the trigger stage's scratch and, for SYNTH, kRingStages tiles per warp (the larger of both)
+  __shared__ __align__(8) unsigned long long ring_bars[kRingMaxWarps * kRingStages];
+  // dynamic shared memory: the trigger stage's scratch and the warps' staging rings (the larger of both)
   extern __shared__ __align__(128) unsigned char ring_smem[];
   const int m = blockIdx.y;
   const bool frozen = *(volatile uint32_t*)&P.sc->err != 0;
@@ -639,9 +698,12 @@ __global__ void __launch_bounds__(LAQ_QUANT_MAX_THREADS, LAQ_QUANT_MIN_BLOCKS) q
     const float s = __fmul_rn(__fmul_rn(2.0f, __fdiv_rn(1.0f, levels)), R);
     if (!(R > 0.f))
       zero_codes<B>(P, m);
-    else if (s >= 0x1p-60f && s <= 0x1p60f)
-      quantize_sweep<SYNTH, B, true, SYNTH>(P, m, k, R, s, sdq, seps, ring_smem, ring_bars);
-    else
+    else if (s >= 0x1p-60f && s <= 0x1p60f) {
+      if (SYNTH || stored_rows_take_ring(P.p, (int)blockDim.x))
+        quantize_sweep<SYNTH, B, true, true>(P, m, k, R, s, sdq, seps, ring_smem, ring_bars);
+      else if constexpr (!SYNTH)
+        quantize_sweep<SYNTH, B, true, false>(P, m, k, R, s, sdq, seps);
+    } else
       quantize_sweep<SYNTH, B, false, false>(P, m, k, R, s, sdq, seps);
   }
   const double tdq = block_sum(sdq, sh);
@@ -1049,8 +1111,8 @@ __global__ void __launch_bounds__(kSmallThreads) small_iteration_kernel(const Pa
 #pragma unroll
           for (int e = 0; e < 4; ++e)
             if (4ll * v + e < p)
-              yy[e] = fast ? quantize_one<true>(gg[e], qq[e], R, s, y, sdq, seps)
-                           : quantize_one<false>(gg[e], qq[e], R, s, y, sdq, seps);
+              yy[e] = fast ? quantize_one<true>(gg[e], qq[e], R, s, y, levels, sdq, seps)
+                           : quantize_one<false>(gg[e], qq[e], R, s, y, levels, sdq, seps);
         }
         store_codes<B>(row, v, yy[0], yy[1], yy[2], yy[3], ok, P.cw);
       }
@@ -1202,8 +1264,10 @@ void launch_quant_one(const Params& P, dim3 grid, int threads, size_t smem, cuda
 
 template <bool SYNTH>
 void launch_quant_b(const Params& P, dim3 grid, int threads, cudaStream_t st) {
-  // rows generated in the kernel: every warp stages its tiles of Q_prev through a ring in dynamic shared memory
-  const size_t ring = SYNTH ? (size_t)(threads / 32) * kRingStages * kRingGroups * 16 : 0;
+  // rows generated in the kernel, long rows read from memory: every warp stages its tiles of Q_prev (and of g)
+  // through a ring in dynamic shared memory
+  const size_t ring = SYNTH ? (size_t)(threads / 32) * kRingStages * kRingTileBytes
+                            : (stored_rows_take_ring(P.p, threads) ? (size_t)(threads / 32) * kRingStages * 2 * kRingTileBytes : 0);
   const size_t smem = ring > kTriggerScratchBytes ? ring : kTriggerScratchBytes;
   switch (P.b) {
     case 1: launch_quant_one<SYNTH, 1>(P, grid, threads, smem, st); break;
@@ -1235,6 +1299,23 @@ int aggregate_blocks(const Params& P, const LaunchShape& ls) {
   return (int)(nb < 1 ? 1 : nb);
 }
 
+int sweep_tile_groups() { return (int)kRingGroups; }
+
+int launch_theta_sq(const Params& P, cudaStream_t st) {
+  theta_sq_kernel<<<1, 1024, 0, st>>>(P);
+  return 1;
+}
+
+bool generated_in_sweeps(const Params& P) { return P.model == LAQ_MODEL_SYNTH && !(P.flags & LAQ_FLAG_STORE_G); }
+
+int launch_synth_fill(const Params& P, cudaStream_t st) {
+  long long nb = (P.nv + 256 * 8 - 1) / (256 * 8);
+  const long long cap = ((long long)kNumSMs * 16 + P.M - 1) / P.M;
+  if (nb > cap) nb = cap;
+  synth_fill_kernel<<<dim3((unsigned)(nb < 1 ? 1 : nb), P.M), 256, 0, st>>>(P);
+  return 1;
+}
+
 bool small_iteration_applies(const Params& P) {
   return P.model != LAQ_MODEL_SYNTH && !(P.flags & LAQ_FLAG_QUANT_OFF) && (long long)P.M * P.ps <= 8192;
 }
@@ -1253,7 +1334,7 @@ int launch_small_iteration(const Params& P, int gbpw_finalize, cudaStream_t st) 
 
 int launch_radius(const Params& P, const LaunchShape& ls, cudaStream_t st) {
   dim3 grid(sweep_blocks_per_worker(P, ls), P.M);
-  if (P.model == LAQ_MODEL_SYNTH)
+  if (generated_in_sweeps(P))
     radius_kernel<true><<<grid, ls.sweep_threads, 0, st>>>(P);
   else
     radius_kernel<false><<<grid, ls.sweep_threads, 0, st>>>(P);
@@ -1262,7 +1343,7 @@ int launch_radius(const Params& P, const LaunchShape& ls, cudaStream_t st) {
 
 int launch_innovation_trigger(const Params& P, const LaunchShape& ls, cudaStream_t st) {
   dim3 grid(sweep_blocks_per_worker(P, ls), P.M);
-  if (P.model == LAQ_MODEL_SYNTH)
+  if (generated_in_sweeps(P))
     innovation_kernel<true><<<grid, ls.sweep_threads, 0, st>>>(P);
   else
     innovation_kernel<false><<<grid, ls.sweep_threads, 0, st>>>(P);
@@ -1271,7 +1352,7 @@ int launch_innovation_trigger(const Params& P, const LaunchShape& ls, cudaStream
 
 int launch_quantize_trigger(const Params& P, const LaunchShape& ls, cudaStream_t st) {
   dim3 grid(sweep_blocks_per_worker(P, ls), P.M);
-  if (P.model == LAQ_MODEL_SYNTH)
+  if (generated_in_sweeps(P))
     launch_quant_b<true>(P, grid, ls.sweep_threads, st);
   else
     launch_quant_b<false>(P, grid, ls.sweep_threads, st);
@@ -1281,7 +1362,7 @@ int launch_quantize_trigger(const Params& P, const LaunchShape& ls, cudaStream_t
 int launch_aggregate(const Params& P, const LaunchShape& ls, cudaStream_t st) {
   const int nb = aggregate_blocks(P, ls);
   if (P.flags & LAQ_FLAG_QUANT_OFF) {
-    if (P.model == LAQ_MODEL_SYNTH)
+    if (generated_in_sweeps(P))
       aggregate_raw_kernel<true><<<nb, ls.agg_threads, 0, st>>>(P);
     else
       aggregate_raw_kernel<false><<<nb, ls.agg_threads, 0, st>>>(P);

@@ -11,14 +11,15 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "csrc", "liblaq_b200.so")
 
-LAQ_OK, LAQ_EINVAL, LAQ_EWORKSPACE, LAQ_ECUDA, LAQ_ENONFINITE, LAQ_ESTATE = range(6)
-STATUS_NAMES = ["LAQ_OK", "LAQ_EINVAL", "LAQ_EWORKSPACE", "LAQ_ECUDA", "LAQ_ENONFINITE", "LAQ_ESTATE"]
+LAQ_OK, LAQ_EINVAL, LAQ_EWORKSPACE, LAQ_ECUDA, LAQ_ENONFINITE, LAQ_ESTATE, LAQ_ETIMEOUT = range(7)
+STATUS_NAMES = ["LAQ_OK", "LAQ_EINVAL", "LAQ_EWORKSPACE", "LAQ_ECUDA", "LAQ_ENONFINITE", "LAQ_ESTATE", "LAQ_ETIMEOUT"]
 MODEL_LOGREG_BIN, MODEL_SOFTMAX, MODEL_MLP2, MODEL_SYNTH, MODEL_EXTERNAL = range(5)
 FLAG_QUANT_OFF = 1
 FLAG_TRIGGER_OFF = 2
+FLAG_STORE_G = 4
 
 EXPORTS = ["laq_workspace_bytes", "laq_init", "laq_load_shards", "laq_set_gradients", "laq_step", "laq_sync",
-           "laq_get_state", "laq_get_worker", "laq_set_state", "laq_kernel_launches", "laq_tune", "laq_set_profiling", "laq_kernel_times", "laq_quantize_worker_static", "laq_last_error", "laq_destroy"]
+           "laq_get_state", "laq_get_worker", "laq_set_state", "laq_kernel_launches", "laq_tune", "laq_query", "laq_set_profiling", "laq_kernel_times", "laq_quantize_worker_static", "laq_last_error", "laq_destroy"]
 
 
 class LaqError(RuntimeError):
@@ -73,6 +74,7 @@ def load_library():
     L.laq_kernel_launches.argtypes = [C.c_void_p]
     L.laq_kernel_launches.restype = C.c_int64
     L.laq_tune.argtypes = [C.c_void_p, C.c_char_p, C.c_int32]
+    L.laq_query.argtypes = [C.c_void_p, C.c_char_p, C.POINTER(C.c_int64)]
     L.laq_set_profiling.argtypes = [C.c_void_p, C.c_int32]
     L.laq_kernel_times.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
     L.laq_quantize_worker_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p,
@@ -247,6 +249,13 @@ class Laq:
     def tune(self, key, value):
         self._check(self._L.laq_tune(self._h, key.encode(), int(value)))
 
+    def query(self, key):
+        v = C.c_int64(0)
+        st = self._L.laq_query(self._h, key.encode(), C.byref(v))
+        if st != LAQ_OK:
+            raise LaqError(st, "unknown query key %r" % key)
+        return int(v.value)
+
 
 def from_workload(w, trace_capacity=0, stream=None, **overrides):
     """Build a context from a ``workloads.Workload`` and make its shards resident."""
@@ -274,10 +283,11 @@ def quantize_worker_static(g, qprev, b, codes, R, norms, stream=None):
     assert norms.dtype == torch.float64 and norms.numel() >= 2 and codes.element_size() == 4
     p = g.numel()
     assert qprev.numel() == p and codes.numel() >= (p * b + 31) // 32
-    st = stream if stream is not None else torch.cuda.current_stream(g.device)
     err = C.create_string_buffer(256)
-    rc = L.laq_quantize_worker_static(C.c_void_p(g.data_ptr()), C.c_void_p(qprev.data_ptr()), p, b,
-                                      C.c_void_p(codes.data_ptr()), C.c_void_p(R.data_ptr()),
-                                      C.c_void_p(norms.data_ptr()), C.c_void_p(st.cuda_stream), err, 256)
+    with torch.cuda.device(g.device):        # the library uses the scratch of the calling thread's current device
+        st = stream if stream is not None else torch.cuda.current_stream(g.device)
+        rc = L.laq_quantize_worker_static(C.c_void_p(g.data_ptr()), C.c_void_p(qprev.data_ptr()), p, b,
+                                          C.c_void_p(codes.data_ptr()), C.c_void_p(R.data_ptr()),
+                                          C.c_void_p(norms.data_ptr()), C.c_void_p(st.cuda_stream), err, 256)
     if rc != LAQ_OK:
         raise LaqError(rc, err.value.decode())

@@ -229,16 +229,106 @@ def test_synthetic_stream_short_rows_and_all_code_widths(b, M, p):
     ctx.close()
 
 
+def _tiles_per_warp(ctx):
+    """Staged tiles each warp of the quantize sweep owns (at least), from the launch plan the library reports."""
+    groups = ctx.query("sweep_tile_groups")
+    warps = ctx.query("sweep_blocks_per_worker") * (ctx.query("sweep_threads") // 32)
+    return (ctx.p // 4) // groups // warps
+
+
+@pytest.mark.parametrize("b", [2, 3, 4, 8])
+@pytest.mark.parametrize("M,p", [(64, 2_000_003), (32, 4_000_001)])
+def test_synthetic_stream_many_tiles_per_warp_bit_exact(b, M, p):
+    """Rows long enough that every warp of the quantize sweep owns several staged tiles: the refill of a stage, the
+    wrap of the stage index and the parity flip of its barrier all run, on non-zero Q_prev from iteration 2 on."""
+    iters = 6
+    w = workloads.c4(M=M, p=p, b=b, iters=iters)
+    ctx = laq.from_workload(w, trace_capacity=iters)
+    assert _tiles_per_warp(ctx) >= 3
+    mir = _mirror_for(w)
+    tr = ctx.step(iters, trace=True)
+    for j in range(iters):
+        _assert_trace_row(tr, j, mir.step())
+    assert tr["skip"][1:].sum() < M * (iters - 1)               # uploads after k = 1: Q_prev changes under the sweep
+    _assert_state_bit_exact(ctx.get_state(codes=True), mir.state(), p, b)
+    ctx.close()
+
+
+@pytest.mark.parametrize("b", [3, 8])
+def test_stored_gradients_many_tiles_per_warp_bit_exact(b):
+    """LAQ_FLAG_STORE_G: the same stream written to memory by step 1 and read back by the sweeps, which then stage
+    tiles of both Q_prev and g (long rows).  Same mirror, same bits."""
+    M, p, iters = 16, 2_000_003, 6
+    w = workloads.c4(M=M, p=p, b=b, iters=iters)
+    ctx = laq.from_workload(w, trace_capacity=iters, flags=laq.FLAG_STORE_G)
+    assert _tiles_per_warp(ctx) >= 3
+    mir = _mirror_for(w)
+    tr = ctx.step(iters, trace=True)
+    for j in range(iters):
+        _assert_trace_row(tr, j, mir.step())
+    gs = ctx.get_state(codes=True, g=True)
+    _assert_state_bit_exact(gs, mir.state(), p, b)
+    for m in (0, M - 1):
+        np.testing.assert_array_equal(gs["g"][m], oracle.synth_gradient(w.seed, m, M, p, iters, w.synth_sigma, w.synth_eta0))
+    ctx.close()
+
+
+@pytest.mark.parametrize("flags", [laq.FLAG_STORE_G, laq.FLAG_STORE_G | laq.FLAG_QUANT_OFF])
+@pytest.mark.parametrize("b,M,p", [(4, 5, 70001), (8, 3, 1_200_007), (1, 4, 4100)])
+def test_stored_gradients_equal_generated_gradients(b, M, p, flags):
+    iters = 10
+    w = workloads.c4(M=M, p=p, b=b, iters=iters)
+    a = laq.from_workload(w, trace_capacity=iters, flags=flags)
+    ref = laq.from_workload(w, trace_capacity=iters, flags=flags & ~laq.FLAG_STORE_G)
+    mir = _mirror_for(w, flags=flags & ~laq.FLAG_STORE_G)
+    ta, tb = a.step(iters, trace=True), ref.step(iters, trace=True)
+    for j in range(iters):
+        _assert_trace_row(ta, j, mir.step())
+    for key in ta:
+        if key in ("n_dq", "n_eps", "rhs"):           # the two sweeps sum in different orders
+            np.testing.assert_allclose(ta[key], tb[key], rtol=NORM_RTOL)
+        else:
+            np.testing.assert_array_equal(ta[key], tb[key])
+    sa, sb = a.get_state(codes=True), ref.get_state(codes=True)
+    for key in ("theta", "agg", "qprev", "clock", "counters", "codes"):
+        np.testing.assert_array_equal(sa[key], sb[key])
+    a.close()
+    ref.close()
+
+
+def test_external_gradients_long_rows_take_the_staged_path():
+    """Caller-supplied gradients with rows of more than 2^20 coordinates: the quantize sweep stages Q_prev and g."""
+    M, p, b, iters = 6, 2_400_011, 4, 5
+    rng = np.random.default_rng(5)
+    c = rng.standard_normal((M, p)).astype(np.float32)
+    Lm = rng.uniform(0.05, 2.0, M).astype(np.float32)
+    ctx = laq.Laq(model=laq.MODEL_EXTERNAL, M=M, p=p, alpha=0.05, b=b, D=4, xi=np.full(4, 0.2), tbar=6, trace_capacity=1)
+    mir = oracle.OracleLaq(32, oracle.MODEL_GIVEN, M, p, alpha=0.05, b=b, D=4, xi=np.full(4, 0.2), tbar=6)
+    theta = np.zeros(p, np.float32)
+    for k in range(iters):
+        g = Lm[:, None] * (theta[None, :] - c)
+        ctx.set_gradients(g)
+        tr = ctx.step(1, trace=True)
+        _assert_trace_row(tr, 0, mir.step_given(g))
+        gs = ctx.get_state(codes=True)
+        _assert_state_bit_exact(gs, mir.state(), p, b)
+        theta = gs["theta"]
+    ctx.close()
+
+
 def test_synthetic_full_size_sampled_workers():
-    """The benchmark's launch configuration (M = 64, p = 25.6 M, b = 8): worker messages of the first
-    iteration against the mirror for sampled workers, the aggregate invariant, and the clock rules."""
+    """The benchmark's launch configuration (M = 64, p = 25.6 M, b = 8): worker messages of the first four
+    iterations against the mirror for sampled workers (from the second iteration on against each worker's own
+    non-zero Q_prev, read back before the step), the aggregate invariant, and the clock rules."""
     M, p, b = 64, 25_600_000, 8
     w = workloads.c4(M=M, p=p, b=b)
     ctx = laq.from_workload(w, trace_capacity=4)
+    assert _tiles_per_warp(ctx) >= 3
     tr = ctx.step(1, trace=True)
     assert not tr["skip"].any() and tr["uploads"][0] == M          # every worker uploads at k = 1
+    sampled = (0, 17, 63)
     zero = np.zeros(p, np.float32)
-    for m in (0, 17, 63):
+    for m in sampled:
         g = oracle.synth_gradient(w.seed, m, M, p, 1, w.synth_sigma, w.synth_eta0)
         r = oracle.quantize(g, zero, b, np.float32)
         got = ctx.get_worker(m)
@@ -248,6 +338,7 @@ def test_synthetic_full_size_sampled_workers():
         assert tr["n_dq"][0, m] == pytest.approx(r["n_dq"], rel=NORM_RTOL)
         assert tr["n_eps"][0, m] == pytest.approx(r["n_eps"], rel=NORM_RTOL)
         del g, r, got
+    del zero
     # grad^1 = sum_m Q_m in ascending worker order (fp32 adds), theta^2 = -alpha grad^1 (theta^1 = 0)
     acc = np.zeros(p, np.float32)
     for m in range(M):
@@ -258,19 +349,126 @@ def test_synthetic_full_size_sampled_workers():
     np.testing.assert_array_equal(s["theta"], -u)
     assert tr["dtheta2"][0] == pytest.approx(np.sum(u.astype(np.float64) ** 2), rel=NORM_RTOL)
     assert s["bits"] == M * (32 + b * p)
-    # three more iterations: skips appear, clocks count them, the aggregate still equals the sum of copies
-    tr = ctx.step(3, trace=True)
-    assert tr["skip"].sum() > 0
-    s = ctx.get_state(big=False)
+    del acc, u
+    # three more iterations, one at a time: the sampled workers' messages against the mirror's quantizer on the
+    # worker's own stored copy; skips appear, clocks count them
     consecutive = np.zeros(M, int)
-    for j in range(3):
-        consecutive = np.where(tr["skip"][j] == 1, consecutive + 1, 0)
+    skipped = 0
+    for k in (2, 3, 4):
+        before = {m: ctx.get_worker(m, codes=False)["qprev"] for m in sampled}
+        tr = ctx.step(1, trace=True)
+        for m in sampled:
+            g = oracle.synth_gradient(w.seed, m, M, p, k, w.synth_sigma, w.synth_eta0)
+            r = oracle.quantize(g, before[m], b, np.float32)
+            got = ctx.get_worker(m)
+            assert got["R"] == r["R"] == tr["R"][0, m]
+            np.testing.assert_array_equal(got["codes"], oracle.pack_codes(r["q"], b))
+            assert tr["n_dq"][0, m] == pytest.approx(r["n_dq"], rel=NORM_RTOL)
+            assert tr["n_eps"][0, m] == pytest.approx(r["n_eps"], rel=NORM_RTOL)
+            # a skipping worker keeps its copy, an uploading one moves to Q_new
+            np.testing.assert_array_equal(got["qprev"], before[m] if tr["skip"][0, m] else r["qnew"])
+            del g, r, got
+        consecutive = np.where(tr["skip"][0] == 1, consecutive + 1, 0)
+        skipped += int(tr["skip"].sum())
+    assert skipped > 0
+    s = ctx.get_state(big=False)
     np.testing.assert_array_equal(s["clock"], consecutive)
     acc64 = np.zeros(p)
     for m in range(M):
         acc64 += ctx.get_worker(m, codes=False)["qprev"]
     assert np.max(np.abs(s["agg"] - acc64)) <= 1e-5 * np.max(np.abs(acc64))
     ctx.close()
+
+
+# ------------------------------------------------------------------------------------------------
+# the quotient shortcut of the quantize sweeps, aimed at its acceptance margin
+# ------------------------------------------------------------------------------------------------
+def _margin_gradients(b, R, rng, p_min=24_001):
+    """One worker's gradient (Q_prev = 0, so d = g) whose coordinates put the cheap candidate quotient
+    u' = fma(d, RN(1/s), RN(R RN(1/s))) within a few units in the last place of f +- (1/2 - 2^(b-21)) for every
+    integer f in [0, 2^b - 1]: the values around which the sweep decides between the candidate and the exact
+    division.  Coordinate 0 carries |d| = R."""
+    f32 = np.float32
+    R = f32(R)
+    levels = f32(2 ** b - 1)
+    s = f32(f32(2.0) * (f32(1.0) / levels)) * R          # (2 tau) R, each operation rounded to fp32
+    y = f32(1.0) / s
+    c = R * y
+    safe = 0.5 - 2.0 ** (b - 21)
+    targets = []
+    for f in range(2 ** b):
+        for sign in (-1.0, 1.0):
+            targets.append(f + sign * safe)
+    targets = np.array(targets)
+    targets = targets[(targets > -0.4) & (targets < 2 ** b - 0.6)]
+    d0 = ((targets - np.float64(c)) / np.float64(y)).astype(f32)      # d with fma(d, y, c) ~ target
+    cols = [d0]
+    up, down = d0.copy(), d0.copy()
+    for _ in range(24):                                               # neighbours of d0, one ulp at a time
+        up = np.nextafter(up, f32(np.inf))
+        down = np.nextafter(down, f32(-np.inf))
+        cols += [up.copy(), down.copy()]
+    d = np.concatenate(cols)
+    d = d[np.abs(d) < R]
+    pad = rng.uniform(-1.0, 1.0, max(0, p_min - d.size - 1)).astype(f32) * R * f32(0.999)
+    return np.concatenate([np.array([R], f32), d, pad]).astype(f32)
+
+
+@pytest.mark.parametrize("b", [1, 2, 3, 4, 8])
+def test_quotient_shortcut_at_its_margin_bit_exact(b):
+    rng = np.random.default_rng(900 + b)
+    levels = 2 ** b - 1
+    radii = [1.0, 0.1, 3.7e-3, 41.5, 2.0 ** -60 * levels * 0.5001, 2.0 ** 60 * levels * 0.4999, 7.3e11, 2.9e-13]
+    rows = [_margin_gradients(b, R, rng) for R in radii]
+    p = max(r.size for r in rows)
+    g = np.zeros((len(rows), p), np.float32)
+    for m, r in enumerate(rows):
+        g[m, :r.size] = r
+    M = len(rows)
+    kw = dict(alpha=0.01, b=b, D=2, xi=[0.0, 0.0], tbar=5)
+    ctx = laq.Laq(model=laq.MODEL_EXTERNAL, M=M, p=p, trace_capacity=1, **kw)
+    mir = oracle.OracleLaq(32, oracle.MODEL_GIVEN, M, p, **kw)
+    # iteration 1: Q_prev = 0, d = g exactly; iteration 2: the same construction on top of the new Q_prev
+    for k in range(2):
+        gk = g if k == 0 else (ctx.get_state()["qprev"] + g).astype(np.float32)
+        ctx.set_gradients(gk)
+        tr = ctx.step(1, trace=True)
+        _assert_trace_row(tr, 0, mir.step_given(gk))
+        _assert_state_bit_exact(ctx.get_state(codes=True), mir.state(), p, b)
+    # the construction did reach both sides of the margin: some coordinates of the unit-radius row have an exact
+    # t whose distance to the nearest half-integer boundary is below the margin, some above
+    t = (g[0].astype(np.float64) + 1.0) / (2.0 / levels)
+    dist = np.abs(t - np.round(t))                     # distance of u to the nearest integer, ~ |w|
+    near = np.abs(dist - (0.5 - 2.0 ** (b - 21))) < 2.0 ** (b - 20)
+    assert near.sum() >= 2 ** b and (dist[near] > 0.5 - 2.0 ** (b - 21)).any() and (dist[near] < 0.5 - 2.0 ** (b - 21)).any()
+    ctx.close()
+
+
+@pytest.mark.parametrize("p", [101, 3001])            # the single-block kernel and the three sweeps
+def test_radius_whose_grid_step_underflows(p):
+    """R > 0 so small that s = 2 tau R is subnormal or zero in fp32: codes stay inside [0, 2^b - 1] (clamped),
+    s = 0 gives code 0, and nothing turns into NaN.  Bit-exact against the mirror."""
+    M = 4
+    rng = np.random.default_rng(12)
+    tiny = np.float32(2.0 ** -149)
+    g = np.zeros((M, p), np.float32)
+    g[0] = rng.integers(-1, 2, p).astype(np.float32) * tiny                  # R = 2^-149: s rounds to 0
+    g[1] = rng.integers(-300, 301, p).astype(np.float32) * tiny              # subnormal s with a few bits
+    g[2] = rng.integers(-5, 6, p).astype(np.float32) * np.float32(2.0 ** -140)
+    g[3] = rng.standard_normal(p).astype(np.float32) * np.float32(1e-30)     # small but normal
+    g[0, 0], g[1, 0] = tiny, np.float32(300) * tiny
+    for b in (4, 8):
+        kw = dict(alpha=0.5, b=b, D=2, xi=[0.1, 0.1], tbar=5)
+        ctx = laq.Laq(model=laq.MODEL_EXTERNAL, M=M, p=p, trace_capacity=1, **kw)
+        mir = oracle.OracleLaq(32, oracle.MODEL_GIVEN, M, p, **kw)
+        for k in range(3):
+            gk = (g * np.float32(1 + k)).astype(np.float32)
+            ctx.set_gradients(gk)
+            tr = ctx.step(1, trace=True)
+            assert np.isfinite(tr["n_dq"]).all() and np.isfinite(tr["n_eps"]).all() and np.isfinite(tr["rhs"]).all()
+            _assert_trace_row(tr, 0, mir.step_given(gk))
+            _assert_state_bit_exact(ctx.get_state(codes=True), mir.state(), p, b)
+        ctx.close()
 
 
 # ------------------------------------------------------------------------------------------------

@@ -174,3 +174,36 @@ def test_bf16_rounding_matches_torch():
     ours = np.array([oracle.round_bf16(v) for v in x], dtype=np.float32)
     ref = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()
     np.testing.assert_array_equal(ours, ref)
+
+
+def test_grid_step_that_underflows_fp32():
+    """Eq. (5) is 0/0 or x/0 when 2 tau R is zero: R = 0, or (fp32 mirror) R so small that the product underflows.
+    The code is then 0 and Eq. (6) is applied as printed; with a subnormal step the codes stay in [0, 2^b - 1].
+    Whatever the worker sends, the server's recovery from (R, codes) reproduces the worker's Q_new bit for bit."""
+    tiny = np.float32(2.0 ** -149)
+    b = 4
+    qp = np.zeros(5, np.float32)
+    g = np.array([1, -1, 0, 1, -1], np.float32) * tiny
+    r = oracle.quantize(g, qp, b, np.float32)
+    assert r["R"] == tiny and np.float32(2.0) * (np.float32(1.0) / np.float32(15)) * tiny == 0.0   # the step is zero
+    assert r["q"].tolist() == [0] * 5
+    np.testing.assert_array_equal(r["dq"], np.full(5, -tiny))           # Eq. (6) with q = 0: -R
+    np.testing.assert_array_equal(r["eps"], g - r["qnew"])
+    assert np.max(np.abs(r["eps"])) <= 2 * tiny
+    qnew, dq = oracle.decode(r["R"], r["q"], qp, b, np.float32)
+    np.testing.assert_array_equal(qnew, r["qnew"])
+    # R = 0 exactly: nothing moves
+    z = oracle.quantize(qp, qp, b, np.float32)
+    assert z["R"] == 0 and not z["q"].any() and not z["dq"].any() and z["n_dq"] == 0 and z["n_eps"] == 0
+    # subnormal step with two or three significant bits: the quotient loses bits, codes are clamped into range
+    for b in (4, 8):
+        g = (np.arange(-300, 301, 7).astype(np.float32)) * tiny
+        g[0] = -np.float32(300) * tiny
+        r = oracle.quantize(g, np.zeros_like(g), b, np.float32)
+        assert r["q"].min() >= 0 and r["q"].max() <= 2 ** b - 1
+        assert np.isfinite(r["dq"]).all() and np.isfinite(r["n_dq"]) and np.isfinite(r["n_eps"])
+        qnew, _ = oracle.decode(r["R"], r["q"], np.zeros_like(g), b, np.float32)
+        np.testing.assert_array_equal(qnew, r["qnew"])
+    # the same tiny innovation in fp64 has a normal step: ordinary codes, the error bound of Sec. 2.1 holds
+    r64 = oracle.quantize(g.astype(np.float64), np.zeros(g.size), 4, np.float64)
+    assert np.max(np.abs(r64["eps"])) <= r64["R"] / 15 * (1 + 1e-12)

@@ -5,13 +5,15 @@ from a loop where allocation calls are forbidden because they stall the device. 
 one quantizer call whose scratch is a fixed array baked into the library instead of caller- or
 library-allocated memory.  This test calls it through the C ABI twice in a row (the scratch is shared and
 keeps the previous call's contents, so the second call checks that stale values are cleared) and compares
-codes, radius and norms with what the regular entry point (laq_step on a one-worker context) produces.
+codes, radius and norms with what the regular entry point (laq_step on a one-worker context) produces, and with
+the CPU oracle's quantizer (the fp32 mirror) directly.
 """
 import ctypes as C
 
 import numpy as np
 import pytest
 
+import oracle
 from paper_1909_07588_b200 import laq
 
 pytestmark = pytest.mark.gpu
@@ -34,7 +36,8 @@ def _regular_entry_point(g, qprev, b):
 def test_static_scratch_quantizer_matches_regular_entry_point_twice_in_a_row():
     import torch
     rng = np.random.default_rng(42)
-    cases = [(70001, 8, 1.0), (5003, 4, 1e-3), (600_000, 2, 30.0)]      # ragged sizes, different b and scales
+    # ragged sizes, every supported b, different scales
+    cases = [(70001, 8, 1.0), (5003, 4, 1e-3), (600_000, 2, 30.0), (33_333, 1, 0.5), (12_345, 16, 7.0)]
     # everything the calls touch is allocated up front; the calls themselves allocate nothing
     bufs = []
     for p, b, scale in cases:
@@ -48,6 +51,12 @@ def test_static_scratch_quantizer_matches_regular_entry_point_twice_in_a_row():
     # Objects of earlier tests that the collector has not yet freed would make the counters move during the
     # calls, so collect first.  Two checks: torch's allocator served no request, and the driver handed out no
     # device memory (which would also catch an allocation made inside the library).
+    # The very first call on a device looks up the scratch's address and loads the module, which the header tells
+    # callers to do at start-up: make that call here, on a tiny buffer, before the counters are sampled, so that the
+    # check holds whether or not earlier tests have used the library in this process.
+    warm = bufs[1]
+    laq.quantize_worker_static(warm["dg"][:16], warm["dq"][:16], 4, warm["codes"], warm["R"], warm["norms"])
+    torch.cuda.synchronize()
     import gc
     gc.collect()
     torch.cuda.synchronize()
@@ -65,6 +74,10 @@ def test_static_scratch_quantizer_matches_regular_entry_point_twice_in_a_row():
         n = c["norms"].cpu().numpy()
         assert n[0] == pytest.approx(ndq_ref, rel=NORM_RTOL)
         assert n[1] == pytest.approx(neps_ref, rel=NORM_RTOL)
+        r = oracle.quantize(c["g"], c["q"], c["b"], np.float32)        # Sec. 2.1, Eq. (5)-(6) on the CPU
+        np.testing.assert_array_equal(c["codes"].cpu().numpy().view(np.uint32), oracle.pack_codes(r["q"], c["b"]))
+        assert c["R"].item() == r["R"]
+        assert n[0] == pytest.approx(r["n_dq"], rel=NORM_RTOL) and n[1] == pytest.approx(r["n_eps"], rel=NORM_RTOL)
 
 
 def test_static_scratch_quantizer_rejects_oversized_and_bad_arguments():
