@@ -17,7 +17,10 @@ pytestmark = pytest.mark.gpu
 
 NORM_RTOL = 1e-5
 TRAJ_RTOL = 1e-4
-GRAD_RTOL = 2e-5     # fp32 gradient kernels against the fp64 model gradient at the same theta
+GRAD_RTOL = 2e-5     # fp32 gradient kernels against the fp64 model gradient at the same theta (2-norm, per worker)
+GRAD_CTOL = 2e-6     # the same coordinate by coordinate, relative to the worker's largest coordinate (observed
+                     # <= 1.2e-6 on the linear models; the network, whose dH is rounded to bf16, gets 2e-4)
+SKIP_TIE_RTOL = 1e-3 # a skip decision may differ from the fp64 oracle's only this close to equality in (7a)
 
 
 def _mirror_for(w, precision=32, **over):
@@ -242,14 +245,16 @@ def test_synthetic_stream_many_tiles_per_warp_bit_exact(b, M, p):
     """Rows long enough that every warp of the quantize sweep owns several staged tiles: the refill of a stage, the
     wrap of the stage index and the parity flip of its barrier all run, on non-zero Q_prev from iteration 2 on."""
     iters = 6
-    w = workloads.c4(M=M, p=p, b=b, iters=iters)
+    w = workloads.c4(M=M, p=p, b=b, iters=iters, eta0=0.4)     # a strong drift: uploads go on after k = 1
     ctx = laq.from_workload(w, trace_capacity=iters)
     assert _tiles_per_warp(ctx) >= 3
     mir = _mirror_for(w)
     tr = ctx.step(iters, trace=True)
     for j in range(iters):
         _assert_trace_row(tr, j, mir.step())
-    assert tr["skip"][1:].sum() < M * (iters - 1)               # uploads after k = 1: Q_prev changes under the sweep
+    assert tr["uploads"][0] == M                                # Q_prev is non-zero from the second iteration on
+    if b == 8:
+        assert tr["skip"][1:].sum() < M * (iters - 1)           # and keeps changing under the sweep
     _assert_state_bit_exact(ctx.get_state(codes=True), mir.state(), p, b)
     ctx.close()
 
@@ -258,7 +263,7 @@ def test_synthetic_stream_many_tiles_per_warp_bit_exact(b, M, p):
 def test_stored_gradients_many_tiles_per_warp_bit_exact(b):
     """LAQ_FLAG_STORE_G: the same stream written to memory by step 1 and read back by the sweeps, which then stage
     tiles of both Q_prev and g (long rows).  Same mirror, same bits."""
-    M, p, iters = 16, 2_000_003, 6
+    M, p, iters = 64, 2_000_003, 6
     w = workloads.c4(M=M, p=p, b=b, iters=iters)
     ctx = laq.from_workload(w, trace_capacity=iters, flags=laq.FLAG_STORE_G)
     assert _tiles_per_warp(ctx) >= 3
@@ -496,23 +501,43 @@ def _oracle_gradients(w, theta, batch=0, k=1):
     return np.array(out)
 
 
-def _run_model_parity(w, iters, batch=0):
-    """Three comparisons per iteration of a model workload:
-      (1) step 1 on identical input: the library's gradients at its own theta^k against the fp64 model gradient;
+def _worker_ties(g64_m, qprev_m, b):
+    """The fp64 oracle's own view of one worker's rounding decisions: R, the grid step s, and per coordinate
+    t = (d + R)/s + 1/2 of Eq. (5), whose floor is the code."""
+    d = g64_m - qprev_m
+    R = np.max(np.abs(d))
+    s = 2.0 * R / (2 ** b - 1)
+    t = (d + R) / s + 0.5 if s > 0 else np.full(d.shape, 0.5)
+    return R, s, t
+
+
+def _run_model_parity(w, iters, batch=0, grad_ctol=GRAD_CTOL, skip_tie_rtol=SKIP_TIE_RTOL):
+    """Per iteration of a model workload (gradients from the library's own kernels):
+      (1) step 1 on identical input: the library's gradients at its own theta^k against the fp64 model gradient,
+          in the 2-norm (GRAD_RTOL) and coordinate by coordinate (grad_ctol x the largest coordinate);
       (2) steps 2-5 on identical input: the fp32 mirror fed with the library's gradients, bit-exact;
-      (3) the whole iteration against the fp64 oracle, restarted every iteration from the library's state: skip
-          masks equal, codes equal except at near-ties (where |code difference| = 1 and both are nearest points up
-          to rounding), theta and loss within TRAJ_RTOL.
-    Besides, a free-running fp64 oracle follows the same problem from the start; the first iteration at which its
-    skip mask differs or theta leaves the TRAJ_RTOL band is reported and returned (None if never): a single
-    near-tie code flip moves one coordinate of theta by alpha 2 tau R, which both trajectories then absorb."""
+      (3) the whole iteration against the fp64 oracle restarted from the library's state.  A code may differ from
+          the oracle's only at a near-tie of the oracle's own Eq. (5): the library's code c must satisfy
+          |c - (t - 1/2)| <= 1/2 + tie, with tie = 4 grad_ctol ||g_m||_inf / s + 2^(b-21) what the gradient
+          tolerance (through d, R and s) and fp32 rounding can move t by.  Every differing code is classified; one
+          that is not a near-tie fails the test.  theta must equal the oracle's up to the classified code steps
+          (alpha s per differing code) within 1e-5, the loss within 1e-5; a skip decision may differ only where the
+          oracle's ||dQ||^2 is within SKIP_TIE_RTOL of its right-hand side.
+      (4) a free-running fp64 oracle from the same start: theta and loss must stay within TRAJ_RTOL for as long as
+          its skip masks equal the library's and none of its codes has differed yet (asserted); the first iteration
+          at which a skip bit differs, a code differs, or the band is left is recorded.
+    Returns the record."""
     ctx = laq.from_workload(w, trace_capacity=1, batch=batch)
     free64 = _mirror_for(w, 64, batch=batch)
     # step64 is stepped once per iteration, so its k (which the window start depends on) stays the library's
     step64 = _mirror_for(w, 64, batch=batch)
     mir = oracle.OracleLaq(32, oracle.MODEL_GIVEN, w.M, w.p, alpha=w.alpha, b=w.b, D=w.D, xi=w.xi, tbar=w.tbar,
                            theta0=w.theta0)
-    first_diff, code_flips, skip_flips, n_resolved = None, 0, 0, 0
+    if w.model == workloads.MODEL_MLP2 and grad_ctol == GRAD_CTOL:
+        grad_ctol = 2e-4                      # its 2-norm tolerance (observed coordinate errors <= 7e-5)
+    rec = dict(name=w.name, iters=iters, first_skip_diff=None, first_code_diff=None, first_band_exit=None,
+               near_tie_flips=0, codes_compared=0, skip_ties=0, max_coord_err=0.0, ctol_needed=0.0, skip_tie_needed=0.0)
+    levels = 2 ** w.b - 1
     prev = ctx.get_state()
     for k in range(iters):
         tr = ctx.step(1, trace=True)
@@ -524,6 +549,9 @@ def _run_model_parity(w, iters, batch=0):
         grad_rtol = 2e-4 if w.model == workloads.MODEL_MLP2 else GRAD_RTOL
         for m in range(w.M):
             assert np.linalg.norm(gs["g"][m] - g_ref[m]) <= grad_rtol * np.linalg.norm(g_ref[m]), (k, m)
+            cerr = np.max(np.abs(gs["g"][m] - g_ref[m])) / np.max(np.abs(g_ref[m]))
+            rec["max_coord_err"] = max(rec["max_coord_err"], float(cerr))
+            assert cerr <= grad_ctol, (k, m, cerr)
         # (2)
         st32 = mir.step_given(gs["g"])
         _assert_trace_row(tr, 0, st32)
@@ -533,47 +561,88 @@ def _run_model_parity(w, iters, batch=0):
                          clock=prev["clock"], hist=prev["ring"])
         st64 = step64.step()
         s64 = step64.state()
-        # codes are comparable while the quantization step 2 tau R is far above the fp32 rounding noise of the
-        # gradients (late in a run the innovation shrinks to that noise and the codes encode it)
-        resolved = bool(np.all(tr["R"][0] >= 0.01 * np.abs(gs["g"]).max(axis=1)))
-        same_skip = np.array_equal(st64["skip"].astype(np.uint8), tr["skip"][0])
         assert tr["loss"][0] == pytest.approx(st64["loss"], rel=1e-5)
-        if resolved:
-            n_resolved += 1
-            codes_gpu = np.stack([oracle.unpack_codes(gs["codes"][m], w.p, w.b) for m in range(w.M)])
-            dc = codes_gpu - s64["codes"]
-            assert np.abs(dc).max() <= 1
-            flips = int(np.count_nonzero(dc))
-            code_flips += flips
-            skip_flips += 0 if same_skip else 1
-            if flips == 0:
+        codes_gpu = np.stack([oracle.unpack_codes(gs["codes"][m], w.p, w.b) for m in range(w.M)])
+        dc = codes_gpu - s64["codes"]
+        steps = np.zeros(w.M)
+        for m in range(w.M):
+            R, s, t = _worker_ties(s64["g"][m], prev["qprev"][m].astype(np.float64), w.b)
+            steps[m] = s
+            idx = np.nonzero(dc[m])[0]
+            if idx.size == 0:
+                continue
+            tie = 4.0 * grad_ctol * np.max(np.abs(s64["g"][m])) / s + 2.0 ** (w.b - 21)
+            off = np.abs(codes_gpu[m, idx] - (t[idx] - 0.5))
+            assert np.all(off <= 0.5 + tie), (k, m, idx[:5], off[:5], tie)      # every flip is a near-tie
+            # the gradient tolerance that would just explain the largest excess (for the report)
+            rec["ctol_needed"] = max(rec["ctol_needed"], float(np.max(off - 0.5 - 2.0 ** (w.b - 21)) * s
+                                                                / (4.0 * np.max(np.abs(s64["g"][m])))))
+        rec["near_tie_flips"] += int(np.count_nonzero(dc))
+        rec["codes_compared"] += dc.size
+        same_skip = np.array_equal(st64["skip"].astype(np.uint8), tr["skip"][0])
+        if not same_skip:
+            # (7a) evaluated by the oracle on the library's codes (all of them validated above): it must give
+            # the library's decision, or be itself within skip_tie_rtol of equality
+            for m in np.nonzero(st64["skip"].astype(np.uint8) != tr["skip"][0])[0]:
+                R, s, _ = _worker_ties(s64["g"][m], prev["qprev"][m].astype(np.float64), w.b)
+                d = s64["g"][m] - prev["qprev"][m]
+                dq = s * codes_gpu[m] - R
+                n_dq, n_eps = np.sum(dq * dq), np.sum((d - dq) ** 2)
+                rhs = st64["rhs"][m] + 3.0 * (n_eps - st64["n_eps"][m])
+                gap = abs(n_dq - rhs) / rhs
+                # the gradient tolerance moves every eps_i (at most s/2 in size) by up to grad_ctol ||g||_inf
+                tie = 4.0 * grad_ctol * np.max(np.abs(s64["g"][m])) / s
+                if (n_dq <= rhs) != bool(tr["skip"][0][m]):
+                    rec["skip_tie_needed"] = max(rec["skip_tie_needed"], float(gap - 2.0 * tie))
+                    assert gap <= skip_tie_rtol + 2.0 * tie, (k, m, gap, tie)
+                rec["skip_ties"] += 1
+        else:
+            up = np.nonzero(tr["skip"][0] == 0)[0]
+            moved = -w.alpha * (steps[up, None] * dc[up]).sum(axis=0) if up.size else 0.0
+            assert np.linalg.norm(gs["theta"] - s64["theta"] - moved) <= 1e-5 * np.linalg.norm(s64["theta"]), k
+            if not dc.any():
                 np.testing.assert_allclose(tr["n_dq"][0], st64["n_dq"], rtol=0.01)
-                if same_skip:
-                    assert np.linalg.norm(gs["theta"] - s64["theta"]) <= 1e-5 * np.linalg.norm(s64["theta"])
-        # free-running fp64 trajectory
-        if first_diff is None:
-            f64 = free64.step()
-            th = free64.state(big=False)["theta"]
-            if (not np.array_equal(f64["skip"].astype(np.uint8), tr["skip"][0])
-                    or np.linalg.norm(gs["theta"] - th) > TRAJ_RTOL * np.linalg.norm(th)
-                    or abs(tr["loss"][0] - f64["loss"]) > TRAJ_RTOL * abs(f64["loss"])):
-                first_diff = k + 1
+        # (4)
+        f64 = free64.step()
+        if rec["first_skip_diff"] is None and not np.array_equal(f64["skip"].astype(np.uint8), tr["skip"][0]):
+            rec["first_skip_diff"] = k + 1
+        if rec["first_code_diff"] is None and rec["first_skip_diff"] is None:
+            fc = free64.state()["codes"]
+            if not np.array_equal(fc, codes_gpu):
+                rec["first_code_diff"] = k + 1
+        th = free64.state(big=False)["theta"]
+        in_band = (np.linalg.norm(gs["theta"] - th) <= TRAJ_RTOL * np.linalg.norm(th)
+                   and abs(tr["loss"][0] - f64["loss"]) <= TRAJ_RTOL * abs(f64["loss"]))
+        if rec["first_band_exit"] is None and not in_band:
+            rec["first_band_exit"] = k + 1
+        if rec["first_skip_diff"] is None and rec["first_code_diff"] is None:
+            assert in_band, "left the %g band at iteration %d with equal skip masks and codes" % (TRAJ_RTOL, k + 1)
         prev = gs
-    print("%s: %d iterations; free-running fp64 trajectory first left the %g band (or changed a skip bit) at "
-          "iteration %s; restarted comparison over %d resolved iterations: %d near-tie code flips of %d codes, "
-          "%d skip-mask differences"
-          % (w.name, iters, TRAJ_RTOL, first_diff, n_resolved, code_flips, n_resolved * w.M * w.p, skip_flips))
-    assert n_resolved >= min(iters, 10)
-    assert code_flips <= max(3, 1e-3 * n_resolved * w.M * w.p)
-    assert skip_flips <= max(1, n_resolved // 25)
+    firsts = [v for v in (rec["first_skip_diff"], rec["first_band_exit"]) if v is not None]
+    rec["first_disagreement"] = min(firsts) if firsts else None
+    print("%(name)s: %(iters)d iterations; against the free-running fp64 oracle: first skip-bit difference at "
+          "iteration %(first_skip_diff)s, first code difference at %(first_code_diff)s, left the band at "
+          "%(first_band_exit)s; restarted comparison: %(near_tie_flips)d near-tie code differences of "
+          "%(codes_compared)d codes (explained by a gradient tolerance of %(ctol_needed).3g), %(skip_ties)d skip "
+          "near-ties (largest gap %(skip_tie_needed).3g); largest coordinate error of a gradient %(max_coord_err).3g "
+          "of its largest coordinate" % rec)
     ctx.close()
-    return first_diff
+    return rec
 
 
+def _first(rec):
+    """Iteration of the first disagreement with the free-running fp64 oracle (skip bit or band), or a number past
+    the run if there was none."""
+    return rec["first_disagreement"] if rec["first_disagreement"] is not None else rec["iters"] + 1
+
+
+# Thresholds below: the first disagreement with the free-running fp64 oracle was observed at iteration 66 (C0),
+# 48 and 11 (minibatch logistic and softmax), 20 and 40 (reduced C2 and C1 shapes), 22 (C2 at full size), and not
+# within the iterations run at full size for C1 (12) and C3 (3); the asserted values leave a quarter of slack.
 def test_c0_logreg_full():
     w = workloads.c0()
-    first = _run_model_parity(w, w.iters)
-    assert first is None or first > 3
+    rec = _run_model_parity(w, w.iters)
+    assert _first(rec) > 50
 
 
 def test_minibatch_logreg_windows_wrap_and_ragged_tiles():
@@ -583,14 +652,14 @@ def test_minibatch_logreg_windows_wrap_and_ragged_tiles():
     w.b = 3
     wraps = sum(oracle.batch_offset(w.seed, m, k, 3001) + 500 > 3001 for m in range(w.M) for k in range(1, 61))
     assert wraps > 0
-    first = _run_model_parity(w, w.iters, batch=500)
-    assert first is None or first > 3
+    rec = _run_model_parity(w, w.iters, batch=500)
+    assert _first(rec) > 35
 
 
 def test_minibatch_softmax():
     w = workloads.c1(n_per=1203, iters=40)
-    first = _run_model_parity(w, w.iters, batch=500)
-    assert first is None or first > 3
+    rec = _run_model_parity(w, w.iters, batch=500)
+    assert _first(rec) > 8
 
 
 def test_minibatch_small_shards_use_every_sample():
@@ -610,30 +679,30 @@ def test_c2_shape_logreg54_reduced():
     # column can have an innovation of exactly 0, which sits midway between the two central grid points
     # (the grid has no zero level); fp32 and fp64 then legitimately pick different, equally near codes.
     w = workloads.c2(n_per=3001, iters=60, theta0_scale=0.01)
-    first = _run_model_parity(w, w.iters)
-    assert first is None or first > 3
+    rec = _run_model_parity(w, w.iters)
+    assert _first(rec) > 15
 
 
 def test_c1_shape_softmax_reduced():
     w = workloads.c1(n_per=333, iters=40)
-    first = _run_model_parity(w, w.iters)
-    assert first is None or first > 3
+    rec = _run_model_parity(w, w.iters)
+    assert _first(rec) > 30
 
 
 def test_c1_full_size_first_iterations():
     """The benchmark's own shape and launch configuration (10 x 6000 rows, 784 features, 10 classes)."""
-    w = workloads.c1(iters=3)
-    _run_model_parity(w, 3)
+    w = workloads.c1(iters=12)
+    assert _first(_run_model_parity(w, 12)) > 12
 
 
 def test_c2_full_size_first_iterations():
-    w = workloads.c2(iters=4, theta0_scale=0.01)
-    _run_model_parity(w, 4)
+    w = workloads.c2(iters=40, theta0_scale=0.01)
+    assert _first(_run_model_parity(w, 40)) > 16
 
 
 def test_c3_full_size_first_iterations():
-    w = workloads.c3(iters=2)
-    _run_model_parity(w, 2)
+    w = workloads.c3(iters=3)
+    assert _first(_run_model_parity(w, 3)) > 3
 
 
 def test_softmax_small_odd_shapes():
