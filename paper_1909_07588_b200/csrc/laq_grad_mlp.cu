@@ -337,22 +337,34 @@ __global__ void __launch_bounds__(kThreads) mlp_dw1_kernel(const Params P, const
   }
 }
 
+// Tile (or block) partials -> g for b1, W2, b2, and the worker's loss term.  Eight neighbouring lanes share an
+// output: lane l adds the partials l, l + 8, ... (all of its loads independent), the eight sums are then added in
+// lane order, so the result does not depend on timing and costs about one trip to the L2 instead of one per tile.
 __global__ void __launch_bounds__(256) mlp_finalize_kernel(const Params P, const MlpDev D, const double* theta_sq) {
   const int H = P.H, C = P.C, F = P.F, m = blockIdx.y;
   const int nsmall = H + C * H + C;
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  const int sub = threadIdx.x & 7;
+  const int i = blockIdx.x * 32 + (threadIdx.x >> 3);
   const double inv_N = 1.0 / (double)P.Ntot, share = (double)P.N[m] / (double)P.Ntot;
+  double s = 0.0;
   if (i < nsmall) {
-    double s = 0.0;
-    for (int b = 0; b < D.gb; ++b) s += (double)D.spart[((long long)m * D.gb + b) * nsmall + i];
+    const float* sp = D.spart + (long long)m * D.gb * nsmall + i;
+    for (int b = sub; b < D.gb; b += 8) s += (double)__ldg(sp + (long long)b * nsmall);
+  }
+  double tot = 0.0;
+#pragma unroll
+  for (int l = 0; l < 8; ++l) tot += __shfl_sync(0xffffffffu, s, (threadIdx.x & 24) + l);
+  if (i < nsmall && sub == 0) {
     const long long pi = (long long)H * F + i;   // b1, W2, b2 follow W1 in theta in the same order as the partials
     P.g[(long long)m * P.ps + pi] =
-        (float)(s * (inv_N * batch_scale(P, m)) + share * (double)P.lambda * (double)P.theta[pi]);
+        (float)(tot * (inv_N * batch_scale(P, m)) + share * (double)P.lambda * (double)P.theta[pi]);
   }
-  if (blockIdx.x == 0 && threadIdx.x == 0) {
+  if (blockIdx.x == 0 && threadIdx.x < 32) {
     double l = 0.0;
-    for (int b = 0; b < D.gb; ++b) l += D.lpart[(long long)m * D.gb + b];
-    P.loss_m[m] = l * (inv_N * batch_scale(P, m)) + share * 0.5 * (double)P.lambda * (*theta_sq);
+    for (int b = threadIdx.x; b < D.gb; b += 32) l += D.lpart[(long long)m * D.gb + b];
+    double lt = 0.0;
+    for (int k = 0; k < 32; ++k) lt += __shfl_sync(0xffffffffu, l, k);
+    if (threadIdx.x == 0) P.loss_m[m] = lt * (inv_N * batch_scale(P, m)) + share * 0.5 * (double)P.lambda * (*theta_sq);
   }
 }
 
@@ -412,83 +424,113 @@ __global__ void __launch_bounds__(umma::kThreads) umma_hidden_kernel(const __gri
 // bf16 dH~ (stored transposed: consecutive lanes = consecutive rows = consecutive addresses) and the tile's
 // contributions to the b1 / W2 / b2 gradients, without writing the hidden activations to memory.
 //   pass 1  h = relu(acc + b1); scores z += h W2^T chunk by chunk; softmax, loss, dZ (kept in registers)
-//   pass 2  the accumulator is read again from tensor memory: dh = (dZ W2) o [h > 0] -> bf16 -> dH~^T; the h chunk
-//           goes through shared memory so that a thread per column can sum over the tile's rows
-//               A[c][j] = sum_r dZ[r][c] h[r][j]         (the W2 gradient)
-//               S[c][j] = sum_r dZ[r][c] [h[r][j] > 0]   (then db1[j] = sum_c W2[c][j] S[c][j])
+//   pass 2  the accumulator is read again from tensor memory: dh = (dZ W2) o [h > 0] -> bf16 -> dH~^T; the h and dh
+//           chunks go through shared memory so that threads that own columns can sum over the tile's rows
+//               A[c][j] = sum_r dZ[r][c] h[r][j]   (the W2 gradient),      db1[j] = sum_r dh[r][j]
 //           in a fixed order (no atomics).
-// Eight epilogue warps: two sets of four, each set taking every other 32-column chunk in both passes.
-constexpr int kFusedStages = 2;   // two stages of ring per block, two blocks per SM
+// Sixteen epilogue warps: four sets of four.  A set's four warps cover the four lane quarters of tensor memory
+// (all 128 rows); the sets share the 16-column chunks of the accumulator round robin in both passes.
 #ifndef LAQ_DW1_STAGES
 #define LAQ_DW1_STAGES 4
 #endif
 constexpr int kDw1Stages = LAQ_DW1_STAGES;   // ring depth of the W1-gradient product (one block per SM)
 
-constexpr int kFusedEpiWarps = 8;                      // two sets of four epilogue warps
-constexpr int kFusedThreads = 64 + 32 * kFusedEpiWarps;
+// The fused kernel is persistent: one block per SM walks the 128-row tiles of all workers.  The loader warp and the
+// tensor-core warp run ahead of the epilogue warps through a ring of kFusedStages stages and TWO accumulators in
+// tensor memory (2 x 256 columns), so the 13 K blocks of the next tile are loaded and multiplied while the
+// epilogue warps work on the current one; the epilogue's scratch is its own shared memory, not the ring.
+constexpr int kFusedStages = 3;
+constexpr int kFusedSets = 4;
+constexpr int kFusedEpiWarps = 4 * kFusedSets;
+constexpr int kFusedEpiThreads = 32 * kFusedEpiWarps;
+constexpr int kFusedThreads = 64 + kFusedEpiThreads;
+constexpr uint32_t kFusedAccCols = 256;                // tensor-memory columns per accumulator
+constexpr int kFusedChunk = 16;                        // columns per chunk
+constexpr int kFusedPitch = kFusedChunk + 1;           // row pitch of a chunk plane in shared memory (floats)
+constexpr int kFusedPlane = 128 * kFusedPitch;         // one plane: 128 rows of a chunk
 
 __host__ __device__ inline size_t fused_extra_floats(int H) {
-  return (size_t)H * 12 + (size_t)((H + 3) & ~3) + 2 * 128 * 33 + 128 * 12 + 2 * (size_t)12 * H + 16;
+  return (size_t)H * 12 + (size_t)((H + 3) & ~3) + (size_t)kFusedSets * 2 * kFusedPlane + 128 * 12 + (size_t)12 * H +
+         (size_t)((H + 3) & ~3) + 16;
+}
+__host__ __device__ inline size_t fused_smem_bytes(int nt, int H) {
+  return kFusedStages * umma::stage_bytes(nt) + 1024 + fused_extra_floats(H) * 4;
 }
 
-// Both sets of epilogue warps own all 128 rows (thread = row) and share the 32-column chunks of the accumulator
-// between them: set 0 takes chunks 0, 2, 4, ..., set 1 chunks 1, 3, 5, ...  The scores are the sum of the two sets'
-// partial scores (set 0's first); every later step is per column, so the sets only meet at three block-wide points.
 struct FusedEpi {
   const Params& P;
   const MlpDev& D;
-  int nt, m, tile;          // worker and tile index within the worker
-  RowWindow win;            // rows of the worker that enter this iteration's gradient
-  static __device__ __forceinline__ void sync_all() { umma::named_sync<1, 32 * kFusedEpiWarps>(); }
+  int nt;
+  float* base;              // the epilogue's scratch (shared memory behind the stage ring)
+  static __device__ __forceinline__ void sync_all() { umma::named_sync<1, kFusedEpiThreads>(); }
   static __device__ __forceinline__ void sync_set(int set) {
-    if (set == 0) umma::named_sync<2, 128>(); else umma::named_sync<3, 128>();
+    switch (set) {
+      case 0: umma::named_sync<2, 128>(); break;
+      case 1: umma::named_sync<3, 128>(); break;
+      case 2: umma::named_sync<4, 128>(); break;
+      default: umma::named_sync<5, 128>(); break;
+    }
   }
-  __device__ __forceinline__ void run(uint32_t tmem_base, int q, int lane, int set) {
+  __device__ __forceinline__ float* w2t() const { return base; }                                   // [H][12]
+  __device__ __forceinline__ float* b1s() const { return base + (size_t)P.H * 12; }               // [H]
+  __device__ __forceinline__ float* chunks() const { return b1s() + ((P.H + 3) & ~3); }           // [sets][h, dh][128][17]
+
+  // once per block: W2 transposed (j-major, rows of 12) and b1 into shared memory
+  __device__ __forceinline__ void load_constants(int et) const {
+    const int H = P.H, C = P.C;
+    const float* __restrict__ b1 = P.theta + (long long)H * P.F;
+    const float* __restrict__ W2 = b1 + H;
+    float* w = w2t();
+    float* b = b1s();
+    for (int i = et; i < H * 12; i += kFusedEpiThreads) {
+      const int j = i / 12, c = i - 12 * j;
+      w[i] = (c < C) ? __ldg(W2 + (size_t)c * H + j) : 0.f;
+    }
+    for (int i = et; i < H; i += kFusedEpiThreads) b[i] = __ldg(b1 + i);
+  }
+
+  // One tile.  tmem_acc: the accumulator's first column; released(): called by every epilogue thread after its last
+  // read of tensor memory (the tensor-core warp may then overwrite the accumulator).
+  template <class Release>
+  __device__ __forceinline__ void run(uint32_t tmem_acc, int q, int lane, int set, int m, int tile, const RowWindow& win,
+                                      Release released) {
     const int H = P.H, C = P.C, F = P.F;
     const int tt = q * 32 + lane;            // 0..127: the tile row this thread owns
-    const int et = set * 128 + tt;           // 0..255 among the epilogue threads
-    float* base = reinterpret_cast<float*>(umma::ring_smem());   // the ring is free once the accumulator is complete
-    float* w2t = base;                       // [H][12]   W2 transposed (j-major), padded rows of 12
-    float* b1s = w2t + (size_t)H * 12;       // [H]
-    float* chunks = b1s + ((H + 3) & ~3);    // [2][128][33] one 32-column chunk of h per set
-    float* dzs = chunks + 2 * 128 * 33;      // [128][12]
+    const int et = set * 128 + tt;           // among the epilogue threads
+    const float* w2 = w2t();
+    const float* b1v = b1s();
+    float* ch = chunks();
+    float* dzs = ch + kFusedSets * 2 * kFusedPlane;   // [128][12]
     float* accA = dzs + 128 * 12;            // [12][H]
-    float* accS = accA + (size_t)12 * H;     // [12][H]
-    double* lossw = reinterpret_cast<double*>(accS + (size_t)12 * H);      // [4] (8-byte aligned: all sizes even)
-    float* chunk = chunks + set * 128 * 33;  // this set's chunk buffer
-    float* red = chunk;                      // [4][2 C][32] partial column sums, reuses the chunk buffer
-    float* zpart = chunks;                   // [2][128][12] partial scores of the two sets, before the chunks are used
-    const float* __restrict__ theta = P.theta;
-    const float* __restrict__ b1 = theta + (long long)H * F;
-    const float* __restrict__ W2 = b1 + H;
-    const float* __restrict__ b2 = W2 + (long long)C * H;
-    for (int i = et; i < H * 12; i += 256) {
-      const int j = i / 12, c = i - 12 * j;
-      w2t[i] = (c < C) ? __ldg(W2 + (size_t)c * H + j) : 0.f;
-    }
-    for (int i = et; i < H; i += 256) b1s[i] = __ldg(b1 + i);
+    float* accB = accA + (size_t)12 * H;     // [H]   column sums of dh: the b1 gradient
+    double* lossw = reinterpret_cast<double*>(accB + ((H + 3) & ~3));      // [4] (8-byte aligned: all sizes even)
+    float* chunk_h = ch + set * (2 * kFusedPlane);   // this set's h chunk, the dh chunk behind it
+    float* chunk_d = chunk_h + kFusedPlane;
+    float* red = chunk_h;                    // [16][11][16] partial column sums, reuses both chunk planes
+    float* zpart = ch;                       // [sets][128][12] partial scores of the sets, before the chunks are used
+    const float* __restrict__ b2 = P.theta + (long long)H * F + H + (long long)C * H;
     const long long n = P.N[m];
     const long long trow = (long long)tile * umma::kTileM + tt;   // row within the worker's shard
     const bool valid = trow < n && win.contains(trow);
     const int yv = valid ? __ldg(P.y[m] + trow) : -1;             // asked for now, used after the first pass
-    sync_all();
-    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+    const uint32_t taddr = tmem_acc + ((uint32_t)(q * 32) << 16);
+    constexpr int kStep = kFusedChunk * kFusedSets;
     // ---- pass 1: partial scores over this set's chunks, as packed pairs of classes z2[k] = (z[2k], z[2k+1])
     unsigned long long z2[6];
 #pragma unroll
     for (int c = 0; c < 6; ++c) z2[c] = 0ull;
-    for (int c0 = 32 * set; c0 < nt; c0 += 64) {
-      uint32_t v[32];
-      umma::tmem_load_32(taddr + (uint32_t)c0, v);
+    for (int c0 = kFusedChunk * set; c0 < nt; c0 += kStep) {
+      uint32_t v[kFusedChunk];
+      umma::tmem_load_16(taddr + (uint32_t)c0, v);
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
+      for (int i = 0; i < kFusedChunk; ++i) {
         const int j = c0 + i;
         if (j < H) {
-          const float h = fmaxf(__uint_as_float(v[i]) + b1s[j], 0.f);
+          const float h = fmaxf(__uint_as_float(v[i]) + b1v[j], 0.f);
           const unsigned long long hh = pack2(h, h);
-          const ulonglong2 wa = *reinterpret_cast<const ulonglong2*>(w2t + j * 12);
-          const ulonglong2 wb = *reinterpret_cast<const ulonglong2*>(w2t + j * 12 + 4);
-          const ulonglong2 wc = *reinterpret_cast<const ulonglong2*>(w2t + j * 12 + 8);
+          const ulonglong2 wa = *reinterpret_cast<const ulonglong2*>(w2 + j * 12);
+          const ulonglong2 wb = *reinterpret_cast<const ulonglong2*>(w2 + j * 12 + 4);
+          const ulonglong2 wc = *reinterpret_cast<const ulonglong2*>(w2 + j * 12 + 8);
           z2[0] = ffma2(hh, wa.x, z2[0]); z2[1] = ffma2(hh, wa.y, z2[1]);
           z2[2] = ffma2(hh, wb.x, z2[2]); z2[3] = ffma2(hh, wb.y, z2[3]);
           z2[4] = ffma2(hh, wc.x, z2[4]); z2[5] = ffma2(hh, wc.y, z2[5]);
@@ -504,10 +546,15 @@ struct FusedEpi {
     sync_all();
     float dz[12];
     double loss = 0.0;
-    {  // both sets do the softmax of the row (the same arithmetic), set 0 keeps the loss and publishes dZ
+    {  // every set does the softmax of the row (the same arithmetic), set 0 keeps the loss and publishes dZ
       float z[12];
 #pragma unroll
-      for (int c = 0; c < 12; ++c) z[c] = zpart[tt * 12 + c] + zpart[(128 + tt) * 12 + c];
+      for (int c = 0; c < 12; ++c) {
+        float zs = zpart[tt * 12 + c];
+#pragma unroll
+        for (int s2 = 1; s2 < kFusedSets; ++s2) zs += zpart[(s2 * 128 + tt) * 12 + c];   // the sets' partials in order
+        z[c] = zs;
+      }
       float zmax = -3.0e38f;
 #pragma unroll
       for (int c = 0; c < 12; ++c)
@@ -538,19 +585,26 @@ struct FusedEpi {
     for (int c = 0; c < 6; ++c) dz2[c] = pack2(dz[2 * c], dz[2 * c + 1]);
     const long long col = D.rowoffT[m] + trow;
     const bool in_segment = col < D.rowoffT[m + 1];        // rows of the padded segment (zeros beyond the shard)
-    const int rq = tt >> 5, cl = tt & 31;                  // reduce phase: column cl, rows 32 rq .. 32 rq + 31
-    for (int c0 = 32 * set; c0 < nt; c0 += 64) {
-      uint32_t v[32];
-      umma::tmem_load_32(taddr + (uint32_t)c0, v);
+    // column phase: this thread sums the columns 2 cg, 2 cg + 1 of a chunk over the rows 32 q + rho + 2 k, k = 0..7;
+    // with rows rho in {0, 1, 16, 17} and a pitch of 17 floats the 32 lanes of a warp read 32 different banks
+    const int cg = lane & 7, rsub = lane >> 3, rho = (rsub & 1) + 16 * (rsub >> 1);
+    bool released_yet = false;
+    for (int c0 = kFusedChunk * set; c0 < nt; c0 += kStep) {
+      uint32_t v[kFusedChunk];
+      umma::tmem_load_16(taddr + (uint32_t)c0, v);
+      if (c0 + kStep >= nt) {                              // that was this thread's last read of the accumulator
+        released();
+        released_yet = true;
+      }
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
+      for (int i = 0; i < kFusedChunk; ++i) {
         const int j = c0 + i;
-        float h = 0.f;
+        float h = 0.f, dh = 0.f;
         if (j < H) {
-          h = fmaxf(__uint_as_float(v[i]) + b1s[j], 0.f);
-          const ulonglong2 wa = *reinterpret_cast<const ulonglong2*>(w2t + j * 12);
-          const ulonglong2 wb = *reinterpret_cast<const ulonglong2*>(w2t + j * 12 + 4);
-          const ulonglong2 wc = *reinterpret_cast<const ulonglong2*>(w2t + j * 12 + 8);
+          h = fmaxf(__uint_as_float(v[i]) + b1v[j], 0.f);
+          const ulonglong2 wa = *reinterpret_cast<const ulonglong2*>(w2 + j * 12);
+          const ulonglong2 wb = *reinterpret_cast<const ulonglong2*>(w2 + j * 12 + 4);
+          const ulonglong2 wc = *reinterpret_cast<const ulonglong2*>(w2 + j * 12 + 8);
           // even and odd classes in the two halves of a packed sum, added at the end
           unsigned long long d2 = ffma2(dz2[0], wa.x, 0ull);
           d2 = ffma2(dz2[1], wa.y, d2); d2 = ffma2(dz2[2], wb.x, d2); d2 = ffma2(dz2[3], wb.y, d2);
@@ -558,53 +612,63 @@ struct FusedEpi {
           float d_even, d_odd;
           unpack2(d2, d_even, d_odd);
           const float d = d_even + d_odd;
-          const float dh = h > 0.f ? d : 0.f;
+          dh = h > 0.f ? d : 0.f;
           if (in_segment) D.dHT[(long long)j * D.ldT + col] = __float2bfloat16_rn(dh);
         }
-        chunk[tt * 33 + i] = h;
+        chunk_h[tt * kFusedPitch + i] = h;
+        chunk_d[tt * kFusedPitch + i] = dh;
       }
       sync_set(set);
-      {  // column sums over this thread's 32 rows
-        unsigned long long a2[6], s2[6];    // packed pairs of classes
+      {
+        unsigned long long a2[2][5];        // [column][pair of classes]
+        float db[2] = {0.f, 0.f};
 #pragma unroll
-        for (int c = 0; c < 6; ++c) a2[c] = s2[c] = 0ull;
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+          for (int c = 0; c < 5; ++c) a2[i][c] = 0ull;
 #pragma unroll 4
-        for (int r = 32 * rq; r < 32 * rq + 32; ++r) {
-          const float h = chunk[r * 33 + cl];
-          const float pos = h > 0.f ? 1.f : 0.f;
-          const unsigned long long hh = pack2(h, h), pp = pack2(pos, pos);
+        for (int k = 0; k < 8; ++k) {
+          const int r = 32 * q + rho + 2 * k;
           const ulonglong2 da = *reinterpret_cast<const ulonglong2*>(dzs + r * 12);
-          const ulonglong2 db = *reinterpret_cast<const ulonglong2*>(dzs + r * 12 + 4);
-          const ulonglong2 dc = *reinterpret_cast<const ulonglong2*>(dzs + r * 12 + 8);
-          a2[0] = ffma2(da.x, hh, a2[0]); a2[1] = ffma2(da.y, hh, a2[1]); a2[2] = ffma2(db.x, hh, a2[2]);
-          a2[3] = ffma2(db.y, hh, a2[3]); a2[4] = ffma2(dc.x, hh, a2[4]); a2[5] = ffma2(dc.y, hh, a2[5]);
-          s2[0] = ffma2(da.x, pp, s2[0]); s2[1] = ffma2(da.y, pp, s2[1]); s2[2] = ffma2(db.x, pp, s2[2]);
-          s2[3] = ffma2(db.y, pp, s2[3]); s2[4] = ffma2(dc.x, pp, s2[4]); s2[5] = ffma2(dc.y, pp, s2[5]);
-        }
-        float a[12], sgn[12];
+          const ulonglong2 dbq = *reinterpret_cast<const ulonglong2*>(dzs + r * 12 + 4);
+          const unsigned long long dc = *reinterpret_cast<const unsigned long long*>(dzs + r * 12 + 8);
 #pragma unroll
-        for (int c = 0; c < 6; ++c) {
-          unpack2(a2[c], a[2 * c], a[2 * c + 1]);
-          unpack2(s2[c], sgn[2 * c], sgn[2 * c + 1]);
+          for (int i = 0; i < 2; ++i) {
+            const float h = chunk_h[r * kFusedPitch + 2 * cg + i];
+            db[i] += chunk_d[r * kFusedPitch + 2 * cg + i];
+            const unsigned long long hh = pack2(h, h);
+            a2[i][0] = ffma2(da.x, hh, a2[i][0]); a2[i][1] = ffma2(da.y, hh, a2[i][1]);
+            a2[i][2] = ffma2(dbq.x, hh, a2[i][2]); a2[i][3] = ffma2(dbq.y, hh, a2[i][3]);
+            a2[i][4] = ffma2(dc, hh, a2[i][4]);
+          }
         }
-        sync_set(set);              // the set has read the chunk: reuse it for the partial sums
+        sync_set(set);              // the set has read the chunks: reuse them for the partial sums
+        float* rp = red + ((q * 4 + rsub) * 11) * kFusedChunk + 2 * cg;
 #pragma unroll
-        for (int c = 0; c < 12; ++c) {
-          red[(rq * 24 + c) * 32 + cl] = a[c];
-          red[(rq * 24 + 12 + c) * 32 + cl] = sgn[c];
+        for (int i = 0; i < 2; ++i) {
+#pragma unroll
+          for (int c = 0; c < 5; ++c) {
+            float lo, hi;
+            unpack2(a2[i][c], lo, hi);
+            rp[(2 * c) * kFusedChunk + i] = lo;
+            rp[(2 * c + 1) * kFusedChunk + i] = hi;
+          }
+          rp[10 * kFusedChunk + i] = db[i];
         }
       }
       sync_set(set);
-      for (int i = tt; i < 24 * 32; i += 128) {   // fixed order over the four row quarters
-        const int k = i >> 5, cc = i & 31, j = c0 + cc;
+      for (int i = tt; i < 11 * kFusedChunk; i += 128) {   // fixed order over the sixteen row groups
+        const int k = i / kFusedChunk, cc = i % kFusedChunk, j = c0 + cc;
         if (j < H) {
-          const float sum4 = ((red[(0 * 24 + k) * 32 + cc] + red[(1 * 24 + k) * 32 + cc]) + red[(2 * 24 + k) * 32 + cc]) +
-                             red[(3 * 24 + k) * 32 + cc];
-          if (k < 12) accA[k * H + j] = sum4; else accS[(k - 12) * H + j] = sum4;
+          float sum = 0.f;
+#pragma unroll
+          for (int gq = 0; gq < 16; ++gq) sum += red[(gq * 11 + k) * kFusedChunk + cc];
+          if (k < 10) accA[k * H + j] = sum; else accB[j] = sum;
         }
       }
       sync_set(set);
     }
+    if (!released_yet) released();                         // a set without chunks never read the accumulator
     // ---- the tile's partials: [db1 (H) | dW2 (C H) | db2 (C)] and the loss
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, o);
@@ -612,10 +676,8 @@ struct FusedEpi {
     sync_all();
     const int gb = D.gb;
     float* sp = D.spart + ((long long)m * gb + tile) * (H + C * H + C);
-    for (int j = et; j < H; j += 256) {
-      float s = 0.f;
-      for (int c = 0; c < C; ++c) s = fmaf(w2t[j * 12 + c], accS[c * H + j], s);
-      sp[j] = s;
+    for (int j = et; j < H; j += kFusedEpiThreads) {
+      sp[j] = accB[j];
       for (int c = 0; c < C; ++c) sp[H + c * H + j] = accA[c * H + j];
     }
     if (set == 1 && tt < C) {
@@ -624,30 +686,175 @@ struct FusedEpi {
       sp[H + C * H + tt] = s;
     }
     if (et == 0) D.lpart[(long long)m * gb + tile] = ((lossw[0] + lossw[1]) + lossw[2]) + lossw[3];
+    sync_all();   // the scratch is free for the next tile
   }
 };
 
-// grid: (tiles per worker, M); tile t of worker m covers the worker's rows 128 t .. 128 t + 127
-__global__ void __launch_bounds__(kFusedThreads, 2) umma_hidden_fused_kernel(const __grid_constant__ CUtensorMap tmX,
+// the tile has rows of the shard that lie in the window (all rows without a minibatch)
+__device__ __forceinline__ bool fused_tile_has_rows(const Params& P, const RowWindow& win, int m, int tile) {
+  const long long t0 = (long long)tile * umma::kTileM, t1 = t0 + umma::kTileM;
+  return t0 < P.N[m] && ((t0 < win.start + win.len_a && t1 > win.start) || t0 < win.len_b);
+}
+
+// grid: one block per SM (at most); block b takes the tiles b, b + gridDim.x, ... of the list (worker m, tile t),
+// tile t of worker m covering the worker's rows 128 t .. 128 t + 127.
+__global__ void __launch_bounds__(kFusedThreads, 1) umma_hidden_fused_kernel(const __grid_constant__ CUtensorMap tmX,
                                                                            const __grid_constant__ CUtensorMap tmW,
                                                                            const Params P, const MlpDev D, int nt) {
-  const int m = blockIdx.y, tile = blockIdx.x;
-  const long long n = P.N[m];
-  const RowWindow win = row_window(P, m);
-  const long long t0 = (long long)tile * umma::kTileM, t1 = t0 + umma::kTileM;
-  // the tile has rows of the shard that lie in the window (all rows without a minibatch)
-  const bool has_rows = t0 < n && ((t0 < win.start + win.len_a && t1 > win.start) || t0 < win.len_b);
-  umma::TileCoord tc{(int)(D.rowoff[m] + t0), 0, 0, has_rows ? (P.F + umma::kBlockK - 1) / umma::kBlockK : 0};
-  if (!has_rows) {   // nothing to add from this tile: its slot holds zeros (dH~ of its rows is not written, and
-                     // the dW1 product does not read it)
-    const int nsmall = P.H + P.C * P.H + P.C;
-    float* sp = D.spart + ((long long)m * D.gb + tile) * nsmall;
-    for (int i = threadIdx.x; i < nsmall; i += blockDim.x) sp[i] = 0.f;
-    if (threadIdx.x == 0) D.lpart[(long long)m * D.gb + tile] = 0.0;
-    return;
+  extern __shared__ unsigned char umma_smem_raw[];
+  __shared__ uint64_t bars[2 * kFusedStages + 5];
+  __shared__ uint32_t tmem_base_sh;
+  __shared__ int abort_sh;      // set by the first thread whose wait runs out: everybody stops waiting
+  __shared__ int never_sh;      // stays 0: for the last waits of a block, which must not be cut short
+  __shared__ int epi_ok[kFusedEpiWarps];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t smem0 = (umma::smem_u32(umma_smem_raw) + 1023u) & ~1023u;   // stages are 1024-byte aligned
+  const uint32_t a_bytes = umma::kTileM * umma::kBlockK * 2, st_bytes = (uint32_t)umma::stage_bytes(nt);
+  const uint32_t full0 = umma::smem_u32(&bars[0]), empty0 = umma::smem_u32(&bars[kFusedStages]);
+  const uint32_t accf0 = umma::smem_u32(&bars[2 * kFusedStages]), acce0 = accf0 + 16, drain = accf0 + 32;
+  float* scratch = reinterpret_cast<float*>(umma_smem_raw + (smem0 - umma::smem_u32(umma_smem_raw)) +
+                                            (size_t)kFusedStages * st_bytes);
+  uint32_t* err_flag = &P.sc->err;
+  volatile int* abort_flag = &abort_sh;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kFusedStages; ++s) {
+      umma::mbar_init(full0 + 8 * s, 1);
+      umma::mbar_init(empty0 + 8 * s, 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      umma::mbar_init(accf0 + 8 * a, 1);
+      umma::mbar_init(acce0 + 8 * a, kFusedEpiThreads);   // every epilogue thread arrives once per tile
+    }
+    umma::mbar_init(drain, 1);
+    abort_sh = 0;
+    never_sh = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  FusedEpi epi{P, D, nt, m, tile, win};
-  umma::gemm_tn_tile<kFusedStages, kFusedEpiWarps>(&tmX, &tmW, nt, tc, &P.sc->err, epi);
+  if (warp == 1) {  // all of the SM's tensor memory: two accumulators (whole warp)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(umma::smem_u32(&tmem_base_sh)),
+                 "r"(2 * kFusedAccCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = tmem_base_sh;
+  const int gb = D.gb, total = gb * P.M;
+  const int nkb = (P.F + umma::kBlockK - 1) / umma::kBlockK;
+  // test hook: the loader of block 0 issues nothing and the block polls with a short limit (laq_tune "starve_copies")
+  const bool starved = P.starve != 0u && blockIdx.x == 0;
+  const uint32_t limit = starved ? kStarvedWaitLimit : umma::kWaitLimit;
+
+  if (warp == 0) {
+    if (lane == 0 && !starved) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int g = blockIdx.x; g < total && ok; g += gridDim.x) {
+        const int m = g / gb, tile = g - m * gb;
+        const RowWindow win = row_window(P, m);
+        if (!fused_tile_has_rows(P, win, m, tile)) continue;
+        const int i0 = (int)(D.rowoff[m] + (long long)tile * umma::kTileM);
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const uint32_t s = it % kFusedStages, par = ((it / kFusedStages) & 1u) ^ 1u;
+          if (!umma::mbar_wait_abortable(empty0 + 8 * s, par, limit, abort_flag, err_flag, 2u)) {
+            ok = false;
+            break;
+          }
+          umma::mbar_expect_tx(full0 + 8 * s, st_bytes);
+          const uint32_t sa = smem0 + s * st_bytes;
+          umma::tma_load_2d(sa, &tmX, full0 + 8 * s, kb * umma::kBlockK, i0);
+          umma::tma_load_2d(sa + a_bytes, &tmW, full0 + 8 * s, kb * umma::kBlockK, 0);
+        }
+      }
+      if (!ok) {
+        // a wait ran out somewhere: give the copies still in flight (at most one per stage) the same bounded time to
+        // land before the block leaves
+        for (uint32_t back = 1; back <= (uint32_t)kFusedStages && back <= it; ++back) {
+          const uint32_t j = it - back;
+          umma::mbar_wait_abortable(full0 + 8 * (j % kFusedStages), (j / kFusedStages) & 1u, umma::kWaitLimit, &never_sh,
+                                    err_flag, 2u);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = umma::instr_desc_bf16(nt);
+      uint32_t it = 0, done = 0;
+      bool ok = true;
+      for (int g = blockIdx.x; g < total && ok; g += gridDim.x) {
+        const int m = g / gb, tile = g - m * gb;
+        const RowWindow win = row_window(P, m);
+        if (!fused_tile_has_rows(P, win, m, tile)) continue;
+        const uint32_t a = done & 1u, use = done >> 1;
+        // the epilogue has drained this accumulator (passes at once on its first use)
+        ok = umma::mbar_wait_abortable(acce0 + 8 * a, (use & 1u) ^ 1u, limit, abort_flag, err_flag, 16u);
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t d_tmem = tmem_base + a * kFusedAccCols;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const uint32_t s = it % kFusedStages;
+          ok = umma::mbar_wait_abortable(full0 + 8 * s, (it / kFusedStages) & 1u, limit, abort_flag, err_flag, 4u);
+          if (!ok) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t sa = smem0 + s * st_bytes;
+          const uint64_t da = umma::smem_desc_sw128(sa), db = umma::smem_desc_sw128(sa + a_bytes);
+#pragma unroll
+          for (int kk = 0; kk < umma::kBlockK / 16; ++kk)   // 16 elements = 32 bytes = 2 descriptor address units
+            umma::mma_bf16_ss(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+          umma::mma_commit(empty0 + 8 * s);                 // the stage is free once these MMAs have read it
+        }
+        if (!ok) break;
+        umma::mma_commit(accf0 + 8 * a);                    // accumulator complete
+        ++done;
+      }
+      // every product issued above has finished before the tensor memory is given back
+      umma::mma_commit(drain);
+      umma::mbar_wait_abortable(drain, 0u, umma::kWaitLimit, &never_sh, err_flag, 32u);
+    }
+  } else {
+    const int ew = warp - 2, q = warp & 3, set = ew >> 2, et = ew * 32 + lane;
+    FusedEpi epi{P, D, nt, scratch};
+    epi.load_constants(et);
+    FusedEpi::sync_all();
+    uint32_t done = 0;
+    for (int g = blockIdx.x; g < total; g += gridDim.x) {
+      const int m = g / gb, tile = g - m * gb;
+      const RowWindow win = row_window(P, m);
+      if (!fused_tile_has_rows(P, win, m, tile)) {
+        // nothing to add from this tile: its slot holds zeros (dH~ of its rows is not written, and the W1 product
+        // does not read it)
+        const int nsmall = P.H + P.C * P.H + P.C;
+        float* sp = D.spart + ((long long)m * gb + tile) * nsmall;
+        for (int i = et; i < nsmall; i += kFusedEpiThreads) sp[i] = 0.f;
+        if (et == 0) D.lpart[(long long)m * gb + tile] = 0.0;
+        continue;
+      }
+      const uint32_t a = done & 1u, use = done >> 1;
+      const bool ok = __all_sync(0xffffffffu, umma::mbar_wait_abortable(accf0 + 8 * a, use & 1u, limit, abort_flag, err_flag, 8u));
+      // all epilogue warps take the same branch (the verdicts are combined): the epilogue uses named barriers
+      if (lane == 0) epi_ok[ew] = ok ? 1 : 0;
+      FusedEpi::sync_all();
+      int all_ok = 1;
+#pragma unroll
+      for (int e = 0; e < kFusedEpiWarps; ++e) all_ok &= epi_ok[e];
+      if (!all_ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t acc_bar = acce0 + 8 * a;
+      epi.run(tmem_base + a * kFusedAccCols, q, lane, set, m, tile, win, [&]() {
+        // every epilogue thread arrives once per tile, after its last read of the accumulator
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        umma::mbar_arrive(acc_bar);
+      });
+      ++done;
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * kFusedAccCols) : "memory");
+  }
 }
 
 struct Dw1Epi {
@@ -731,9 +938,9 @@ size_t forward_smem_tc(int H) {
 
 // tiles per worker of the fused hidden kernel, or 0 if the fused epilogue cannot be used for this shape
 int fused_tiles_for(int F, int H, int C, const long long* N, int M) {
-  if (!tc_shape_ok(F, H) || C > 12) return 0;
+  if (!tc_shape_ok(F, H) || C > 10) return 0;        // the epilogue sums five pairs of classes
   const int nt1 = (H + 15) / 16 * 16;
-  if (fused_extra_floats(H) * 4 > kFusedStages * umma::stage_bytes(nt1)) return 0;   // the epilogue's scratch lives in the ring
+  if (fused_smem_bytes(nt1, H) > 226 * 1024) return 0;   // stage ring + the epilogue's scratch must fit one SM
   long long tiles = 0;
   for (int m = 0; m < M; ++m) {
     const long long t = (N[m] + umma::kTileM - 1) / umma::kTileM;
@@ -863,7 +1070,7 @@ laq_status mlp_setup_tensor_path(MlpPlan& mp, const Params& P, cudaStream_t st) 
   hp->tc = true;
   const int ft = fused_tiles_for(P.F, P.H, P.C, hp->N_host.data(), M);
   if (ft > 0 && cudaFuncSetAttribute(umma_hidden_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)umma::smem_bytes(hp->nt1, kFusedStages)) == cudaSuccess) {
+                                     (int)fused_smem_bytes(hp->nt1, P.H)) == cudaSuccess) {
     hp->fused_tiles = ft;
     hp->d.gb = ft;        // one partial slot per tile
     hp->d.window_tiles = P.batch > 0 ? 1 : 0;
@@ -891,12 +1098,12 @@ int mlp_launch_gradients(MlpPlan& mp, const Params& P, const double* theta_sq, c
   if (hp->tc) {
     mlp_pack_w1b_kernel<<<(F * H + 255) / 256, 256, 0, st>>>(P.theta, hp->d.W1b, F * H);
     if (hp->fused_tiles > 0) {
-      umma_hidden_fused_kernel<<<dim3(hp->fused_tiles, P.M), kFusedThreads,
-                                 umma::smem_bytes(hp->nt1, kFusedStages), st>>>(hp->tmX, hp->tmW, P, hp->d,
-                                                                                              hp->nt1);
+      const int tiles = hp->fused_tiles * P.M;
+      umma_hidden_fused_kernel<<<tiles < kNumSMs ? tiles : kNumSMs, kFusedThreads, fused_smem_bytes(hp->nt1, H), st>>>(
+          hp->tmX, hp->tmW, P, hp->d, hp->nt1);
       umma_dw1_kernel<<<dim3((F + hp->nt2 - 1) / hp->nt2, (H + umma::kTileM - 1) / umma::kTileM, P.M), umma::kThreads,
                         umma::smem_bytes(hp->nt2, kDw1Stages), st>>>(hp->tmD, hp->tmXT, P, hp->d, hp->nt2);
-      mlp_finalize_kernel<<<dim3((nsmall + 255) / 256, P.M), 256, 0, st>>>(P, hp->d, theta_sq);
+      mlp_finalize_kernel<<<dim3((nsmall + 31) / 32, P.M), 256, 0, st>>>(P, hp->d, theta_sq);
       return 4;
     }
     umma_hidden_kernel<<<(unsigned)((P.Ntot + umma::kTileM - 1) / umma::kTileM), umma::kThreads,
@@ -904,13 +1111,13 @@ int mlp_launch_gradients(MlpPlan& mp, const Params& P, const double* theta_sq, c
     mlp_forward_kernel<true><<<dim3(hp->d.gb, P.M), kThreads, forward_smem_tc(H), st>>>(P, hp->d);
     umma_dw1_kernel<<<dim3((F + hp->nt2 - 1) / hp->nt2, (H + umma::kTileM - 1) / umma::kTileM, P.M), umma::kThreads,
                       umma::smem_bytes(hp->nt2, kDw1Stages), st>>>(hp->tmD, hp->tmXT, P, hp->d, hp->nt2);
-    mlp_finalize_kernel<<<dim3((nsmall + 255) / 256, P.M), 256, 0, st>>>(P, hp->d, theta_sq);
+    mlp_finalize_kernel<<<dim3((nsmall + 31) / 32, P.M), 256, 0, st>>>(P, hp->d, theta_sq);
     return 5;
   }
   mlp_pack_w1_kernel<<<(F * H + 255) / 256, 256, 0, st>>>(P.theta, hp->d.W1T, F, H);
   mlp_forward_kernel<false><<<dim3(hp->d.gb, P.M), kThreads, hp->fwd_smem, st>>>(P, hp->d);
   mlp_dw1_kernel<<<dim3((F + kTK - 1) / kTK, (H + kTJ - 1) / kTJ, P.M), kThreads, 0, st>>>(P, hp->d);
-  mlp_finalize_kernel<<<dim3((nsmall + 255) / 256, P.M), 256, 0, st>>>(P, hp->d, theta_sq);
+  mlp_finalize_kernel<<<dim3((nsmall + 31) / 32, P.M), 256, 0, st>>>(P, hp->d, theta_sq);
   return 4;
 }
 

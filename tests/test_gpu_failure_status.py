@@ -53,6 +53,33 @@ def test_starved_ring_wait_runs_out_and_is_reported_as_timeout():
     ref.close()
 
 
+def test_starved_tensor_core_stage_runs_out_and_is_reported_as_timeout():
+    """The network's fused hidden-layer kernel: the loader of one block issues no tile copies, the tensor-core warp's
+    wait for the first stage runs out, the block gives its tensor memory back and returns."""
+    w = workloads.c3(n_per=300, M=3, iters=6)
+    ctx = laq.from_workload(w, trace_capacity=4)
+    ref = laq.from_workload(w, trace_capacity=4)
+    ctx.step(2)
+    ref.step(2)
+    before = ctx.get_state()
+    ctx.tune("starve_copies", 1)
+    with pytest.raises(laq.LaqError) as e:
+        ctx.step(1, trace=True)
+    assert e.value.status == laq.LAQ_ETIMEOUT
+    tr_ref = ref.step(3, trace=True)                  # the device is fine
+    ctx.tune("starve_copies", 0)
+    ctx.set_state()
+    after = ctx.get_state()
+    assert after["k"] == before["k"] == 2
+    np.testing.assert_array_equal(after["theta"], before["theta"])
+    tr = ctx.step(3, trace=True)
+    for key in tr:
+        np.testing.assert_array_equal(tr[key], tr_ref[key])
+    np.testing.assert_array_equal(ctx.get_state()["theta"], ref.get_state()["theta"])
+    ctx.close()
+    ref.close()
+
+
 def test_timeout_status_is_distinct_from_the_other_failures():
     assert len({laq.LAQ_OK, laq.LAQ_EINVAL, laq.LAQ_EWORKSPACE, laq.LAQ_ECUDA, laq.LAQ_ENONFINITE, laq.LAQ_ESTATE,
                 laq.LAQ_ETIMEOUT}) == 7
