@@ -37,7 +37,7 @@ STAGE_KERNELS = {"radius": "radius_kernel", "quantize_norms_trigger": "quantize_
                  "aggregate_theta_step": "aggregate_kernel", "local_gradient": "grad_*_kernel"}
 TRAJ_RTOL = 1e-4          # band of theta and loss around the fp64 oracle's while skip decisions agree
 
-MODE_FLAGS = {"lag": 1, "qgd": 2, "gd": 3, "stored": 4}   # quantizer off, trigger off, both, g through memory (LAQ_FLAG_*)
+MODE_FLAGS = {"lag": 1, "qgd": 2, "gd": 3, "stored": 4, "sharded": 0}   # quantizer off, trigger off, both, g through memory (LAQ_FLAG_*)
 
 # short runs of the other configurations in the default line: (workload, timed steps)
 CONFIG_RUNS = [("c0", 2000), ("c1", 500), ("c2", 1000), ("c3", 300), ("c4_b4", 100), ("c4_b2", 100),
@@ -535,6 +535,42 @@ def run_e2e(w, Ke, world, barrier):
                         "(theta and the aggregate D2H)"}
 
 
+def run_sharded(args, w, K, Wm, world, rank, local_rank, barrier):
+    """Workload suffix _sharded: the M workers are spread over the ranks (strong scaling) and every iteration
+    exchanges the uploaders' messages (radius + code stream) over NCCL; see paper_1909_07588_b200/sharded.py.
+    With one rank it runs the same split iteration without a collective."""
+    import torch
+    from paper_1909_07588_b200 import laq, sharded
+    job = sharded.ShardedLaq(lambda wd, r: laq.from_workload(w, flags=w.flags, batch=w.batch, world=wd if wd > 1 else 0,
+                                                             rank=r if wd > 1 else 0), world, rank)
+    job.step(Wm)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = job.ctx.kernel_launches()
+    sent0 = job.sent_payload_bytes
+    barrier()
+    e0.record()
+    job.step(K)
+    e1.record()
+    barrier()
+    ms = max_over_ranks(e0.elapsed_time(e1), world)
+    clocks = sampler.stop()
+    s = job.ctx.get_state(big=False)
+    line = {"metric": METRIC, "value": K / (ms * 1e-3), "unit": "iters/s", "n_gpus": world, "steps": K, "warmup": Wm,
+            "ms_per_step": ms / K, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "config": dict(workload_config(w, args.workload, world, job.ctx),
+                                                parallelism="workers spread over %d ranks, (R, codes) exchange" % world),
+            "clocks": clocks, "gpu_launches": int(job.ctx.kernel_launches() - launches0),
+            "exchange": {"payload_bytes_sent_per_step_this_rank": (job.sent_payload_bytes - sent0) / float(K),
+                         "uploads_per_step_all_ranks": None, "bits_counted": int(s["bits"]),
+                         "host_round_trips_per_step": 1},
+            "e2e": None, "roofline": None, "cpu_baseline": None}
+    job.close()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+
+
 def config_summary(name, K, local_rank, with_oracle):
     """One short run of another configuration for the default line's "configs" key."""
     w = make_workload(name)
@@ -576,6 +612,7 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     w = make_workload(args.workload)
+    sharded_run = "sharded" in args.workload.split("_")
 
     if args.impl == "reference":
         run_reference(args, w, args.workload, rank)
@@ -605,6 +642,11 @@ def main():
         torch.cuda.synchronize()
 
     K, Wm = args.steps, args.warmup
+    if sharded_run:
+        run_sharded(args, w, K, Wm, world, rank, local_rank, barrier)
+        if world > 1:
+            dist.destroy_process_group()
+        return
     ctx, r = run_timed(w, K, Wm, world, local_rank, barrier)
     sustained = run_sustained(ctx, w, args.sustained_steps, local_rank) if extras and args.sustained_steps > 0 else None
     cfg = workload_config(w, args.workload, world, ctx)

@@ -122,6 +122,14 @@ typedef struct {
                                o = fmix32(fmix32(seed_lo + (uint32) k) ^ (seed_hi + 0x9e3779b9 (m+1))) mod N_m, and
                                g_m = (N_m / B_m)(1/N) sum_window grad l_i + (N_m/N) lambda theta; the reported loss
                                is the same estimate of f */
+  int32_t world;            /* 0 or 1: all M workers live in this context.  > 1: the workers are spread over `world`
+                               contexts (one per GPU), round robin: this context runs steps 1-4 for the workers
+                               m = rank, rank + world, ... and holds their Q_m; every context holds theta, grad and
+                               the stored differences, and applies every upload (the server's side of Fig. 2 is
+                               replicated).  M, N and p keep their global meaning.  Needs the quantizer
+                               (no LAQ_FLAG_QUANT_OFF) and M >= world; driven with laq_step_local,
+                               laq_local_uploads, laq_apply_uploads instead of laq_step */
+  int32_t rank;             /* 0 .. world-1 */
 } laq_config;
 
 /* Per-iteration report of laq_step.  All pointers HOST, each may be NULL; n = n_iters of that call.
@@ -143,7 +151,8 @@ typedef struct {
 typedef struct {
   float* theta;       /* (S) [p]        theta^k */
   float* agg;         /* (S) [p]        grad^{k-1}, the server's lazily aggregated gradient */
-  float* qprev;       /* (S) [M][p]     Q_m(theta_hat_m^{k-1}) */
+  float* qprev;       /* (S) [M][p]     Q_m(theta_hat_m^{k-1}); per-worker arrays of this struct have one row per LOCAL
+                                        worker when laq_config.world > 1 */
   double* n_eps_hat;  /* (S) [M]        ||eps_hat_m||^2, the error at worker m's last upload */
   int32_t* clock;     /* (S) [M]        t_m */
   double* ring;       /* (S) [D]        stored squared differences, newest first */
@@ -185,6 +194,27 @@ laq_status laq_set_gradients(laq_ctx* ctx, const float* g, int32_t on_device);
  * while per-stage timing is on, or after laq_tune(ctx, "graphs", 0)). */
 laq_status laq_step(laq_ctx* ctx, int32_t n_iters, const laq_trace* trace);
 
+/* One iteration in two halves, for workers spread over several contexts (laq_config.world > 1; also valid for
+ * world <= 1, where the two halves together equal laq_step(ctx, 1, NULL) bit for bit).
+ *
+ * laq_step_local enqueues steps 1-4 of Algorithm 2 for this context's workers: local gradients, quantizer, norms,
+ * skip rule and clocks.  Every uploading worker's message (Eq. (6) and the text after it: the radius, 32 bits, and
+ * the b p-bit code stream) is then ready in this context: the radius through laq_local_uploads, the code stream in
+ * the workspace at byte offset  codes_offset_bytes + l code_row_bytes  for the l-th local worker (laq_query).
+ *
+ * laq_local_uploads synchronises and returns the local uploaders of the iteration in flight: *n of them, their
+ * GLOBAL worker indices m[0..*n) in ascending order and radii R[0..*n).  m, R: HOST, room for the local worker count.
+ *
+ * laq_apply_uploads enqueues step 5, the server's update, with ALL uploads of the iteration, local and remote:
+ * n uploaders, global indices m[] ascending, radii R[] (HOST).  Before the call the caller must have put the code
+ * stream of every REMOTE uploader m into this context's mailbox, at byte offset
+ * mailbox_offset_bytes + m code_row_bytes of the workspace (laq_query), ordered before this call on the context's
+ * stream.  Uploads are applied in ascending worker order, as laq_step does; Q_m is updated for local uploaders.
+ * The upload and bit counters count all n uploads, so they agree on every context. */
+laq_status laq_step_local(laq_ctx* ctx);
+laq_status laq_local_uploads(laq_ctx* ctx, int32_t* n, int32_t* m, float* R);
+laq_status laq_apply_uploads(laq_ctx* ctx, int32_t n, const int32_t* m, const float* R);
+
 /* Wait for the stream and report device-detected errors. */
 laq_status laq_sync(laq_ctx* ctx);
 
@@ -215,7 +245,9 @@ laq_status laq_tune(laq_ctx* ctx, const char* key, int32_t value);
 
 /* Read-only facts about the launch plan, for tests and reports: key "sweep_blocks_per_worker", "sweep_threads",
  * "sweep_tile_groups" (16-byte groups per staged tile of the quantize sweep over generated or stored rows),
- * "aggregate_blocks", "grad_blocks_per_worker".  Unknown keys return LAQ_EINVAL. */
+ * "aggregate_blocks", "grad_blocks_per_worker", "local_workers" (workers whose steps 1-4 run in this context),
+ * "codes_offset_bytes", "code_row_bytes", "mailbox_offset_bytes" (see laq_step_local).  Unknown keys return
+ * LAQ_EINVAL. */
 laq_status laq_query(const laq_ctx* ctx, const char* key, int64_t* value /* HOST */);
 
 /* Per-kernel device timing for measurement.  While enabled, laq_step brackets every stage of an iteration

@@ -13,7 +13,10 @@
 using namespace laq;
 
 struct laq_ctx {
-  laq_config cfg;
+  laq_config cfg;                      // cfg.M and cfg.N describe the LOCAL workers (all of them unless world > 1)
+  int world = 1, rank = 0, M_total = 0;
+  int32_t* d_up_m_in = nullptr;        // device staging of laq_apply_uploads' arguments
+  float* d_up_R_in = nullptr;
   std::vector<int64_t> N;
   std::vector<float> xi;
   Params P;
@@ -82,6 +85,14 @@ const char* check_config(const laq_config* c) {
   if (c->flags & ~(uint32_t)(LAQ_FLAG_TRIGGER_OFF | LAQ_FLAG_QUANT_OFF | LAQ_FLAG_STORE_G)) return "unknown flag";
   if ((c->flags & LAQ_FLAG_STORE_G) && c->model != LAQ_MODEL_SYNTH) return "LAQ_FLAG_STORE_G needs LAQ_MODEL_SYNTH";
   if (c->batch < 0) return "batch must be >= 0";
+  if (c->world < 0 || c->world > kMaxWorkers) return "world must be in 0..1024";
+  if (c->world > 1) {
+    if (c->rank < 0 || c->rank >= c->world) return "rank must be in 0..world-1";
+    if (c->M < c->world) return "world > 1 needs at least one worker per context (M >= world)";
+    if (c->flags & LAQ_FLAG_QUANT_OFF) return "world > 1 needs the quantizer (the upload is the coded message)";
+  } else if (c->rank != 0) {
+    return "rank must be 0 unless world > 1";
+  }
   if (c->batch > 0 && (c->model == LAQ_MODEL_SYNTH || c->model == LAQ_MODEL_EXTERNAL))
     return "batch > 0 needs a model with samples";
   const bool data = c->model == LAQ_MODEL_LOGREG_BIN || c->model == LAQ_MODEL_SOFTMAX || c->model == LAQ_MODEL_MLP2;
@@ -108,8 +119,32 @@ const char* check_config(const laq_config* c) {
   return nullptr;
 }
 
+// The workers of this context: all M, or (world > 1) the global workers rank, rank + world, ...
+int local_workers(const laq_config& c) {
+  return c.world > 1 ? (c.M - c.rank + c.world - 1) / c.world : c.M;
+}
+
+// The configuration as the rest of this file uses it: M and N describe the local workers.  Nl receives the local
+// shard sizes; *n_total the number of samples of ALL workers (the 1/N of the global loss).
+laq_config localize(const laq_config& c, std::vector<int64_t>& Nl, long long* n_total) {
+  laq_config l = c;
+  const bool data = c.model == LAQ_MODEL_LOGREG_BIN || c.model == LAQ_MODEL_SOFTMAX || c.model == LAQ_MODEL_MLP2;
+  const int Ml = local_workers(c), stride = c.world > 1 ? c.world : 1, first = c.world > 1 ? c.rank : 0;
+  Nl.assign(Ml, 0);
+  long long tot = 0;
+  if (data && c.N) {
+    for (int m = 0; m < c.M; ++m) tot += c.N[m];
+    for (int i = 0; i < Ml; ++i) Nl[i] = c.N[first + stride * i];
+  }
+  if (n_total) *n_total = tot;
+  l.M = Ml;
+  l.N = Nl.data();
+  return l;
+}
+
 struct Plan {
   size_t total = 0;
+  size_t mailbox = 0, up_q = 0, up_in_m = 0, up_in_R = 0;
   size_t sc, theta, agg, qp, g, codes, Rbits, norms, n_epshat, clock, skip, up_m, up_R, up_s, ring, xi, loss_m,
       part_q, part_d, part_t, t_skip, t_R, t_ndq, t_neps, t_rhs, t_d2, t_loss, t_up, Xptr, yptr, Ndev, cnt_grad,
       gpart, lpart, state_end, mlp;
@@ -125,9 +160,11 @@ int default_gbpw(const laq_config& c) {
   return g < 1 ? 1 : g;
 }
 
-Plan make_plan(const laq_config& c) {
+// c: the localized configuration; M_total: all workers (= c.M unless the workers are spread over contexts)
+Plan make_plan(const laq_config& c, int M_total) {
   Plan pl;
-  const size_t M = (size_t)c.M;
+  const size_t M = (size_t)c.M, Mt = (size_t)M_total;
+  const bool spread = M_total != c.M;
   pl.ps = (c.p + 15) / 16 * 16;
   pl.nv = pl.ps / 4;
   pl.cw = ((pl.ps * c.b + 31) / 32 + 3) / 4 * 4;
@@ -144,15 +181,20 @@ Plan make_plan(const laq_config& c) {
   pl.agg = take(pl.ps * 4);
   pl.qp = take(M * pl.ps * 4);
   pl.g = (c.model == LAQ_MODEL_SYNTH && !(c.flags & LAQ_FLAG_STORE_G)) ? off : take(M * pl.ps * 4);
-  pl.codes = take(M * pl.cw * 4);
+  // local code rows, then (workers spread over contexts) one mailbox row per global worker for received messages
+  pl.codes = take((M + (spread ? Mt : 0)) * pl.cw * 4);
+  pl.mailbox = pl.codes + M * pl.cw * 4;
   pl.Rbits = take(2 * M * 4);
   pl.norms = take(3 * M * 8);
   pl.n_epshat = take(M * 8);
   pl.clock = take(M * 4);
   pl.skip = take(M);
-  pl.up_m = take(M * 4);
-  pl.up_R = take(M * 4);
-  pl.up_s = take(M * 4);
+  pl.up_m = take(Mt * 4);
+  pl.up_q = take(Mt * 4);
+  pl.up_R = take(Mt * 4);
+  pl.up_s = take(Mt * 4);
+  pl.up_in_m = take(Mt * 4);
+  pl.up_in_R = take(Mt * 4);
   pl.ring = take((size_t)c.D * 8);
   pl.xi = take((size_t)c.D * 4);
   pl.loss_m = take(M * 8);
@@ -235,14 +277,14 @@ constexpr int kGraphIters = 8;       // iterations per replay of the larger grap
 constexpr int kGraphMinIters = 4;    // shorter calls go out as plain launches
 
 // The kernels of one iteration on stream st; ev (5 events) brackets the four stages when profiling.
-void enqueue_iteration(laq_ctx* ctx, cudaStream_t st, cudaEvent_t* ev) {
+void enqueue_iteration(laq_ctx* ctx, cudaStream_t st, cudaEvent_t* ev, bool first_half = false) {
   const laq_config& c = ctx->cfg;
   const Params& P = ctx->P;
   if (ev) cudaEventRecord(ev[0], st);
   const int64_t l0 = ctx->launches;
   // small problems: steps 2-5 (and, when cheap, the combination of the gradient kernels' block partials)
   // run in one single-block kernel
-  const bool small = small_iteration_applies(P);
+  const bool small = small_iteration_applies(P) && !first_half;   // the single-block kernel runs steps 2-5 as one
   const bool linear = c.model == LAQ_MODEL_LOGREG_BIN || c.model == LAQ_MODEL_SOFTMAX;
   const bool fuse_finalize = small && linear && ctx->gbpw <= 64;
   // mid-size linear models: the kernel that combines the gradient partials also takes the quantizer's radius
@@ -285,7 +327,7 @@ void enqueue_iteration(laq_ctx* ctx, cudaStream_t st, cudaEvent_t* ev) {
       ctx->launches += launch_quantize_trigger(P, ctx->ls, st);
     }
     if (ev) cudaEventRecord(ev[3], st);
-    ctx->launches += launch_aggregate(P, ctx->ls, st);
+    if (!first_half) ctx->launches += launch_aggregate(P, ctx->ls, st);
   }
   if (ev) {
     cudaEventRecord(ev[4], st);
@@ -341,7 +383,9 @@ extern "C" {
 
 size_t laq_workspace_bytes(const laq_config* cfg) {
   if (check_config(cfg)) return 0;
-  return make_plan(*cfg).total;
+  std::vector<int64_t> Nl;
+  const laq_config l = localize(*cfg, Nl, nullptr);
+  return make_plan(l, cfg->M).total;
 }
 
 laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, size_t workspace_bytes,
@@ -354,14 +398,16 @@ laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, siz
   std::memset(&ctx->P, 0, sizeof(Params));
   std::memset(&ctx->cfg, 0, sizeof(laq_config));
   if (const char* e = check_config(cfg)) return fail(ctx, LAQ_EINVAL, e);
-  ctx->cfg = *cfg;
+  long long n_total = 0;
+  ctx->cfg = localize(*cfg, ctx->N, &n_total);
   ctx->xi.assign(cfg->xi, cfg->xi + cfg->D);
   ctx->cfg.xi = ctx->xi.data();
-  ctx->N.assign(cfg->M, 0);
-  if (cfg->N && (cfg->model <= LAQ_MODEL_MLP2)) ctx->N.assign(cfg->N, cfg->N + cfg->M);
   ctx->cfg.N = ctx->N.data();
+  ctx->world = cfg->world > 1 ? cfg->world : 1;
+  ctx->rank = cfg->world > 1 ? cfg->rank : 0;
+  ctx->M_total = cfg->M;
   ctx->st = (cudaStream_t)cuda_stream;
-  const Plan pl = make_plan(ctx->cfg);
+  const Plan pl = make_plan(ctx->cfg, ctx->M_total);
   if (!d_workspace) return fail(ctx, LAQ_EWORKSPACE, "workspace is null");
   if ((uintptr_t)d_workspace % kAlign) return fail(ctx, LAQ_EWORKSPACE, "workspace must be 256-byte aligned");
   if (workspace_bytes < pl.total) return fail(ctx, LAQ_EWORKSPACE, "workspace is smaller than laq_workspace_bytes(cfg)");
@@ -377,13 +423,14 @@ laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, siz
   Params& P = ctx->P;
   const laq_config& c = ctx->cfg;
   P.M = c.M; P.b = c.b; P.D = c.D; P.tbar = c.tbar; P.clock_mode = c.clock_mode; P.model = c.model;
+  P.M_total = ctx->M_total; P.m_first = ctx->rank; P.m_stride = ctx->world;
   P.flags = c.flags;
   P.F = c.n_features; P.C = c.n_classes; P.H = c.n_hidden;
   P.p = c.p; P.ps = pl.ps; P.nv = pl.nv; P.cw = pl.cw;
   P.alpha = c.alpha; P.lambda = c.lambda;
   {
     const double a = (double)c.alpha;
-    P.trig_c = (a * a) * ((double)c.M * (double)c.M);
+    P.trig_c = (a * a) * ((double)ctx->M_total * (double)ctx->M_total);   // (7a) divides by alpha^2 M^2, M = all workers
   }
   P.sc = (DevScalars*)(ws + pl.sc);
   P.theta = (float*)(ws + pl.theta);
@@ -397,6 +444,9 @@ laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, siz
   P.clock = (int32_t*)(ws + pl.clock);
   P.skip = (uint8_t*)(ws + pl.skip);
   P.up_m = (int32_t*)(ws + pl.up_m);
+  P.up_q = (int32_t*)(ws + pl.up_q);
+  ctx->d_up_m_in = (int32_t*)(ws + pl.up_in_m);
+  ctx->d_up_R_in = (float*)(ws + pl.up_in_R);
   P.up_R = (float*)(ws + pl.up_R);
   P.up_s = (float*)(ws + pl.up_s);
   P.ring = (double*)(ws + pl.ring);
@@ -427,8 +477,9 @@ laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, siz
   P.cnt_grad = (uint32_t*)(ws + pl.cnt_grad);
   P.gpart = (float*)(ws + pl.gpart);
   P.lpart = (double*)(ws + pl.lpart);
-  P.Ntot = 0;
-  for (int m = 0; m < c.M; ++m) P.Ntot += ctx->N[m];
+  P.Ntot = n_total;      // samples of ALL workers: f = (1/N) sum_m f_m
+  P.Nloc = 0;
+  for (int m = 0; m < c.M; ++m) P.Nloc += ctx->N[m];
   ctx->gbpw_cap = pl.gbpw_cap;
   ctx->gbpw = default_gbpw(c);
   if (c.model == LAQ_MODEL_LOGREG_BIN || c.model == LAQ_MODEL_SOFTMAX) {
@@ -514,6 +565,8 @@ laq_status laq_step(laq_ctx* ctx, int32_t n_iters, const laq_trace* trace) {
     if (n_iters == 1 && !ctx->ext_g_set) return fail(ctx, LAQ_ESTATE, "laq_set_gradients has not been called");
   }
   if (trace && n_iters > c.trace_capacity) return fail(ctx, LAQ_EINVAL, "n_iters exceeds trace_capacity");
+  if (ctx->world > 1 && n_iters > 0)
+    return fail(ctx, LAQ_ESTATE, "workers are spread over contexts: use laq_step_local, laq_local_uploads, laq_apply_uploads");
   LAQ_CUDA(ctx, cudaMemsetAsync(&P.sc->trace_pos, trace ? 0 : 0xff, 4, ctx->st));  // 0xffffffff = tracing off
   int it = 0;
   if (graphs_usable(ctx) && n_iters >= kGraphMinIters) {
@@ -582,6 +635,56 @@ laq_status laq_step(laq_ctx* ctx, int32_t n_iters, const laq_trace* trace) {
   LAQ_CUDA(ctx, pull(trace->loss, P.t_loss, n * 8));
   LAQ_CUDA(ctx, pull(trace->uploads, P.t_up, n * 4));
   return check_device_error(ctx);
+}
+
+laq_status laq_step_local(laq_ctx* ctx) {
+  if (!ctx || !ctx->ws) return LAQ_EINVAL;
+  const laq_config& c = ctx->cfg;
+  if (c.flags & LAQ_FLAG_QUANT_OFF) return fail(ctx, LAQ_ESTATE, "the split iteration needs the quantizer");
+  if (needs_shards(ctx))
+    for (int m = 0; m < c.M; ++m)
+      if (!ctx->shard_loaded[m]) return fail(ctx, LAQ_ESTATE, "laq_load_shards has not been called for every worker");
+  if (c.model == LAQ_MODEL_EXTERNAL && !ctx->ext_g_set) return fail(ctx, LAQ_ESTATE, "laq_set_gradients has not been called");
+  LAQ_CUDA(ctx, cudaMemsetAsync(&ctx->P.sc->trace_pos, 0xff, 4, ctx->st));   // no per-iteration report
+  enqueue_iteration(ctx, ctx->st, nullptr, /*first_half=*/true);
+  LAQ_CUDA(ctx, cudaGetLastError());
+  ctx->ext_g_set = false;
+  return LAQ_OK;
+}
+
+laq_status laq_local_uploads(laq_ctx* ctx, int32_t* n, int32_t* m, float* R) {
+  if (!ctx || !ctx->ws) return LAQ_EINVAL;
+  if (!n || !m || !R) return fail(ctx, LAQ_EINVAL, "null pointer");
+  const Params& P = ctx->P;
+  DevScalars sc;
+  LAQ_CUDA(ctx, cudaMemcpyAsync(&sc, P.sc, sizeof(sc), cudaMemcpyDeviceToHost, ctx->st));
+  LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));
+  *n = 0;
+  if (const laq_status st = status_of_error_word(ctx, sc.err)) return st;
+  if ((int)sc.n_up > P.M) return fail(ctx, LAQ_ESTATE, "laq_local_uploads must follow laq_step_local");
+  LAQ_CUDA(ctx, cudaMemcpyAsync(m, P.up_m, 4 * (size_t)sc.n_up, cudaMemcpyDeviceToHost, ctx->st));
+  LAQ_CUDA(ctx, cudaMemcpyAsync(R, P.up_R, 4 * (size_t)sc.n_up, cudaMemcpyDeviceToHost, ctx->st));
+  LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));
+  for (uint32_t u = 0; u < sc.n_up; ++u) m[u] = ctx->rank + ctx->world * m[u];   // local row -> global worker index
+  *n = (int32_t)sc.n_up;
+  return LAQ_OK;
+}
+
+laq_status laq_apply_uploads(laq_ctx* ctx, int32_t n, const int32_t* m, const float* R) {
+  if (!ctx || !ctx->ws) return LAQ_EINVAL;
+  if (n < 0 || n > ctx->M_total || (n > 0 && (!m || !R))) return fail(ctx, LAQ_EINVAL, "bad upload list");
+  for (int u = 0; u < n; ++u)
+    if (m[u] < 0 || m[u] >= ctx->M_total || (u > 0 && m[u] <= m[u - 1]))
+      return fail(ctx, LAQ_EINVAL, "upload list must hold distinct global worker indices in ascending order");
+  if (n > 0) {
+    LAQ_CUDA(ctx, cudaMemcpyAsync(ctx->d_up_m_in, m, 4 * (size_t)n, cudaMemcpyHostToDevice, ctx->st));
+    LAQ_CUDA(ctx, cudaMemcpyAsync(ctx->d_up_R_in, R, 4 * (size_t)n, cudaMemcpyHostToDevice, ctx->st));
+    LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));      // m and R are the caller's pageable host memory
+  }
+  ctx->launches += launch_merge_uploads(ctx->P, n, ctx->d_up_m_in, ctx->d_up_R_in, ctx->st);
+  ctx->launches += launch_aggregate(ctx->P, ctx->ls, ctx->st);
+  LAQ_CUDA(ctx, cudaGetLastError());
+  return LAQ_OK;
 }
 
 laq_status laq_sync(laq_ctx* ctx) {
@@ -725,6 +828,11 @@ laq_status laq_query(const laq_ctx* ctx, const char* key, int64_t* value) {
   else if (k == "sweep_tile_groups") *value = sweep_tile_groups();
   else if (k == "aggregate_blocks") *value = aggregate_blocks(ctx->P, ctx->ls);
   else if (k == "grad_blocks_per_worker") *value = ctx->gbpw;
+  else if (k == "local_workers") *value = ctx->P.M;
+  else if (k == "codes_offset_bytes") *value = (int64_t)((const char*)ctx->P.codes - ctx->ws);
+  else if (k == "code_row_bytes") *value = (int64_t)ctx->P.cw * 4;
+  else if (k == "mailbox_offset_bytes")
+    *value = ctx->M_total != ctx->P.M ? (int64_t)((const char*)(ctx->P.codes + (size_t)ctx->P.M * ctx->P.cw) - ctx->ws) : -1;
   else return LAQ_EINVAL;
   return LAQ_OK;
 }

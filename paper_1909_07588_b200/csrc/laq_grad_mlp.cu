@@ -416,7 +416,7 @@ __global__ void __launch_bounds__(umma::kThreads) umma_hidden_kernel(const __gri
                                                                      const __grid_constant__ CUtensorMap tmW,
                                                                      const Params P, const MlpDev D, int nt) {
   umma::TileCoord tc{(int)blockIdx.x * umma::kTileM, 0, 0, (P.F + umma::kBlockK - 1) / umma::kBlockK};
-  umma::ChunkEpilogue<HiddenEpi> epi{HiddenEpi{D.Hbuf, P.theta + (long long)P.H * P.F, P.Ntot, P.H, tc.i0}, nt};
+  umma::ChunkEpilogue<HiddenEpi> epi{HiddenEpi{D.Hbuf, P.theta + (long long)P.H * P.F, P.Nloc, P.H, tc.i0}, nt};
   umma::gemm_tn_tile(&tmX, &tmW, nt, tc, &P.sc->err, epi);
 }
 
@@ -997,8 +997,8 @@ laq_status mlp_setup(MlpPlan& mp, const Params& P, const long long* N_host, void
   const size_t nsmall = (size_t)P.H + (size_t)P.C * P.H + P.C;
   hp->d.gb = forward_blocks_per_worker(P.M);
   hp->d.W1T = (__nv_bfloat16*)p; p += align256((size_t)P.F * P.H * 2);
-  hp->d.Xb = (__nv_bfloat16*)p; p += align256((size_t)P.Ntot * P.F * 2);
-  hp->d.dHb = (__nv_bfloat16*)p; p += align256((size_t)P.Ntot * P.H * 2);
+  hp->d.Xb = (__nv_bfloat16*)p; p += align256((size_t)P.Nloc * P.F * 2);
+  hp->d.dHb = (__nv_bfloat16*)p; p += align256((size_t)P.Nloc * P.H * 2);
   hp->d.spart = (float*)p; p += align256((size_t)P.M * gb_alloc * nsmall * 4);
   hp->d.lpart = (double*)p; p += align256((size_t)P.M * gb_alloc * 8);
   hp->d.rowoff = (long long*)p; p += align256((size_t)(P.M + 1) * 8);
@@ -1037,10 +1037,10 @@ laq_status mlp_setup_tensor_path(MlpPlan& mp, const Params& P, cudaStream_t st) 
   offT[0] = 0;
   for (int m = 0; m < M; ++m) offT[m + 1] = offT[m] + (hp->N_host[m] + 63) / 64 * 64;
   const long long ldT = offT[M];
-  if (ldT >= (1ll << 31) || P.Ntot >= (1ll << 31)) return LAQ_OK;
+  if (ldT >= (1ll << 31) || P.Nloc >= (1ll << 31)) return LAQ_OK;
   char* p = hp->scratch_tc;
   hp->d.W1b = (__nv_bfloat16*)p; p += align256((size_t)P.H * P.F * 2);
-  hp->d.Hbuf = (float*)p; p += align256((size_t)P.Ntot * P.H * 4);
+  hp->d.Hbuf = (float*)p; p += align256((size_t)P.Nloc * P.H * 4);
   hp->d.dHT = (__nv_bfloat16*)p; p += align256((size_t)P.H * ldT * 2);
   hp->d.XbT = (__nv_bfloat16*)p; p += align256((size_t)P.F * ldT * 2);
   hp->d.rowoffT = (long long*)p;
@@ -1052,7 +1052,7 @@ laq_status mlp_setup_tensor_path(MlpPlan& mp, const Params& P, cudaStream_t st) 
   if (cudaMemcpyAsync(hp->d.rowoffT, offT, sizeof(long long) * (M + 1), cudaMemcpyHostToDevice, st) != cudaSuccess)
     return LAQ_ECUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return LAQ_ECUDA;
-  bool ok = umma::make_map_bf16_2d(&hp->tmX, hp->d.Xb, (uint64_t)P.Ntot, (uint64_t)P.F, (uint64_t)P.F * 2, umma::kTileM);
+  bool ok = umma::make_map_bf16_2d(&hp->tmX, hp->d.Xb, (uint64_t)P.Nloc, (uint64_t)P.F, (uint64_t)P.F * 2, umma::kTileM);
   ok = ok && umma::make_map_bf16_2d(&hp->tmW, hp->d.W1b, (uint64_t)P.H, (uint64_t)P.F, (uint64_t)P.F * 2, hp->nt1);
   ok = ok && umma::make_map_bf16_2d(&hp->tmD, hp->d.dHT, (uint64_t)P.H, (uint64_t)ldT, (uint64_t)ldT * 2, umma::kTileM);
   ok = ok && umma::make_map_bf16_2d(&hp->tmXT, hp->d.XbT, (uint64_t)P.F, (uint64_t)ldT, (uint64_t)ldT * 2, hp->nt2);
@@ -1106,7 +1106,7 @@ int mlp_launch_gradients(MlpPlan& mp, const Params& P, const double* theta_sq, c
       mlp_finalize_kernel<<<dim3((nsmall + 31) / 32, P.M), 256, 0, st>>>(P, hp->d, theta_sq);
       return 4;
     }
-    umma_hidden_kernel<<<(unsigned)((P.Ntot + umma::kTileM - 1) / umma::kTileM), umma::kThreads,
+    umma_hidden_kernel<<<(unsigned)((P.Nloc + umma::kTileM - 1) / umma::kTileM), umma::kThreads,
                          umma::smem_bytes(hp->nt1), st>>>(hp->tmX, hp->tmW, P, hp->d, hp->nt1);
     mlp_forward_kernel<true><<<dim3(hp->d.gb, P.M), kThreads, forward_smem_tc(H), st>>>(P, hp->d);
     umma_dw1_kernel<<<dim3((F + hp->nt2 - 1) / hp->nt2, (H + umma::kTileM - 1) / umma::kTileM, P.M), umma::kThreads,

@@ -30,7 +30,8 @@ struct DevScalars {
 
 // Everything a kernel needs, passed by value.
 struct Params {
-  int M, b, D, tbar, clock_mode, model;
+  int M, b, D, tbar, clock_mode, model;   // M: workers whose rows live in this context
+  int M_total, m_first, m_stride;         // all workers; local worker m is global worker m_first + m_stride m
   uint32_t flags;
   int F, C, H;               // model shape
   long long p, ps, nv, cw;   // coordinates, padded row stride (floats), ps/4, code words per row
@@ -47,8 +48,9 @@ struct Params {
   double* n_epshat; // [M]
   int32_t* clock;   // [M]
   uint8_t* skip;    // [M]
-  int32_t* up_m;    // [M] uploaders in ascending order
-  float* up_R;      // [M] their radii
+  int32_t* up_m;    // [M_total] uploaders in ascending order: row of the code buffer that holds the message
+  int32_t* up_q;    // [M_total] row of Q_prev to update, -1 for an uploader whose Q_m lives in another context
+  float* up_R;      // [M_total] their radii
   float* up_s;      // [M] their grid steps 2 tau R
   double* ring;     // [D] circular
   float* xi;        // [D]
@@ -71,7 +73,8 @@ struct Params {
   uint32_t starve;           // test hook (laq_tune "starve_copies"): one loader issues no copies, see laq.h
   float cz, eta0;
   // shards
-  long long Ntot;
+  long long Ntot;            // samples of ALL workers (the 1/N of the global loss)
+  long long Nloc;            // samples resident in this context (= Ntot unless the workers are spread over contexts)
   const float* const* X;     // device array of M device pointers
   const int32_t* const* y;   // device array of M device pointers
   const long long* N;        // device [M]
@@ -192,7 +195,8 @@ __device__ __forceinline__ RowWindow row_window(const Params& P, int m) {
     return w;
   }
   const uint32_t k = (uint32_t)(P.sc->k + 1ull);
-  const uint32_t h = fmix32(fmix32(P.seed_lo + k) ^ (P.seed_hi + 0x9e3779b9u * (uint32_t)(m + 1)));
+  const uint32_t gid = (uint32_t)(P.m_first + P.m_stride * m);   // the worker's global index
+  const uint32_t h = fmix32(fmix32(P.seed_lo + k) ^ (P.seed_hi + 0x9e3779b9u * (gid + 1u)));
   w.start = (long long)(h % (uint32_t)n);
   const long long to_end = n - w.start;
   w.len_a = P.batch < to_end ? P.batch : to_end;
@@ -224,6 +228,7 @@ int launch_small_iteration(const Params& P, int gbpw_finalize, cudaStream_t st);
 int launch_innovation_trigger(const Params& P, const LaunchShape& ls, cudaStream_t st);
 int launch_quantize_trigger(const Params& P, const LaunchShape& ls, cudaStream_t st);
 int launch_aggregate(const Params& P, const LaunchShape& ls, cudaStream_t st);
+int launch_merge_uploads(const Params& P, int n, const int32_t* d_m, const float* d_R, cudaStream_t st);
 int launch_grad_logreg(const Params& P, const LaunchShape& ls, int gbpw, cudaStream_t st);
 int launch_grad_softmax(const Params& P, const LaunchShape& ls, int gbpw, cudaStream_t st);
 int launch_grad_finalize(const Params& P, int gbpw, const double* theta_sq, bool with_radius, cudaStream_t st);

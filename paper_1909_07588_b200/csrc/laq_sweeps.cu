@@ -23,9 +23,10 @@ struct Synth {
   uint32_t key;
   float cz, drift;
   __device__ __forceinline__ void init(const Params& P, int m, unsigned long long k_iter) {
-    key = fmix32(P.seed_lo ^ fmix32(P.seed_hi + 0x9e3779b9u * (uint32_t)(m + 1)));
+    const int gid = P.m_first + P.m_stride * m;     // the worker's global index
+    key = fmix32(P.seed_lo ^ fmix32(P.seed_hi + 0x9e3779b9u * (uint32_t)(gid + 1)));
     cz = P.cz;
-    float eta_m = (float)((double)P.eta0 * (double)(m + 1) / (double)P.M);
+    float eta_m = (float)((double)P.eta0 * (double)(gid + 1) / (double)P.M_total);
     drift = __fmul_rn((float)k_iter, eta_m);
   }
   // coordinates 4v .. 4v+3
@@ -447,6 +448,7 @@ __device__ void trigger_stage(const Params& P, int bpw, unsigned char* scratch) 
       if (!(s_Rb[m] & 0x80000000u)) {
         const float R = __uint_as_float(s_Rb[m]);
         P.up_m[n] = m;
+        P.up_q[n] = m;
         P.up_R[n] = R;
         P.up_s[n] = __fmul_rn(two_tau, R);
         ++n;
@@ -891,7 +893,8 @@ __device__ __forceinline__ const void* code_address(const uint32_t* row, uint32_
 // lines of the uploaders ahead, and of theta, into L2 before they are needed.
 template <int B>
 __global__ void __launch_bounds__(256, LAQ_AGG_MIN_BLOCKS) aggregate_kernel(const Params P) {
-  __shared__ int s_m[kMaxWorkers];
+  __shared__ int s_m[kMaxWorkers];     // row of the code buffer
+  __shared__ int s_q[kMaxWorkers];     // row of Q_prev, -1: the uploader's Q_m lives in another context
   __shared__ float s_R[kMaxWorkers];
   __shared__ float s_s[kMaxWorkers];
   __shared__ double sh[32];
@@ -900,6 +903,7 @@ __global__ void __launch_bounds__(256, LAQ_AGG_MIN_BLOCKS) aggregate_kernel(cons
   const int n_up = (int)P.sc->n_up;
   for (int u = threadIdx.x; u < n_up; u += blockDim.x) {
     s_m[u] = P.up_m[u];
+    s_q[u] = P.up_q[u];
     s_R[u] = P.up_R[u];
     s_s[u] = P.up_s[u];
   }
@@ -913,21 +917,18 @@ __global__ void __launch_bounds__(256, LAQ_AGG_MIN_BLOCKS) aggregate_kernel(cons
 #pragma unroll
     for (int j = 0; j < kAggAhead; ++j)
       if (j < n_up) {
-        const int m = s_m[j];
-        prefetch_l2(reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps) + v);
-        prefetch_l2(code_address<B>(P.codes + (long long)m * P.cw, v));
+        if (s_q[j] >= 0) prefetch_l2(reinterpret_cast<const float4*>(P.qp + (long long)s_q[j] * P.ps) + v);
+        prefetch_l2(code_address<B>(P.codes + (long long)s_m[j] * P.cw, v));
       }
     for (int u = 0; u < n_up; ++u) {
       if (u + kAggAhead < n_up) {
-        const int m = s_m[u + kAggAhead];
-        prefetch_l2(reinterpret_cast<const float4*>(P.qp + (long long)m * P.ps) + v);
-        prefetch_l2(code_address<B>(P.codes + (long long)m * P.cw, v));
+        const int qa = s_q[u + kAggAhead];
+        if (qa >= 0) prefetch_l2(reinterpret_cast<const float4*>(P.qp + (long long)qa * P.ps) + v);
+        prefetch_l2(code_address<B>(P.codes + (long long)s_m[u + kAggAhead] * P.cw, v));
       }
-      const int m = s_m[u];
-      float4* qptr = reinterpret_cast<float4*>(P.qp + (long long)m * P.ps) + v;
-      float4 q = *qptr;
+      const int qrow = s_q[u];
       uint32_t c[4];
-      load_codes<B>(P.codes + (long long)m * P.cw, v, c);
+      load_codes<B>(P.codes + (long long)s_m[u] * P.cw, v, c);
       const float R = s_R[u], s = s_s[u];
       // the server's recovery of the innovation from the message: dQ = 2 tau R q - R
       float d0 = __fsub_rn(__fmul_rn(s, code_to_float(c[0])), R);
@@ -941,11 +942,15 @@ __global__ void __launch_bounds__(256, LAQ_AGG_MIN_BLOCKS) aggregate_kernel(cons
         if (i + 2 >= P.p) d2 = 0.f;
         d3 = 0.f;
       }
-      q.x = __fadd_rn(q.x, d0);
-      q.y = __fadd_rn(q.y, d1);
-      q.z = __fadd_rn(q.z, d2);
-      q.w = __fadd_rn(q.w, d3);
-      *qptr = q;
+      if (qrow >= 0) {    // the worker's own copy of Q_m moves with the server's (text after Eq. (6))
+        float4* qptr = reinterpret_cast<float4*>(P.qp + (long long)qrow * P.ps) + v;
+        float4 q = *qptr;
+        q.x = __fadd_rn(q.x, d0);
+        q.y = __fadd_rn(q.y, d1);
+        q.z = __fadd_rn(q.z, d2);
+        q.w = __fadd_rn(q.w, d3);
+        *qptr = q;
+      }
       a.x = __fadd_rn(a.x, d0);  // uploads are applied in ascending worker order
       a.y = __fadd_rn(a.y, d1);
       a.z = __fadd_rn(a.z, d2);
@@ -954,6 +959,33 @@ __global__ void __launch_bounds__(256, LAQ_AGG_MIN_BLOCKS) aggregate_kernel(cons
     theta_step(P, v, a, dsum, tsum);
   }
   aggregate_finish(P, dsum, tsum, sh, &is_last);
+}
+
+// Workers spread over several contexts: the list of ALL uploaders of the iteration (global indices, ascending, with
+// their radii) replaces the list of local uploaders that the skip-rule stage left; the counters take the uploads of
+// the other contexts.  Local uploaders read their code row and own a row of Q_prev; remote ones read the mailbox row
+// of their global index.  One block.
+__global__ void __launch_bounds__(256) merge_uploads_kernel(const Params P, int n, const int32_t* __restrict__ m_global,
+                                                            const float* __restrict__ R) {
+  DevScalars* sc = P.sc;
+  if (*(volatile uint32_t*)&sc->err) return;
+  const float levels = (float)((1u << P.b) - 1u);
+  const float two_tau = __fmul_rn(2.0f, __fdiv_rn(1.0f, levels));
+  for (int u = threadIdx.x; u < n; u += blockDim.x) {
+    const int g = m_global[u];
+    const int off = g - P.m_first;
+    const bool local = off >= 0 && off % P.m_stride == 0 && off / P.m_stride < P.M;
+    P.up_m[u] = local ? off / P.m_stride : P.M + g;     // mailbox rows follow the local rows
+    P.up_q[u] = local ? off / P.m_stride : -1;
+    P.up_R[u] = R[u];
+    P.up_s[u] = __fmul_rn(two_tau, R[u]);
+  }
+  if (threadIdx.x == 0) {
+    const unsigned long long extra = (unsigned long long)n - (unsigned long long)sc->n_up;   // the remote uploads
+    sc->uploads += extra;
+    sc->bits += extra * (32ull + (unsigned long long)P.b * (unsigned long long)P.p);
+    sc->n_up = (uint32_t)n;
+  }
 }
 
 // Quantizer off: an uploader's innovation is g_m - Q_prev itself and Q_prev becomes g_m.
@@ -1317,7 +1349,8 @@ int launch_synth_fill(const Params& P, cudaStream_t st) {
 }
 
 bool small_iteration_applies(const Params& P) {
-  return P.model != LAQ_MODEL_SYNTH && !(P.flags & LAQ_FLAG_QUANT_OFF) && (long long)P.M * P.ps <= 8192;
+  return P.model != LAQ_MODEL_SYNTH && !(P.flags & LAQ_FLAG_QUANT_OFF) && (long long)P.M * P.ps <= 8192 &&
+         P.M_total == P.M;
 }
 
 int launch_small_iteration(const Params& P, int gbpw_finalize, cudaStream_t st) {
@@ -1356,6 +1389,11 @@ int launch_quantize_trigger(const Params& P, const LaunchShape& ls, cudaStream_t
     launch_quant_b<true>(P, grid, ls.sweep_threads, st);
   else
     launch_quant_b<false>(P, grid, ls.sweep_threads, st);
+  return 1;
+}
+
+int launch_merge_uploads(const Params& P, int n, const int32_t* d_m, const float* d_R, cudaStream_t st) {
+  merge_uploads_kernel<<<1, 256, 0, st>>>(P, n, d_m, d_R);
   return 1;
 }
 

@@ -18,7 +18,7 @@ FLAG_QUANT_OFF = 1
 FLAG_TRIGGER_OFF = 2
 FLAG_STORE_G = 4
 
-EXPORTS = ["laq_workspace_bytes", "laq_init", "laq_load_shards", "laq_set_gradients", "laq_step", "laq_sync",
+EXPORTS = ["laq_workspace_bytes", "laq_init", "laq_load_shards", "laq_set_gradients", "laq_step", "laq_step_local", "laq_local_uploads", "laq_apply_uploads", "laq_sync",
            "laq_get_state", "laq_get_worker", "laq_set_state", "laq_kernel_launches", "laq_tune", "laq_query", "laq_set_profiling", "laq_kernel_times", "laq_quantize_worker_static", "laq_last_error", "laq_destroy"]
 
 
@@ -34,7 +34,8 @@ class laq_config(C.Structure):
                 ("alpha", C.c_float), ("lam", C.c_float), ("b", C.c_int32), ("D", C.c_int32),
                 ("xi", C.POINTER(C.c_float)), ("tbar", C.c_int32), ("clock_mode", C.c_int32),
                 ("flags", C.c_uint32), ("seed", C.c_uint64), ("synth_sigma", C.c_float),
-                ("synth_eta0", C.c_float), ("trace_capacity", C.c_int32), ("batch", C.c_int32)]
+                ("synth_eta0", C.c_float), ("trace_capacity", C.c_int32), ("batch", C.c_int32),
+                ("world", C.c_int32), ("rank", C.c_int32)]
 
 
 class laq_trace(C.Structure):
@@ -67,6 +68,9 @@ def load_library():
     L.laq_load_shards.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int64, C.c_int32]
     L.laq_set_gradients.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
     L.laq_step.argtypes = [C.c_void_p, C.c_int32, C.POINTER(laq_trace)]
+    L.laq_step_local.argtypes = [C.c_void_p]
+    L.laq_local_uploads.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.c_void_p, C.c_void_p]
+    L.laq_apply_uploads.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
     L.laq_sync.argtypes = [C.c_void_p]
     L.laq_get_state.argtypes = [C.c_void_p, C.POINTER(laq_state)]
     L.laq_set_state.argtypes = [C.c_void_p, C.POINTER(laq_state)]
@@ -89,13 +93,13 @@ def load_library():
 
 def make_config(model, M, p, N=None, n_features=0, n_classes=0, n_hidden=0, alpha=0.02, lam=0.0, b=4, D=10,
                 xi=None, tbar=100, clock_mode=0, flags=0, seed=0, synth_sigma=0.1, synth_eta0=0.05,
-                trace_capacity=0, batch=0):
+                trace_capacity=0, batch=0, world=0, rank=0):
     """Returns (laq_config, keepalive) -- keepalive holds the numpy arrays the struct points to."""
     N_arr = np.ascontiguousarray(N if N is not None else np.zeros(max(M, 1)), dtype=np.int64)
     xi_arr = np.ascontiguousarray(xi if xi is not None else np.full(max(D, 1), 0.8 / max(D, 1)), dtype=np.float32)
     cfg = laq_config(model, M, p, N_arr.ctypes.data_as(C.POINTER(C.c_int64)), n_features, n_classes, n_hidden,
                      alpha, lam, b, D, xi_arr.ctypes.data_as(C.POINTER(C.c_float)), tbar, clock_mode, flags,
-                     seed, synth_sigma, synth_eta0, trace_capacity, batch)
+                     seed, synth_sigma, synth_eta0, trace_capacity, batch, world, rank)
     return cfg, (N_arr, xi_arr)
 
 
@@ -120,7 +124,11 @@ class Laq:
         self.device = torch.device(device if device is not None else "cuda:%d" % torch.cuda.current_device())
         self.theta0 = config.pop("theta0", None)
         self.cfg, self._keep = make_config(**config)
-        self.M, self.p, self.D, self.b = self.cfg.M, int(self.cfg.p), self.cfg.D, self.cfg.b
+        # per-worker arrays of a context have one row per LOCAL worker (all M unless the workers are spread over
+        # several contexts with world > 1); M_total keeps the global count
+        self.M_total, self.world, self.rank = self.cfg.M, max(self.cfg.world, 1), self.cfg.rank
+        self.M = (self.M_total - self.rank + self.world - 1) // self.world
+        self.p, self.D, self.b = int(self.cfg.p), self.cfg.D, self.cfg.b
         self.model = self.cfg.model
         self.trace_capacity = self.cfg.trace_capacity
         nbytes = workspace_bytes(self.cfg)
@@ -200,6 +208,38 @@ class Laq:
     def sync(self):
         self._check(self._L.laq_sync(self._h))
 
+    # -- one iteration in two halves (workers spread over several contexts) ------------------------
+    def step_local(self):
+        """Steps 1-4 for this context's workers (enqueue only)."""
+        self._check(self._L.laq_step_local(self._h))
+
+    def local_uploads(self):
+        """(global worker indices, radii) of the local uploaders of the iteration in flight (synchronises)."""
+        n = C.c_int32(0)
+        m, R = np.zeros(max(self.M, 1), np.int32), np.zeros(max(self.M, 1), np.float32)
+        self._check(self._L.laq_local_uploads(self._h, C.byref(n), _np_ptr(m), _np_ptr(R)))
+        return m[:n.value].copy(), R[:n.value].copy()
+
+    def apply_uploads(self, m, R):
+        """Step 5 with all uploads of the iteration: global worker indices (ascending) and radii."""
+        m = np.ascontiguousarray(m, dtype=np.int32)
+        R = np.ascontiguousarray(R, dtype=np.float32)
+        assert m.size == R.size
+        self._check(self._L.laq_apply_uploads(self._h, int(m.size), _np_ptr(m), _np_ptr(R)))
+
+    def code_row(self, local_worker):
+        """The code stream of a LOCAL worker's message as a view (int32 words) into the workspace."""
+        off, row = self.query("codes_offset_bytes"), self.query("code_row_bytes")
+        a = off + local_worker * row
+        return self.workspace[a:a + row].view(self._torch.int32)
+
+    def mailbox_row(self, global_worker):
+        """Where the code stream of a REMOTE worker's message must be put before apply_uploads (view, int32 words)."""
+        off, row = self.query("mailbox_offset_bytes"), self.query("code_row_bytes")
+        assert off >= 0, "this context holds all workers: it has no mailbox"
+        a = off + global_worker * row
+        return self.workspace[a:a + row].view(self._torch.int32)
+
     def get_state(self, big=True, g=False, codes=False):
         M, p, D = self.M, self.p, self.D
         W = (p * self.b + 31) // 32
@@ -264,8 +304,9 @@ def from_workload(w, trace_capacity=0, stream=None, **overrides):
               synth_sigma=w.synth_sigma, synth_eta0=w.synth_eta0, trace_capacity=trace_capacity, theta0=w.theta0)
     kw.update(overrides)
     ctx = Laq(stream=stream, **kw)
-    for m in range(len(w.X)):
-        ctx.load_shards(m, w.X[m], w.y[m])
+    world, rank = max(kw.get("world", 0), 1), kw.get("rank", 0)
+    for l, m in enumerate(range(rank, len(w.X), world)):      # shards of the local workers, by local index
+        ctx.load_shards(l, w.X[m], w.y[m])
     return ctx
 
 
