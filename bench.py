@@ -571,6 +571,31 @@ def run_sharded(args, w, K, Wm, world, rank, local_rank, barrier):
         print(json.dumps(line), flush=True)
 
 
+def two_kernel_graph_floor_us(iters=2000):
+    """Launch floor of a two-kernel iteration on this machine: a CUDA graph of eight iterations of two dependent,
+    almost empty kernels (torch element-wise adds on one float), replayed back to back; microseconds per iteration."""
+    import torch
+    x = torch.zeros(1, device="cuda")
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        for _ in range(3):
+            x.add_(1.0)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            for _ in range(8):
+                x.add_(1.0)
+                x.mul_(0.5)
+        for _ in range(20):
+            g.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(s)
+        for _ in range(iters // 8):
+            g.replay()
+        e1.record(s)
+        e1.synchronize()
+    return e0.elapsed_time(e1) * 1000.0 / (iters // 8 * 8)
+
+
 def config_summary(name, K, local_rank, with_oracle):
     """One short run of another configuration for the default line's "configs" key."""
     w = make_workload(name)
@@ -583,6 +608,14 @@ def config_summary(name, K, local_rank, with_oracle):
            "stages": [{k: s[k] for k in ("stage", "kernel", "ms", "GB/s", "frac")} for s in rf["stages"]],
            "whole_path_frac": rf["whole_path"]["frac"]}
     base = name.split("_")[0]
+    if name == "c0":
+        try:
+            out["launch_floor"] = {"us_per_iteration": two_kernel_graph_floor_us(),
+                                   "what": "graph replay of two dependent, almost empty kernels per iteration (eight "
+                                           "iterations per graph, as laq_step replays them): the floor of a two-kernel "
+                                           "iteration that is bound by launches and kernel boundaries"}
+        except Exception as e:
+            out["launch_floor"] = {"error": repr(e)[:200]}
     if with_oracle and base in ORACLE_ITERS and name == base:
         n = ORACLE_ITERS[base]
         first, cpu = first_disagreement(w, n)

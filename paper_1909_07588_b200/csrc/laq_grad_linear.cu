@@ -259,6 +259,201 @@ __global__ void __launch_bounds__(kLrThreads) grad_logreg_pair_kernel(const Para
 }
 
 // ------------------------------------------------------------------------------------------------
+// Binary logistic regression with F = 54 or 22 features (the shapes of the paper's two logistic tests; F / 2 odd).
+// A block is one loader warp and eight worker warps around a ring of kLwStages shared-memory stages of 128
+// consecutive rows.  The loader asks the copy engine for a whole tile with ONE request (cp.async.bulk, 128 F floats,
+// completion counted in bytes on the stage's "full" mbarrier); few large requests matter: an SM starts a bulk copy
+// only about every 100 ns.  A worker warp waits for the stage, works on its 16 rows of the tile and arrives on the
+// stage's "empty" mbarrier, on which the loader waits before it refills the stage: no block-wide barrier in the
+// loop, every wait bounded.
+//   scores     lane = (row, half): 8-byte reads of half of its row (row pitch F floats: the 16 lanes of a half warp
+//              hit 32 different banks), that half of theta in registers; the halves meet by one shuffle;
+//   gradient   lane = feature pair: acc += residual[row] x[row][pair] over the warp's 16 rows, the residual fetched
+//              by a shuffle, the pair by one conflict-free 8-byte read.
+// Rows start 8-byte aligned (F even).  A tile that starts 8 bytes past a 16-byte boundary (minibatch windows that
+// begin at an odd row) is placed 8 bytes into its stage, so that the bulk copy runs between 16-byte boundaries on
+// both sides; its first two floats, and the up to three floats that follow the last whole 16 bytes of a tile (the
+// last rows of a shard), are copied by lanes of the loader warp with plain loads before the request goes out.
+// ------------------------------------------------------------------------------------------------
+constexpr int kLwWarps = 8;                       // worker warps
+constexpr int kLwThreads = 32 * (kLwWarps + 1);
+constexpr int kLwRows = 128;                      // rows per tile
+constexpr int kLwWarpRows = kLwRows / kLwWarps;   // 16
+constexpr int kLwStages = 3;
+
+static size_t logreg_warp_smem(int F) { return (size_t)kLwStages * (kLwRows * F + 4) * sizeof(float); }
+static bool logreg_warp_path(int F) { return F == 54 || F == 22; }
+
+template <int FT>
+__global__ void __launch_bounds__(kLwThreads) grad_logreg_ring_kernel(const Params P, int gbpw) {
+  static_assert((FT & 3) == 2 && FT <= 64, "F / 2 must be odd and fit one lane per feature pair");
+  constexpr int F2 = FT / 2, FH = (F2 + 1) / 2;    // pairs per row; pairs of the first half
+  constexpr uint32_t kTileFloats = kLwRows * FT + 4;   // 16 bytes of slack: a tile may sit 8 bytes into its stage
+  extern __shared__ __align__(128) float smem[];
+  __shared__ __align__(8) unsigned long long bars[2 * kLwStages];
+  __shared__ float red[kLwWarps][FT];
+  __shared__ double shd[kLwWarps];
+  const int m = blockIdx.y, t = threadIdx.x, lane = t & 31, w = t >> 5;
+  const float* __restrict__ X = P.X[m];
+  const int32_t* __restrict__ y = P.y[m];
+  const uint32_t full_a = smem_addr(bars), empty_a = full_a + 8 * kLwStages;
+  if (t == 0) {
+    for (int st = 0; st < kLwStages; ++st) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(full_a + 8 * st) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty_a + 8 * st), "r"(kLwWarps) : "memory");
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  RowWindow win = row_window(P, m);
+  const int ntiles = (int)win.tiles(kLwRows);                    // N_m < 2^31
+  const int n_my = ntiles > (int)blockIdx.x ? (ntiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  float acc0 = 0.f, acc1 = 0.f;
+  double loss = 0.0;
+  if (w == kLwWarps) {
+    // ---- loader warp
+    uint32_t st = 0, round = 0;
+    for (int i = 0; i < n_my; ++i) {
+      long long r0;
+      int nr;
+      win.tile((long long)blockIdx.x + (long long)i * gridDim.x, kLwRows, r0, nr);
+      // the workers are done with what the stage held (passes at once in the first round)
+      if (!__all_sync(0xffffffffu, ring_wait(empty_a + 8 * st, (round & 1u) ^ 1u))) {
+        if (lane == 0) atomicOr(&P.sc->err, kErrRingWait);
+        break;
+      }
+      const float* src = X + r0 * FT;
+      const int total = nr * FT;                                             // floats of the tile
+      const int shift = (int)((reinterpret_cast<uintptr_t>(src) & 15u) >> 2);   // 0 or 2 floats
+      float* dst = smem + st * kTileFloats + shift;                          // row 0 of the tile in the stage
+      const int head = shift ? 2 : 0;                                        // floats before the first 16-byte boundary
+      const int body = (total - head) & ~3;                                  // whole 16-byte units
+      if (lane < head) dst[lane] = __ldg(src + lane);
+      if (lane >= 8 && lane - 8 < total - head - body) dst[head + body + lane - 8] = __ldg(src + head + body + lane - 8);
+      __syncwarp();
+      if (lane == 0) {
+        if (body > 0) {
+          ring_fetch(smem_addr(dst + head), src + head, (uint32_t)body * 4u, full_a + 8 * st);
+        } else {
+          asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(full_a + 8 * st) : "memory");
+        }
+      }
+      if (++st == (uint32_t)kLwStages) {
+        st = 0;
+        ++round;
+      }
+    }
+  } else {
+    // ---- worker warps
+    const int row = lane & 15, half = lane >> 4;
+    constexpr int kMaxHalf = FH;                   // the second half has F2 - FH = FH - 1 pairs
+    float2 thr[kMaxHalf];
+#pragma unroll
+    for (int j = 0; j < kMaxHalf; ++j)
+      thr[j] = (half == 0 || j < F2 - FH) ? __ldg(reinterpret_cast<const float2*>(P.theta) + half * FH + j) : make_float2(0.f, 0.f);
+    uint32_t st = 0, round = 0;
+    for (int i = 0; i < n_my; ++i) {
+      long long r0;
+      int nr;
+      win.tile((long long)blockIdx.x + (long long)i * gridDim.x, kLwRows, r0, nr);
+      const int wr0 = w * kLwWarpRows;               // this warp's rows of the tile: wr0 .. wr0 + 15
+      const int wnr = nr - wr0 < kLwWarpRows ? (nr - wr0 > 0 ? nr - wr0 : 0) : kLwWarpRows;
+      const int y_row = (half == 0 && row < wnr) ? __ldg(y + r0 + wr0 + row) : 0;   // asked for now, used after the scores
+      if (!__all_sync(0xffffffffu, ring_wait(full_a + 8 * st, round & 1u))) {
+        if (lane == 0) atomicOr(&P.sc->err, kErrRingWait);
+        break;
+      }
+      const int shift = (int)((reinterpret_cast<uintptr_t>(X + r0 * FT) & 15u) >> 2);   // as the loader placed the tile
+      const float* xs = smem + st * kTileFloats + shift + wr0 * FT;
+      // ---- scores: lane = (row, half of the features)
+      float res = 0.f;
+      {
+        float z0 = 0.f, z1 = 0.f;
+        if (row < wnr) {
+          const float2* xr = reinterpret_cast<const float2*>(xs + row * FT) + half * FH;
+#pragma unroll
+          for (int j = 0; j < kMaxHalf; ++j)
+            if (j < F2 - FH || half == 0) {          // only the last pair of the second half is missing
+              const float2 a = xr[j];
+              z0 = fmaf(a.x, thr[j].x, z0);
+              z1 = fmaf(a.y, thr[j].y, z1);
+            }
+        }
+        float z = z0 + z1;
+        z += __shfl_xor_sync(0xffffffffu, z, 16);    // both halves now hold the row's score (same sum in both)
+        if (half == 0 && row < wnr) {
+          const float yv = (float)y_row;
+          float sig, sp;
+          if (z >= 0.f) {
+            const float e = expf(-z);
+            sig = 1.0f / (1.0f + e);
+            sp = z + log1pf(e);
+          } else {
+            const float e = expf(z);
+            sig = e / (1.0f + e);
+            sp = log1pf(e);
+          }
+          res = sig - yv;
+          loss += (double)(sp - yv * z);
+        }
+      }
+      // ---- gradient: lane = feature pair (rows beyond a short tile are skipped: the stage may hold anything there)
+      {
+        const float2* xc = reinterpret_cast<const float2*>(xs) + (lane < F2 ? lane : 0);
+        float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
+        if (wnr == kLwWarpRows) {
+#pragma unroll
+          for (int r = 0; r < kLwWarpRows; r += 2) {
+            const float ra = __shfl_sync(0xffffffffu, res, r), rb = __shfl_sync(0xffffffffu, res, r + 1);
+            const float2 xa = xc[r * F2], xb = xc[(r + 1) * F2];
+            a0 = fmaf(ra, xa.x, a0);
+            a1 = fmaf(ra, xa.y, a1);
+            b0 = fmaf(rb, xb.x, b0);
+            b1 = fmaf(rb, xb.y, b1);
+          }
+        } else {
+          for (int r = 0; r < wnr; ++r) {
+            const float ra = __shfl_sync(0xffffffffu, res, r);
+            const float2 xa = xc[r * F2];
+            a0 = fmaf(ra, xa.x, a0);
+            a1 = fmaf(ra, xa.y, a1);
+          }
+        }
+        acc0 += a0 + b0;
+        acc1 += a1 + b1;
+      }
+      __syncwarp();                                  // every lane has read the stage
+      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_a + 8 * st) : "memory");
+      if (++st == (uint32_t)kLwStages) {
+        st = 0;
+        ++round;
+      }
+    }
+    if (lane < F2) {
+      red[w][2 * lane] = acc0;
+      red[w][2 * lane + 1] = acc1;
+    }
+    loss = warp_sum_d(loss);
+    if (lane == 0) shd[w] = loss;
+  }
+  // ---- block partial: the warps' sums in warp order.  If a wait ran out some warps stopped early; the error word
+  // is set and nothing of this iteration is used.
+  __syncthreads();
+  if (t < FT) {
+    float sum = red[0][t];
+#pragma unroll
+    for (int k = 1; k < kLwWarps; ++k) sum += red[k][t];
+    P.gpart[((long long)m * gbpw + blockIdx.x) * P.ps + t] = sum;
+  }
+  if (t == 0) {
+    double l = 0.0;
+    for (int k = 0; k < kLwWarps; ++k) l += shd[k];
+    P.lpart[(long long)m * gbpw + blockIdx.x] = l;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // C-class softmax regression, F <= 1024
 // ------------------------------------------------------------------------------------------------
 constexpr int kSmThreads = 256;
@@ -822,7 +1017,7 @@ static size_t logreg_smem(int F) {
 static size_t softmax_smem(int F, int C) { return sizeof(float) * ((size_t)kSmRows * F + (size_t)kSmRows * C); }
 
 int grad_tiles_per_worker(int model, int F, int C, long long n_max) {
-  const long long rows = (model == LAQ_MODEL_LOGREG_BIN) ? ((F & 1) ? logreg_rows(F) : kLr2Rows)
+  const long long rows = (model == LAQ_MODEL_LOGREG_BIN) ? (logreg_warp_path(F) ? kLwRows : (F & 1) ? logreg_rows(F) : kLr2Rows)
                                                          : (softmax_wide_path(F, C) ? kSwRows : 8);
   const long long t = (n_max + rows - 1) / rows;
   return (int)(t > 1024 ? 1024 : (t < 1 ? 1 : t));
@@ -831,11 +1026,24 @@ int grad_tiles_per_worker(int model, int F, int C, long long n_max) {
 // Blocks of the gradient kernel that fit on one SM (shared memory bound): the grid is sized to one such wave.
 int grad_blocks_per_sm(int model, int F, int C) {
   if (model != LAQ_MODEL_LOGREG_BIN) return softmax_wide_path(F, C) ? 1 : 2;
+  if (logreg_warp_path(F)) return (int)((227 * 1024) / (logreg_warp_smem(F) + 2048));
   const int fit = (int)((227 * 1024) / (logreg_smem(F) + 1024));
   return fit < 1 ? 1 : (fit > 8 ? 8 : fit);
 }
 
 int launch_grad_logreg(const Params& P, const LaunchShape&, int gbpw, cudaStream_t st) {
+  if (logreg_warp_path(P.F)) {
+    const size_t smw = logreg_warp_smem(P.F);
+    const dim3 gridw(gbpw, P.M);
+    if (P.F == 54) {
+      cudaFuncSetAttribute(grad_logreg_ring_kernel<54>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smw);
+      grad_logreg_ring_kernel<54><<<gridw, kLwThreads, smw, st>>>(P, gbpw);
+    } else {
+      cudaFuncSetAttribute(grad_logreg_ring_kernel<22>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smw);
+      grad_logreg_ring_kernel<22><<<gridw, kLwThreads, smw, st>>>(P, gbpw);
+    }
+    return 1;
+  }
   const size_t sm = logreg_smem(P.F);
   const dim3 grid(gbpw, P.M);
   // more than the default 48 KB of dynamic shared memory is asked for per kernel and per device; the call is cheap

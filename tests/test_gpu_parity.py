@@ -564,14 +564,15 @@ def _run_model_parity(w, iters, batch=0, grad_ctol=GRAD_CTOL, skip_tie_rtol=SKIP
         assert tr["loss"][0] == pytest.approx(st64["loss"], rel=1e-5)
         codes_gpu = np.stack([oracle.unpack_codes(gs["codes"][m], w.p, w.b) for m in range(w.M)])
         dc = codes_gpu - s64["codes"]
-        steps = np.zeros(w.M)
+        steps, ties = np.zeros(w.M), np.zeros(w.M)
         for m in range(w.M):
             R, s, t = _worker_ties(s64["g"][m], prev["qprev"][m].astype(np.float64), w.b)
             steps[m] = s
+            tie = 4.0 * grad_ctol * np.max(np.abs(s64["g"][m])) / s + 2.0 ** (w.b - 21) if s > 0 else np.inf
+            ties[m] = tie
             idx = np.nonzero(dc[m])[0]
             if idx.size == 0:
                 continue
-            tie = 4.0 * grad_ctol * np.max(np.abs(s64["g"][m])) / s + 2.0 ** (w.b - 21)
             off = np.abs(codes_gpu[m, idx] - (t[idx] - 0.5))
             assert np.all(off <= 0.5 + tie), (k, m, idx[:5], off[:5], tie)      # every flip is a near-tie
             # the gradient tolerance that would just explain the largest excess (for the report)
@@ -600,8 +601,8 @@ def _run_model_parity(w, iters, batch=0, grad_ctol=GRAD_CTOL, skip_tie_rtol=SKIP
             up = np.nonzero(tr["skip"][0] == 0)[0]
             moved = -w.alpha * (steps[up, None] * dc[up]).sum(axis=0) if up.size else 0.0
             assert np.linalg.norm(gs["theta"] - s64["theta"] - moved) <= 1e-5 * np.linalg.norm(s64["theta"]), k
-            if not dc.any():
-                np.testing.assert_allclose(tr["n_dq"][0], st64["n_dq"], rtol=0.01)
+            if not dc.any():                     # equal codes: the norms differ by the radii only
+                assert np.all(np.abs(tr["n_dq"][0] - st64["n_dq"]) <= (0.01 + 4.0 * ties) * st64["n_dq"]), k
         # (4)
         f64 = free64.step()
         if rec["first_skip_diff"] is None and not np.array_equal(f64["skip"].astype(np.uint8), tr["skip"][0]):
