@@ -37,7 +37,7 @@ STAGE_KERNELS = {"radius": "radius_kernel", "quantize_norms_trigger": "quantize_
                  "aggregate_theta_step": "aggregate_kernel", "local_gradient": "grad_*_kernel"}
 TRAJ_RTOL = 1e-4          # band of theta and loss around the fp64 oracle's while skip decisions agree
 
-MODE_FLAGS = {"lag": 1, "qgd": 2, "gd": 3, "stored": 4, "sharded": 0}   # quantizer off, trigger off, both, g through memory (LAQ_FLAG_*)
+MODE_FLAGS = {"lag": 1, "qgd": 2, "gd": 3, "stored": 4, "sparse": 8, "sharded": 0}   # quantizer off, trigger off, both, g through memory (LAQ_FLAG_*)
 
 # short runs of the other configurations in the default line: (workload, timed steps)
 CONFIG_RUNS = [("c0", 2000), ("c1", 500), ("c2", 1000), ("c3", 300), ("c4_b4", 100), ("c4_b2", 100),

@@ -87,6 +87,11 @@ enum {
                                (LAG) of Sec. 4.  R is still reported; no codes are written (they stay zero) */
   LAQ_FLAG_TRIGGER_OFF = 2u,/* every worker uploads every iteration: Algorithm 1 (QGD); with LAQ_FLAG_QUANT_OFF
                                as well: gradient descent, Eq. (2) */
+  LAQ_FLAG_SPARSE_X = 8u,   /* LAQ_MODEL_SOFTMAX only (2..10 classes, at most 896 features): laq_load_shards also
+                               makes a compressed copy of the shard (its non-zeros by rows and by columns, in tiles
+                               of 128 rows) and step 1 runs over the non-zeros only.  Same gradient up to the order
+                               of the fp32 sums.  The copies may take as many entries (6 bytes each) as the shard has
+                               elements; a denser shard makes laq_load_shards return LAQ_EWORKSPACE */
   LAQ_FLAG_STORE_G = 4u     /* LAQ_MODEL_SYNTH only: step 1 writes the M x p gradients of the iteration to the
                                workspace (as a gradient kernel does, Algorithm 2's worker step) and steps 2-5 read
                                them from memory instead of regenerating them; same values, same results */

@@ -31,6 +31,7 @@ struct laq_ctx {
   size_t ws_bytes = 0;
   std::vector<const float*> Xptr;
   std::vector<const int32_t*> yptr;
+  std::vector<void*> sp_region;        // LAQ_FLAG_SPARSE_X: where each worker's compressed copies go
   MlpPlan mlp;
   // optional per-stage timing
   bool profiling = false;
@@ -82,7 +83,9 @@ const char* check_config(const laq_config* c) {
   if (!(c->alpha > 0.f) || !std::isfinite(c->alpha)) return "alpha must be positive and finite";
   if (c->clock_mode != 0 && c->clock_mode != 1) return "clock_mode must be 0 or 1";
   if (c->trace_capacity < 0) return "trace_capacity must be >= 0";
-  if (c->flags & ~(uint32_t)(LAQ_FLAG_TRIGGER_OFF | LAQ_FLAG_QUANT_OFF | LAQ_FLAG_STORE_G)) return "unknown flag";
+  if (c->flags & ~(uint32_t)(LAQ_FLAG_TRIGGER_OFF | LAQ_FLAG_QUANT_OFF | LAQ_FLAG_STORE_G | LAQ_FLAG_SPARSE_X)) return "unknown flag";
+  if ((c->flags & LAQ_FLAG_SPARSE_X) && (c->model != LAQ_MODEL_SOFTMAX || !sparse_shape_ok(c->n_features, c->n_classes)))
+    return "LAQ_FLAG_SPARSE_X needs LAQ_MODEL_SOFTMAX with 2..10 classes and at most 896 features";
   if ((c->flags & LAQ_FLAG_STORE_G) && c->model != LAQ_MODEL_SYNTH) return "LAQ_FLAG_STORE_G needs LAQ_MODEL_SYNTH";
   if (c->batch < 0) return "batch must be >= 0";
   if (c->world < 0 || c->world > kMaxWorkers) return "world must be in 0..1024";
@@ -148,7 +151,8 @@ struct Plan {
   size_t sc, theta, agg, qp, g, codes, Rbits, norms, n_epshat, clock, skip, up_m, up_R, up_s, ring, xi, loss_m,
       part_q, part_d, part_t, t_skip, t_R, t_ndq, t_neps, t_rhs, t_d2, t_loss, t_up, Xptr, yptr, Ndev, cnt_grad,
       gpart, lpart, state_end, mlp;
-  std::vector<size_t> X, y;
+  std::vector<size_t> X, y, sp;
+  size_t sp_desc = 0;
   long long ps, nv, cw;
   int gbpw_cap;
 };
@@ -228,6 +232,10 @@ Plan make_plan(const laq_config& c, int M_total) {
       pl.X.push_back(take((size_t)c.N[m] * c.n_features * 4));
       pl.y.push_back(take((size_t)c.N[m] * 4));
     }
+    if (c.flags & LAQ_FLAG_SPARSE_X) {
+      pl.sp_desc = take(M * sizeof(SparseShard));
+      for (size_t m = 0; m < M; ++m) pl.sp.push_back(take(sparse_region_bytes(c.N[m], c.n_features)));
+    }
   }
   pl.total = off;
   return pl;
@@ -295,7 +303,8 @@ void enqueue_iteration(laq_ctx* ctx, cudaStream_t st, cudaEvent_t* ev, bool firs
       if (!fuse_finalize) ctx->launches += launch_grad_finalize(P, ctx->gbpw, &P.sc->theta_sq, fuse_radius, st);
       break;
     case LAQ_MODEL_SOFTMAX:
-      ctx->launches += launch_grad_softmax(P, ctx->ls, ctx->gbpw, st);
+      ctx->launches += (c.flags & LAQ_FLAG_SPARSE_X) ? launch_grad_softmax_sparse(P, ctx->gbpw, st)
+                                                     : launch_grad_softmax(P, ctx->ls, ctx->gbpw, st);
       if (!fuse_finalize) ctx->launches += launch_grad_finalize(P, ctx->gbpw, &P.sc->theta_sq, fuse_radius, st);
       break;
     case LAQ_MODEL_MLP2:
@@ -480,9 +489,15 @@ laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, siz
   P.Ntot = n_total;      // samples of ALL workers: f = (1/N) sum_m f_m
   P.Nloc = 0;
   for (int m = 0; m < c.M; ++m) P.Nloc += ctx->N[m];
+  P.sp = (const SparseShard*)(ws + pl.sp_desc);
+  for (size_t m = 0; m < pl.sp.size(); ++m) ctx->sp_region.push_back(ws + pl.sp[m]);
   ctx->gbpw_cap = pl.gbpw_cap;
   ctx->gbpw = default_gbpw(c);
-  if (c.model == LAQ_MODEL_LOGREG_BIN || c.model == LAQ_MODEL_SOFTMAX) {
+  if (c.flags & LAQ_FLAG_SPARSE_X) {
+    ctx->gbpw = sparse_blocks_per_worker((const long long*)ctx->N.data(), c.M);
+    if (ctx->gbpw > kGradBlocksCap) ctx->gbpw = kGradBlocksCap;
+  }
+  if ((c.model == LAQ_MODEL_LOGREG_BIN || c.model == LAQ_MODEL_SOFTMAX) && !(c.flags & LAQ_FLAG_SPARSE_X)) {
     long long n_max = 1;
     for (int m = 0; m < c.M; ++m) n_max = ctx->N[m] > n_max ? ctx->N[m] : n_max;
     const int tiles = grad_tiles_per_worker(c.model, c.n_features, c.n_classes, n_max);
@@ -533,6 +548,13 @@ laq_status laq_load_shards(laq_ctx* ctx, int32_t m, const float* X, const int32_
     long long row_offset = 0;
     for (int i = 0; i < m; ++i) row_offset += ctx->N[i];
     ctx->launches += mlp_convert_shard(ctx->mlp, ctx->P, m, ctx->Xptr[m], N_m, row_offset, ctx->st);
+  }
+  if (ctx->cfg.flags & LAQ_FLAG_SPARSE_X) {
+    std::string why;
+    const laq_status s = sparse_build(m, ctx->Xptr[m], N_m, ctx->cfg.n_features, ctx->sp_region[m],
+                                      const_cast<SparseShard*>(ctx->P.sp), ctx->st, &why);
+    if (s != LAQ_OK) return fail(ctx, s, why);
+    ctx->launches += 2;
   }
   LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));  // the caller may reuse its buffers on return
   ctx->shard_loaded[m] = 1;

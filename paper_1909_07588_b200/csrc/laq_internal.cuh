@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <string>
+
 #include "laq.h"
 
 namespace laq {
@@ -26,6 +28,15 @@ struct DevScalars {
   unsigned long long uploads;  // sum_k |M^k|
   unsigned long long bits;     // uploads x (32 + b p)
   double theta_sq;             // ||theta^k||^2 (for the regulariser term of the reported loss)
+};
+
+// A worker's shard in compressed form (LAQ_FLAG_SPARSE_X), see laq_grad_sparse.cu.
+struct SparseShard {
+  const float* val;          // values of both copies
+  const uint16_t* idx;       // feature index (copy by rows) or row in tile (copy by columns)
+  const long long* off_r;    // [tiles + 1] first entry of each tile's copy by rows
+  const long long* off_c;    // [tiles + 1] first entry of each tile's copy by columns
+  int tiles;
 };
 
 // Everything a kernel needs, passed by value.
@@ -82,6 +93,7 @@ struct Params {
   float* gpart;              // gradient partials [M][gbpw][ps]
   double* lpart;             // loss partials [M][gbpw]
   uint32_t* cnt_grad;        // [M] tickets
+  const SparseShard* sp;     // device [M], LAQ_FLAG_SPARSE_X only
 };
 
 #ifdef __CUDACC__
@@ -233,6 +245,10 @@ int launch_grad_logreg(const Params& P, const LaunchShape& ls, int gbpw, cudaStr
 int launch_grad_softmax(const Params& P, const LaunchShape& ls, int gbpw, cudaStream_t st);
 int launch_grad_finalize(const Params& P, int gbpw, const double* theta_sq, bool with_radius, cudaStream_t st);
 bool softmax_classes_supported(int C);
+bool sparse_shape_ok(int F, int C);
+size_t sparse_region_bytes(long long n, int F);
+int sparse_blocks_per_worker(const long long* N, int M);
+int launch_grad_softmax_sparse(const Params& P, int gbpw, cudaStream_t st);
 int grad_tiles_per_worker(int model, int F, int C, long long n_max);
 int grad_blocks_per_sm(int model, int F, int C);
 
@@ -250,6 +266,8 @@ int mlp_convert_shard(MlpPlan& mp, const Params& P, int m, const float* X, long 
                       cudaStream_t st);
 int mlp_launch_gradients(MlpPlan& mp, const Params& P, const double* theta_sq, cudaStream_t st);
 void mlp_teardown(MlpPlan& mp);
+laq_status sparse_build(int m, const float* X, long long n, int F, void* region, SparseShard* desc_dev, cudaStream_t st,
+                        std::string* err);
 int sweep_blocks_per_worker(const Params& P, const LaunchShape& ls);
 int sweep_tile_groups();
 int launch_theta_sq(const Params& P, cudaStream_t st);

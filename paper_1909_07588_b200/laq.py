@@ -17,6 +17,7 @@ MODEL_LOGREG_BIN, MODEL_SOFTMAX, MODEL_MLP2, MODEL_SYNTH, MODEL_EXTERNAL = range
 FLAG_QUANT_OFF = 1
 FLAG_TRIGGER_OFF = 2
 FLAG_STORE_G = 4
+FLAG_SPARSE_X = 8
 
 EXPORTS = ["laq_workspace_bytes", "laq_init", "laq_load_shards", "laq_set_gradients", "laq_step", "laq_step_local", "laq_local_uploads", "laq_apply_uploads", "laq_sync",
            "laq_get_state", "laq_get_worker", "laq_set_state", "laq_kernel_launches", "laq_tune", "laq_query", "laq_set_profiling", "laq_kernel_times", "laq_quantize_worker_static", "laq_last_error", "laq_destroy"]

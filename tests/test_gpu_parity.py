@@ -511,7 +511,7 @@ def _worker_ties(g64_m, qprev_m, b):
     return R, s, t
 
 
-def _run_model_parity(w, iters, batch=0, grad_ctol=GRAD_CTOL, skip_tie_rtol=SKIP_TIE_RTOL):
+def _run_model_parity(w, iters, batch=0, grad_ctol=GRAD_CTOL, skip_tie_rtol=SKIP_TIE_RTOL, lib_flags=0):
     """Per iteration of a model workload (gradients from the library's own kernels):
       (1) step 1 on identical input: the library's gradients at its own theta^k against the fp64 model gradient,
           in the 2-norm (GRAD_RTOL) and coordinate by coordinate (grad_ctol x the largest coordinate);
@@ -527,7 +527,7 @@ def _run_model_parity(w, iters, batch=0, grad_ctol=GRAD_CTOL, skip_tie_rtol=SKIP
           its skip masks equal the library's and none of its codes has differed yet (asserted); the first iteration
           at which a skip bit differs, a code differs, or the band is left is recorded.
     Returns the record."""
-    ctx = laq.from_workload(w, trace_capacity=1, batch=batch)
+    ctx = laq.from_workload(w, trace_capacity=1, batch=batch, flags=lib_flags)   # lib_flags: layout choices of the library
     free64 = _mirror_for(w, 64, batch=batch)
     # step64 is stepped once per iteration, so its k (which the window start depends on) stays the library's
     step64 = _mirror_for(w, 64, batch=batch)
@@ -704,6 +704,44 @@ def test_c2_full_size_first_iterations():
 def test_c3_full_size_first_iterations():
     w = workloads.c3(iters=3)
     assert _first(_run_model_parity(w, 3)) > 3
+
+
+# ---- softmax regression over a compressed copy of the shards (LAQ_FLAG_SPARSE_X): the same comparisons
+def test_sparse_softmax_reduced_ragged_tiles():
+    w = workloads.c1(n_per=333, iters=40)                 # 333 = 2 x 128 + 77 rows: a short last tile
+    rec = _run_model_parity(w, w.iters, lib_flags=laq.FLAG_SPARSE_X)
+    assert _first(rec) > 30
+
+
+def test_sparse_softmax_odd_shapes_and_odd_class_count():
+    w = workloads.c1(n_per=37, F=50, C=3, M=4, iters=15)  # three classes: padded to four inside the kernel
+    _run_model_parity(w, w.iters, lib_flags=laq.FLAG_SPARSE_X)
+
+
+def test_sparse_softmax_minibatch_windows():
+    w = workloads.c1(n_per=1203, iters=40)
+    rec = _run_model_parity(w, w.iters, batch=500, lib_flags=laq.FLAG_SPARSE_X)
+    assert _first(rec) > 8
+
+
+def test_sparse_softmax_full_size_first_iterations():
+    w = workloads.c1(iters=6)
+    assert _first(_run_model_parity(w, 6, lib_flags=laq.FLAG_SPARSE_X)) > 6
+
+
+def test_sparse_copy_rejects_a_dense_shard():
+    rng = np.random.default_rng(0)
+    M, n, F, C = 2, 300, 40, 4
+    X = [rng.standard_normal((n, F)).astype(np.float32) for _ in range(M)]       # no zeros at all
+    y = [rng.integers(0, C, n).astype(np.int32) for _ in range(M)]
+    ctx = laq.Laq(model=laq.MODEL_SOFTMAX, M=M, p=C * F, N=[n] * M, n_features=F, n_classes=C, alpha=0.1, lam=0.01,
+                  b=4, flags=laq.FLAG_SPARSE_X)
+    with pytest.raises(laq.LaqError) as e:
+        ctx.load_shards(0, X[0], y[0])
+    assert e.value.status == laq.LAQ_EWORKSPACE and "too dense" in str(e.value)
+    ctx.close()
+    with pytest.raises(laq.LaqError):
+        laq.Laq(model=laq.MODEL_LOGREG_BIN, M=2, p=10, N=[5, 5], n_features=10, flags=laq.FLAG_SPARSE_X)
 
 
 def test_softmax_small_odd_shapes():
