@@ -44,11 +44,19 @@ struct MlpDev {          // device pointers inside the scratch area
   // tensor-core path
   __nv_bfloat16* W1b;    // [H][F]
   float* Hbuf;           // [Ntot][H]  hidden activations
-  __nv_bfloat16* dHT;    // [H][ldT]   dH~ transposed
-  __nv_bfloat16* XbT;    // [F][ldT]   X~ transposed
+  // The transposed copies are stored in blocks of 64 rows of the data (= 64 columns of the transposed matrix):
+  // element (j, col) at ((col / 64) rpk + j) 64 + col mod 64, so that the tile of a K block that the W1-gradient
+  // product loads is one contiguous piece of memory instead of one 128-byte piece per row, 2 ldT bytes apart.
+  __nv_bfloat16* dHT;    // dH~ transposed, rpk = rpk_d (H rounded up to the 128-row tiles of the product)
+  __nv_bfloat16* XbT;    // X~ transposed, rpk = rpk_x (F rounded up to the product's column tiles)
   long long* rowoffT;    // [M+1] prefix sums of N_m rounded up to 64
   long long ldT;         // sum of the rounded shard sizes
+  int rpk_d, rpk_x;
 };
+
+__host__ __device__ __forceinline__ long long blocked_index(long long j, long long col, int rpk) {
+  return ((col >> 6) * rpk + j) * 64 + (col & 63);
+}
 
 __global__ void __launch_bounds__(256) mlp_pack_w1_kernel(const float* __restrict__ theta, __nv_bfloat16* __restrict__ W1T,
                                                           int F, int H) {
@@ -247,7 +255,7 @@ __global__ void __launch_bounds__(kThreads) mlp_forward_kernel(const Params P, c
 #pragma unroll
           for (int c = 0; c < 8; ++c) {
             __nv_bfloat16 v4[4] = {dht[0][c], dht[1][c], dht[2][c], dht[3][c]};   // rows >= nr hold dh = 0
-            *reinterpret_cast<uint2*>(D.dHT + (long long)(8 * cg + c) * D.ldT + col) = *reinterpret_cast<const uint2*>(v4);
+            *reinterpret_cast<uint2*>(D.dHT + blocked_index(8 * cg + c, col, D.rpk_d)) = *reinterpret_cast<const uint2*>(v4);
           }
         }
       }
@@ -377,7 +385,7 @@ __global__ void __launch_bounds__(256) mlp_pack_w1b_kernel(const float* __restri
 
 // XbT[k][col0 + r] = bf16(X[r][k]) for one shard (done once, when the shard is loaded)
 __global__ void __launch_bounds__(256) mlp_transpose_x_kernel(const float* __restrict__ X, __nv_bfloat16* __restrict__ XbT,
-                                                              long long n, int F, long long ldT, long long col0) {
+                                                              long long n, int F, int rpk, long long col0) {
   __shared__ float tile[32][33];
   const long long r0 = (long long)blockIdx.x * 32;
   const int k0 = blockIdx.y * 32, tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
@@ -385,7 +393,7 @@ __global__ void __launch_bounds__(256) mlp_transpose_x_kernel(const float* __res
     tile[i][tx] = (r0 + i < n && k0 + tx < F) ? __ldg(X + (r0 + i) * F + k0 + tx) : 0.f;
   __syncthreads();
   for (int i = ty; i < 32; i += 8)
-    if (k0 + i < F && r0 + tx < n) XbT[(long long)(k0 + i) * ldT + col0 + r0 + tx] = __float2bfloat16_rn(tile[tx][i]);
+    if (k0 + i < F && r0 + tx < n) XbT[blocked_index(k0 + i, col0 + r0 + tx, rpk)] = __float2bfloat16_rn(tile[tx][i]);
 }
 
 struct HiddenEpi {
@@ -613,7 +621,7 @@ struct FusedEpi {
           unpack2(d2, d_even, d_odd);
           const float d = d_even + d_odd;
           dh = h > 0.f ? d : 0.f;
-          if (in_segment) D.dHT[(long long)j * D.ldT + col] = __float2bfloat16_rn(dh);
+          if (in_segment) D.dHT[blocked_index(j, col, D.rpk_d)] = __float2bfloat16_rn(dh);
         }
         chunk_h[tt * kFusedPitch + i] = h;
         chunk_d[tt * kFusedPitch + i] = dh;
@@ -882,6 +890,8 @@ __global__ void __launch_bounds__(umma::kThreads) umma_dw1_kernel(const __grid_c
   const int m = blockIdx.z;
   const long long c0 = D.rowoffT[m], c1 = D.rowoffT[m + 1];
   umma::TileCoord tc{(int)blockIdx.y * umma::kTileM, (int)blockIdx.x * nt, (int)c0, (int)((c1 - c0) / umma::kBlockK)};
+  tc.a_rpk = D.rpk_d;
+  tc.b_rpk = D.rpk_x;
   const long long n = P.N[m];
   if (D.window_tiles) {
     // minibatch: only the 128-row tiles that meet the window were written by the hidden kernel in this iteration;
@@ -927,6 +937,11 @@ int forward_blocks_per_worker(int M) {
   int g = (2 * kNumSMs + M - 1) / M;
   return g < 1 ? 1 : (g > 64 ? 64 : g);
 }
+
+// column tile of the W1-gradient product and the rows per K block of the two blocked transposed copies
+int dw1_nt(int F) { return (F % 112 == 0) ? 112 : ((F >= 128) ? 128 : (F + 15) / 16 * 16); }
+int rpk_d_for(int H) { return (H + umma::kTileM - 1) / umma::kTileM * umma::kTileM; }
+int rpk_x_for(int F) { return (F + dw1_nt(F) - 1) / dw1_nt(F) * dw1_nt(F); }
 
 // the tcgen05 path needs 16-byte row pitches for its tensor maps
 bool tc_shape_ok(int F, int H) { return (F % 8) == 0 && (H % 8) == 0 && H >= 16 && H <= 256; }
@@ -982,8 +997,8 @@ size_t mlp_scratch_bytes(const laq_config& c) {
     for (int m = 0; m < c.M; ++m) ldT += (c.N[m] + 63) / 64 * 64;
     b += align256((size_t)c.n_hidden * c.n_features * 2);        // W1b
     b += align256((size_t)Ntot * c.n_hidden * 4);                // Hbuf
-    b += align256((size_t)c.n_hidden * ldT * 2);                 // dHT
-    b += align256((size_t)c.n_features * ldT * 2);               // XbT
+    b += align256((size_t)rpk_d_for(c.n_hidden) * ldT * 2);      // dHT
+    b += align256((size_t)rpk_x_for(c.n_features) * ldT * 2);    // XbT
     b += align256((size_t)(c.M + 1) * 8);                        // rowoffT
   }
   return b;
@@ -1041,21 +1056,24 @@ laq_status mlp_setup_tensor_path(MlpPlan& mp, const Params& P, cudaStream_t st) 
   char* p = hp->scratch_tc;
   hp->d.W1b = (__nv_bfloat16*)p; p += align256((size_t)P.H * P.F * 2);
   hp->d.Hbuf = (float*)p; p += align256((size_t)P.Nloc * P.H * 4);
-  hp->d.dHT = (__nv_bfloat16*)p; p += align256((size_t)P.H * ldT * 2);
-  hp->d.XbT = (__nv_bfloat16*)p; p += align256((size_t)P.F * ldT * 2);
+  hp->d.rpk_d = rpk_d_for(P.H);
+  hp->d.rpk_x = rpk_x_for(P.F);
+  hp->d.dHT = (__nv_bfloat16*)p; p += align256((size_t)hp->d.rpk_d * ldT * 2);
+  hp->d.XbT = (__nv_bfloat16*)p; p += align256((size_t)hp->d.rpk_x * ldT * 2);
   hp->d.rowoffT = (long long*)p;
   hp->d.ldT = ldT;
   hp->nt1 = (P.H + 15) / 16 * 16;
-  hp->nt2 = (P.F % 112 == 0) ? 112 : ((P.F >= 128) ? 128 : (P.F + 15) / 16 * 16);
-  if (cudaMemsetAsync(hp->d.dHT, 0, (size_t)P.H * ldT * 2, st) != cudaSuccess) return LAQ_ECUDA;
-  if (cudaMemsetAsync(hp->d.XbT, 0, (size_t)P.F * ldT * 2, st) != cudaSuccess) return LAQ_ECUDA;
+  hp->nt2 = dw1_nt(P.F);
+  if (cudaMemsetAsync(hp->d.dHT, 0, (size_t)hp->d.rpk_d * ldT * 2, st) != cudaSuccess) return LAQ_ECUDA;
+  if (cudaMemsetAsync(hp->d.XbT, 0, (size_t)hp->d.rpk_x * ldT * 2, st) != cudaSuccess) return LAQ_ECUDA;
   if (cudaMemcpyAsync(hp->d.rowoffT, offT, sizeof(long long) * (M + 1), cudaMemcpyHostToDevice, st) != cudaSuccess)
     return LAQ_ECUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return LAQ_ECUDA;
   bool ok = umma::make_map_bf16_2d(&hp->tmX, hp->d.Xb, (uint64_t)P.Nloc, (uint64_t)P.F, (uint64_t)P.F * 2, umma::kTileM);
   ok = ok && umma::make_map_bf16_2d(&hp->tmW, hp->d.W1b, (uint64_t)P.H, (uint64_t)P.F, (uint64_t)P.F * 2, hp->nt1);
-  ok = ok && umma::make_map_bf16_2d(&hp->tmD, hp->d.dHT, (uint64_t)P.H, (uint64_t)ldT, (uint64_t)ldT * 2, umma::kTileM);
-  ok = ok && umma::make_map_bf16_2d(&hp->tmXT, hp->d.XbT, (uint64_t)P.F, (uint64_t)ldT, (uint64_t)ldT * 2, hp->nt2);
+  // blocked copies: 64 columns, (ldT / 64) rpk rows
+  ok = ok && umma::make_map_bf16_2d(&hp->tmD, hp->d.dHT, (uint64_t)(ldT / 64) * hp->d.rpk_d, 64, 128, umma::kTileM);
+  ok = ok && umma::make_map_bf16_2d(&hp->tmXT, hp->d.XbT, (uint64_t)(ldT / 64) * hp->d.rpk_x, 64, 128, hp->nt2);
   if (!ok) return LAQ_OK;   // plain kernels
   if (cudaFuncSetAttribute(umma_hidden_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)umma::smem_bytes(hp->nt1)) != cudaSuccess ||
@@ -1087,7 +1105,7 @@ int mlp_convert_shard(MlpPlan& mp, const Params& P, int m, const float* X, long 
   mlp_pack_x_kernel<<<kNumSMs * 4, 256, 0, st>>>(X, hp->d.Xb + row_offset * P.F, cnt);
   if (!hp->tc) return 1;
   mlp_transpose_x_kernel<<<dim3((unsigned)((n + 31) / 32), (unsigned)((P.F + 31) / 32)), 256, 0, st>>>(
-      X, hp->d.XbT, n, P.F, hp->d.ldT, hp->offT_host[m]);
+      X, hp->d.XbT, n, P.F, hp->d.rpk_x, hp->offT_host[m]);
   return 2;
 }
 

@@ -146,9 +146,13 @@ __host__ __device__ constexpr uint32_t tmem_cols(int nt) { return nt <= 32 ? 32u
 // Which part of the problem a CTA works on: tile origin in A rows (i0) and B rows (j0), and the K range
 // [k0, k0 + 64 nkb) in elements.  With nkb_first < nkb the range is in two pieces: the first nkb_first blocks
 // start at k0, the remaining ones at k1 (a row window that wraps around the end of a shard).
+// a_rpk / b_rpk > 0: the operand is stored in K blocks, element (row r, column k) at
+// ((k / 64) rpk + r) 64 + k mod 64, so that a tile of a K block is one contiguous piece of memory; its tensor map
+// then has 64 columns and (K / 64) rpk rows.
 struct TileCoord {
   int i0, j0, k0, nkb;
   int k1 = 0, nkb_first = 0x7fffffff;
+  int a_rpk = 0, b_rpk = 0;
   __device__ __forceinline__ int k_of(int kb) const {
     return kb < nkb_first ? k0 + kb * kBlockK : k1 + (kb - nkb_first) * kBlockK;
   }
@@ -239,8 +243,9 @@ __device__ __forceinline__ void gemm_tn_tile(const CUtensorMap* tmA, const CUten
         if (!mbar_wait(empty0 + 8 * s, par, err_flag, 2u)) break;
         mbar_expect_tx(full0 + 8 * s, st_bytes);
         const uint32_t sa = smem0 + s * st_bytes;
-        tma_load_2d(sa, tmA, full0 + 8 * s, tc.k_of(kb), tc.i0);
-        tma_load_2d(sa + a_bytes, tmB, full0 + 8 * s, tc.k_of(kb), tc.j0);
+        const int k = tc.k_of(kb);
+        tma_load_2d(sa, tmA, full0 + 8 * s, tc.a_rpk ? 0 : k, tc.a_rpk ? (k / kBlockK) * tc.a_rpk + tc.i0 : tc.i0);
+        tma_load_2d(sa + a_bytes, tmB, full0 + 8 * s, tc.b_rpk ? 0 : k, tc.b_rpk ? (k / kBlockK) * tc.b_rpk + tc.j0 : tc.j0);
       }
     }
   } else if (warp == 1) {
