@@ -530,19 +530,26 @@ struct FusedEpi {
     for (int c0 = kFusedChunk * set; c0 < nt; c0 += kStep) {
       uint32_t v[kFusedChunk];
       umma::tmem_load_16(taddr + (uint32_t)c0, v);
+      const float* wch = w2 + c0 * 12;                 // this chunk's rows of W2^T and entries of b1
+      const float* bch = b1v + c0;
+      const int ncol = H - c0 < kFusedChunk ? H - c0 : kFusedChunk;   // columns of the chunk that exist (<= 0: none)
+      auto score = [&](int i) {
+        const float h = fmaxf(__uint_as_float(v[i]) + bch[i], 0.f);
+        const unsigned long long hh = pack2(h, h);
+        const ulonglong2 wa = *reinterpret_cast<const ulonglong2*>(wch + i * 12);
+        const ulonglong2 wb = *reinterpret_cast<const ulonglong2*>(wch + i * 12 + 4);
+        const ulonglong2 wc = *reinterpret_cast<const ulonglong2*>(wch + i * 12 + 8);
+        z2[0] = ffma2(hh, wa.x, z2[0]); z2[1] = ffma2(hh, wa.y, z2[1]);
+        z2[2] = ffma2(hh, wb.x, z2[2]); z2[3] = ffma2(hh, wb.y, z2[3]);
+        z2[4] = ffma2(hh, wc.x, z2[4]); z2[5] = ffma2(hh, wc.y, z2[5]);
+      };
+      if (ncol == kFusedChunk) {                       // every chunk but the last: no per-column test
 #pragma unroll
-      for (int i = 0; i < kFusedChunk; ++i) {
-        const int j = c0 + i;
-        if (j < H) {
-          const float h = fmaxf(__uint_as_float(v[i]) + b1v[j], 0.f);
-          const unsigned long long hh = pack2(h, h);
-          const ulonglong2 wa = *reinterpret_cast<const ulonglong2*>(w2 + j * 12);
-          const ulonglong2 wb = *reinterpret_cast<const ulonglong2*>(w2 + j * 12 + 4);
-          const ulonglong2 wc = *reinterpret_cast<const ulonglong2*>(w2 + j * 12 + 8);
-          z2[0] = ffma2(hh, wa.x, z2[0]); z2[1] = ffma2(hh, wa.y, z2[1]);
-          z2[2] = ffma2(hh, wb.x, z2[2]); z2[3] = ffma2(hh, wb.y, z2[3]);
-          z2[4] = ffma2(hh, wc.x, z2[4]); z2[5] = ffma2(hh, wc.y, z2[5]);
-        }
+        for (int i = 0; i < kFusedChunk; ++i) score(i);
+      } else {
+#pragma unroll
+        for (int i = 0; i < kFusedChunk; ++i)
+          if (i < ncol) score(i);
       }
     }
     {
@@ -604,27 +611,41 @@ struct FusedEpi {
         released();
         released_yet = true;
       }
+      const float* wch = w2 + c0 * 12;
+      const float* bch = b1v + c0;
+      const int ncol = H - c0 < kFusedChunk ? H - c0 : kFusedChunk;
+      __nv_bfloat16* dcol = D.dHT + blocked_index(c0, col, D.rpk_d);   // column c0 + i of this row: dcol[64 i]
+      float* ph = chunk_h + tt * kFusedPitch;
+      float* pd = chunk_d + tt * kFusedPitch;
+      auto back = [&](int i) {
+        const float h = fmaxf(__uint_as_float(v[i]) + bch[i], 0.f);
+        const ulonglong2 wa = *reinterpret_cast<const ulonglong2*>(wch + i * 12);
+        const ulonglong2 wb = *reinterpret_cast<const ulonglong2*>(wch + i * 12 + 4);
+        const ulonglong2 wc = *reinterpret_cast<const ulonglong2*>(wch + i * 12 + 8);
+        // even and odd classes in the two halves of a packed sum, added at the end
+        unsigned long long d2 = ffma2(dz2[0], wa.x, 0ull);
+        d2 = ffma2(dz2[1], wa.y, d2); d2 = ffma2(dz2[2], wb.x, d2); d2 = ffma2(dz2[3], wb.y, d2);
+        d2 = ffma2(dz2[4], wc.x, d2); d2 = ffma2(dz2[5], wc.y, d2);
+        float d_even, d_odd;
+        unpack2(d2, d_even, d_odd);
+        const float dh = h > 0.f ? d_even + d_odd : 0.f;
+        if (in_segment) dcol[64 * i] = __float2bfloat16_rn(dh);
+        ph[i] = h;
+        pd[i] = dh;
+      };
+      if (ncol == kFusedChunk) {
 #pragma unroll
-      for (int i = 0; i < kFusedChunk; ++i) {
-        const int j = c0 + i;
-        float h = 0.f, dh = 0.f;
-        if (j < H) {
-          h = fmaxf(__uint_as_float(v[i]) + b1v[j], 0.f);
-          const ulonglong2 wa = *reinterpret_cast<const ulonglong2*>(w2 + j * 12);
-          const ulonglong2 wb = *reinterpret_cast<const ulonglong2*>(w2 + j * 12 + 4);
-          const ulonglong2 wc = *reinterpret_cast<const ulonglong2*>(w2 + j * 12 + 8);
-          // even and odd classes in the two halves of a packed sum, added at the end
-          unsigned long long d2 = ffma2(dz2[0], wa.x, 0ull);
-          d2 = ffma2(dz2[1], wa.y, d2); d2 = ffma2(dz2[2], wb.x, d2); d2 = ffma2(dz2[3], wb.y, d2);
-          d2 = ffma2(dz2[4], wc.x, d2); d2 = ffma2(dz2[5], wc.y, d2);
-          float d_even, d_odd;
-          unpack2(d2, d_even, d_odd);
-          const float d = d_even + d_odd;
-          dh = h > 0.f ? d : 0.f;
-          if (in_segment) D.dHT[blocked_index(j, col, D.rpk_d)] = __float2bfloat16_rn(dh);
+        for (int i = 0; i < kFusedChunk; ++i) back(i);
+      } else {
+#pragma unroll
+        for (int i = 0; i < kFusedChunk; ++i) {
+          if (i < ncol) {
+            back(i);
+          } else {
+            ph[i] = 0.f;
+            pd[i] = 0.f;
+          }
         }
-        chunk_h[tt * kFusedPitch + i] = h;
-        chunk_d[tt * kFusedPitch + i] = dh;
       }
       sync_set(set);
       {
