@@ -2,7 +2,7 @@
 // products of the ReLU-network gradient:
 //     D[i][j] = sum_k A[i][k] * B[j][k]        A: [rows_a][K] row-major, B: [rows_b][K] row-major (both K-major)
 // One CTA computes one 128 x NT tile of D (NT a multiple of 16, 16 <= NT <= 256):
-//   warp 0     one lane issues the TMA loads (cp.async.bulk.tensor, 128-byte swizzle, no multicast) of the
+//   warp 0     one lane issues the TMA loads (cp.async.bulk.tensor, 128-byte swizzle; every block fetches its own tiles) of the
 //              128 x 64 tile of A and the NT x 64 tile of B into a ring of kStages shared-memory stages;
 //   warp 1     allocates tensor memory; one lane issues tcgen05.mma (M = 128, N = NT, K = 16, four per stage) with
 //              the accumulator in tensor memory, and commits each stage back to the loader through an mbarrier;
