@@ -521,6 +521,9 @@ laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, siz
       if (s == LAQ_OK) s = mlp_set_row_offsets(ctx->mlp, (const long long*)ctx->N.data(), c.M, ctx->st);
       if (s == LAQ_OK) s = mlp_setup_tensor_path(ctx->mlp, P, ctx->st);
       if (s != LAQ_OK) return fail(ctx, s, "network scratch set-up failed");
+      // tensor-core path: the theta step keeps the bf16 copy of W1 current (H F is a multiple of 4 there)
+      P.w1b = (uint16_t*)mlp_w1_copy(ctx->mlp);
+      P.w1b_n = P.w1b ? (long long)c.n_hidden * c.n_features : 0;
     }
   }
   std::vector<int32_t> clocks(c.M, c.tbar + 1);  // every worker uploads at k = 1
@@ -530,6 +533,7 @@ laq_status laq_init(laq_ctx** out, const laq_config* cfg, void* d_workspace, siz
     LAQ_CUDA(ctx, cudaMemcpyAsync(P.theta, theta0, 4 * (size_t)c.p, cudaMemcpyHostToDevice, ctx->st));
     ctx->launches += launch_theta_sq(P, ctx->st);        // ||theta^0||^2 for the regulariser term of the loss
   }
+  if (c.model == LAQ_MODEL_MLP2) ctx->launches += mlp_refresh_w1_copy(ctx->mlp, P, ctx->st);   // theta^0 (or zeros)
   LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));  // the host vectors above go out of scope
   return LAQ_OK;
 }
@@ -820,6 +824,7 @@ laq_status laq_set_state(laq_ctx* ctx, const laq_state* in) {
   LAQ_CUDA(ctx, cudaMemsetAsync(P.Rbits, 0, 2 * M * 4, ctx->st));
   LAQ_CUDA(ctx, cudaMemcpyAsync(P.sc, &sc, sizeof(sc), cudaMemcpyHostToDevice, ctx->st));
   if (in->theta) ctx->launches += launch_theta_sq(P, ctx->st);   // after the scalars: it overwrites theta_sq
+  if (in->theta && ctx->cfg.model == LAQ_MODEL_MLP2) ctx->launches += mlp_refresh_w1_copy(ctx->mlp, P, ctx->st);
   LAQ_CUDA(ctx, cudaStreamSynchronize(ctx->st));
   return LAQ_OK;
 }

@@ -950,6 +950,9 @@ struct HostPlan {
   int nt1 = 0, nt2 = 0;     // N tiles of the two products
   int fused_tiles = 0;      // > 0: the hidden product runs with the fused epilogue, this many tiles per worker
   CUtensorMap tmX, tmW, tmD, tmXT;
+  // the small-gradient kernel runs beside the W1 product (both only read what the fused kernel wrote)
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 };
 
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
@@ -1107,6 +1110,12 @@ laq_status mlp_setup_tensor_path(MlpPlan& mp, const Params& P, cudaStream_t st) 
   }
   hp->offT_host.assign(offT, offT + M + 1);
   hp->tc = true;
+  if (cudaStreamCreateWithFlags(&hp->side, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&hp->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&hp->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+    cudaGetLastError();
+    hp->side = nullptr;            // everything on the caller's stream then
+  }
   const int ft = fused_tiles_for(P.F, P.H, P.C, hp->N_host.data(), M);
   if (ft > 0 && cudaFuncSetAttribute(umma_hidden_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)fused_smem_bytes(hp->nt1, P.H)) == cudaSuccess) {
@@ -1135,15 +1144,26 @@ int mlp_launch_gradients(MlpPlan& mp, const Params& P, const double* theta_sq, c
   const int F = P.F, H = P.H, C = P.C;
   const int nsmall = H + C * H + C;
   if (hp->tc) {
-    mlp_pack_w1b_kernel<<<(F * H + 255) / 256, 256, 0, st>>>(P.theta, hp->d.W1b, F * H);
+    // the bf16 copy of W1 is kept up to date by the theta step (Params::w1b); without that hook it is made here
+    int extra = 0;
+    if (P.w1b == nullptr) {
+      mlp_pack_w1b_kernel<<<(F * H + 255) / 256, 256, 0, st>>>(P.theta, hp->d.W1b, F * H);
+      extra = 1;
+    }
     if (hp->fused_tiles > 0) {
       const int tiles = hp->fused_tiles * P.M;
       umma_hidden_fused_kernel<<<tiles < kNumSMs ? tiles : kNumSMs, kFusedThreads, fused_smem_bytes(hp->nt1, H), st>>>(
           hp->tmX, hp->tmW, P, hp->d, hp->nt1);
+      // fork: the small-gradient kernel on a side stream, the W1 product on the caller's; join before the sweeps
+      // (the same pattern inside a stream capture makes the two kernels siblings in the graph)
+      const bool forked = hp->side != nullptr && cudaEventRecord(hp->ev_fork, st) == cudaSuccess &&
+                          cudaStreamWaitEvent(hp->side, hp->ev_fork, 0) == cudaSuccess;
+      mlp_finalize_kernel<<<dim3((nsmall + 31) / 32, P.M), 256, 0, forked ? hp->side : st>>>(P, hp->d, theta_sq);
+      if (forked) cudaEventRecord(hp->ev_join, hp->side);
       umma_dw1_kernel<<<dim3((F + hp->nt2 - 1) / hp->nt2, (H + umma::kTileM - 1) / umma::kTileM, P.M), umma::kThreads,
                         umma::smem_bytes(hp->nt2, kDw1Stages), st>>>(hp->tmD, hp->tmXT, P, hp->d, hp->nt2);
-      mlp_finalize_kernel<<<dim3((nsmall + 31) / 32, P.M), 256, 0, st>>>(P, hp->d, theta_sq);
-      return 4;
+      if (forked) cudaStreamWaitEvent(st, hp->ev_join, 0);
+      return 3 + extra;
     }
     umma_hidden_kernel<<<(unsigned)((P.Nloc + umma::kTileM - 1) / umma::kTileM), umma::kThreads,
                          umma::smem_bytes(hp->nt1), st>>>(hp->tmX, hp->tmW, P, hp->d, hp->nt1);
@@ -1151,7 +1171,7 @@ int mlp_launch_gradients(MlpPlan& mp, const Params& P, const double* theta_sq, c
     umma_dw1_kernel<<<dim3((F + hp->nt2 - 1) / hp->nt2, (H + umma::kTileM - 1) / umma::kTileM, P.M), umma::kThreads,
                       umma::smem_bytes(hp->nt2, kDw1Stages), st>>>(hp->tmD, hp->tmXT, P, hp->d, hp->nt2);
     mlp_finalize_kernel<<<dim3((nsmall + 31) / 32, P.M), 256, 0, st>>>(P, hp->d, theta_sq);
-    return 5;
+    return 4 + extra;
   }
   mlp_pack_w1_kernel<<<(F * H + 255) / 256, 256, 0, st>>>(P.theta, hp->d.W1T, F, H);
   mlp_forward_kernel<false><<<dim3(hp->d.gb, P.M), kThreads, hp->fwd_smem, st>>>(P, hp->d);
@@ -1160,7 +1180,25 @@ int mlp_launch_gradients(MlpPlan& mp, const Params& P, const double* theta_sq, c
   return 4;
 }
 
+void* mlp_w1_copy(const MlpPlan& mp) {
+  const HostPlan* hp = (const HostPlan*)mp.scratch;
+  return (hp && hp->tc) ? (void*)hp->d.W1b : nullptr;
+}
+
+int mlp_refresh_w1_copy(MlpPlan& mp, const Params& P, cudaStream_t st) {
+  HostPlan* hp = (HostPlan*)mp.scratch;
+  if (!hp || !hp->tc) return 0;
+  mlp_pack_w1b_kernel<<<(P.F * P.H + 255) / 256, 256, 0, st>>>(P.theta, hp->d.W1b, P.F * P.H);
+  return 1;
+}
+
 void mlp_teardown(MlpPlan& mp) {
+  HostPlan* hp = (HostPlan*)mp.scratch;
+  if (hp) {
+    if (hp->side) cudaStreamDestroy(hp->side);
+    if (hp->ev_fork) cudaEventDestroy(hp->ev_fork);
+    if (hp->ev_join) cudaEventDestroy(hp->ev_join);
+  }
   delete (HostPlan*)mp.scratch;
   mp.scratch = nullptr;
 }

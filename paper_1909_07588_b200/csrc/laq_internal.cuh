@@ -94,6 +94,8 @@ struct Params {
   double* lpart;             // loss partials [M][gbpw]
   uint32_t* cnt_grad;        // [M] tickets
   const SparseShard* sp;     // device [M], LAQ_FLAG_SPARSE_X only
+  uint16_t* w1b;             // network, tensor-core path: bf16 copy of theta's first w1b_n coordinates (W1), kept up
+  long long w1b_n;           // to date by the theta step (null / 0 otherwise)
 };
 
 #ifdef __CUDACC__
@@ -265,6 +267,8 @@ laq_status mlp_setup_tensor_path(MlpPlan& mp, const Params& P, cudaStream_t st);
 int mlp_convert_shard(MlpPlan& mp, const Params& P, int m, const float* X, long long n, long long row_offset,
                       cudaStream_t st);
 int mlp_launch_gradients(MlpPlan& mp, const Params& P, const double* theta_sq, cudaStream_t st);
+void* mlp_w1_copy(const MlpPlan& mp);   // the bf16 copy of W1 that the tensor-core path reads (null: plain path)
+int mlp_refresh_w1_copy(MlpPlan& mp, const Params& P, cudaStream_t st);   // after theta was set from outside
 void mlp_teardown(MlpPlan& mp);
 laq_status sparse_build(int m, const float* X, long long n, int F, void* region, SparseShard* desc_dev, cudaStream_t st,
                         std::string* err);

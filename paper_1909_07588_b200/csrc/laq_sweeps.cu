@@ -11,6 +11,8 @@
 //
 // Compiled with -fmad=false: every fp32 operation below is a single IEEE round-to-nearest
 // operation, in the order documented in laq.h; fused multiply-adds appear only where written.
+#include <cuda_bf16.h>
+
 #include "laq_internal.cuh"
 
 namespace laq {
@@ -831,6 +833,13 @@ __device__ __forceinline__ void theta_step(const Params& P, uint32_t v, const fl
   th.z = __fsub_rn(th.z, u2);
   th.w = __fsub_rn(th.w, u3);
   th4[v] = th;
+  if (P.w1b != nullptr && 4ll * v < P.w1b_n) {   // the network's first-layer weights, as the tensor cores read them
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(th.x, th.y), hi = __floats2bfloat162_rn(th.z, th.w);
+    uint2 pk;
+    pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+    pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+    reinterpret_cast<uint2*>(P.w1b)[v] = pk;
+  }
   dsum = fma((double)u0, (double)u0, dsum);
   dsum = fma((double)u1, (double)u1, dsum);
   dsum = fma((double)u2, (double)u2, dsum);
