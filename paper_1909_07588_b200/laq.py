@@ -241,15 +241,20 @@ class Laq:
         a = off + global_worker * row
         return self.workspace[a:a + row].view(self._torch.int32)
 
-    def get_state(self, big=True, g=False, codes=False):
+    def get_state(self, big=True, g=False, codes=False, agg=True, buffers=None):
+        """Copies state to host arrays (synchronises).  big / g / codes / agg select the large fields;
+        ``buffers`` may supply the destination arrays by field name (e.g. views of pinned host memory, which the
+        copies then land in at PCIe speed); the others are allocated here."""
         M, p, D = self.M, self.p, self.D
         W = (p * self.b + 31) // 32
-        out = dict(theta=np.zeros(p, np.float32), agg=np.zeros(p, np.float32),
+        out = dict(theta=np.zeros(p, np.float32) if not (buffers and "theta" in buffers) else buffers["theta"],
+                   agg=(np.zeros(p, np.float32) if not (buffers and "agg" in buffers) else buffers["agg"]) if agg else None,
                    qprev=np.zeros((M, p), np.float32) if big else None,
                    n_eps_hat=np.zeros(M), clock=np.zeros(M, np.int32), ring=np.zeros(D), counters=np.zeros(3, np.int64),
                    g=np.zeros((M, p), np.float32) if g else None,
                    codes=np.zeros((M, W), np.uint32) if codes else None,
                    R=np.zeros(M, np.float32), n_dq=np.zeros(M), n_eps=np.zeros(M), skip=np.zeros(M, np.uint8))
+        assert out["theta"].dtype == np.float32 and out["theta"].size == p and out["theta"].flags["C_CONTIGUOUS"]
         st = laq_state(*[_np_ptr(out[k]) for k in ("theta", "agg", "qprev", "n_eps_hat", "clock", "ring", "counters",
                                                    "g", "codes", "R", "n_dq", "n_eps", "skip")])
         self._check(self._L.laq_get_state(self._h, C.byref(st)))
