@@ -861,7 +861,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) umma_hidden_fused_kernel(con
       }
       const uint32_t a = done & 1u, use = done >> 1;
       const bool ok = __all_sync(0xffffffffu, umma::mbar_wait_abortable(accf0 + 8 * a, use & 1u, limit, abort_flag, err_flag, 8u));
-      // all epilogue warps take the same branch (the verdicts are combined): the epilogue uses named barriers
+      // all epilogue warps take the same branch (the outcomes are combined): the epilogue uses named barriers
       if (lane == 0) epi_ok[ew] = ok ? 1 : 0;
       FusedEpi::sync_all();
       int all_ok = 1;

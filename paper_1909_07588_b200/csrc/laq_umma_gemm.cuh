@@ -270,7 +270,7 @@ __device__ __forceinline__ void gemm_tn_tile(const CUtensorMap* tmA, const CUten
     const int q = warp & 3;                         // the TMEM lane quarter this warp may read
     const bool ok = __all_sync(0xffffffffu, mbar_wait(accum, 0u, err_flag, 8u));
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    // all epilogue warps take the same branch (the verdicts are combined), so an epilogue may use
+    // all epilogue warps take the same branch (the outcomes are combined), so an epilogue may use
     // its named barriers
     __shared__ int epi_ok[EPI_WARPS];
     if (lane == 0) epi_ok[warp - 2] = (ok && tc.nkb > 0) ? 1 : 0;
