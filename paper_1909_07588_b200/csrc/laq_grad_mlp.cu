@@ -439,7 +439,7 @@ __global__ void __launch_bounds__(umma::kThreads) umma_hidden_kernel(const __gri
 // Sixteen epilogue warps: four sets of four.  A set's four warps cover the four lane quarters of tensor memory
 // (all 128 rows); the sets share the 16-column chunks of the accumulator round robin in both passes.
 #ifndef LAQ_DW1_STAGES
-#define LAQ_DW1_STAGES 4
+#define LAQ_DW1_STAGES 5
 #endif
 constexpr int kDw1Stages = LAQ_DW1_STAGES;   // ring depth of the W1-gradient product (one block per SM)
 
