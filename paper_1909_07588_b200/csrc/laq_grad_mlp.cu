@@ -458,8 +458,7 @@ constexpr int kFusedPitch = kFusedChunk + 1;           // row pitch of a chunk p
 constexpr int kFusedPlane = 128 * kFusedPitch;         // one plane: 128 rows of a chunk
 
 __host__ __device__ inline size_t fused_extra_floats(int H) {
-  return (size_t)H * 12 + (size_t)((H + 3) & ~3) + (size_t)kFusedSets * 2 * kFusedPlane + 128 * 12 + (size_t)12 * H +
-         (size_t)((H + 3) & ~3) + 16;
+  return (size_t)H * 12 + (size_t)kFusedSets * 2 * kFusedPlane + 128 * 12 + (size_t)12 * H + (size_t)((H + 3) & ~3) + 16;
 }
 __host__ __device__ inline size_t fused_smem_bytes(int nt, int H) {
   return kFusedStages * umma::stage_bytes(nt) + 1024 + fused_extra_floats(H) * 4;
@@ -480,21 +479,19 @@ struct FusedEpi {
     }
   }
   __device__ __forceinline__ float* w2t() const { return base; }                                   // [H][12]
-  __device__ __forceinline__ float* b1s() const { return base + (size_t)P.H * 12; }               // [H]
-  __device__ __forceinline__ float* chunks() const { return b1s() + ((P.H + 3) & ~3); }           // [sets][h, dh][128][17]
+  __device__ __forceinline__ float* chunks() const { return base + (size_t)P.H * 12; }            // [sets][h, dh][128][17]
 
-  // once per block: W2 transposed (j-major, rows of 12) and b1 into shared memory
+  // once per block: W2 transposed (j-major, rows of 12: ten classes at most, then b1[j], then zero) into shared
+  // memory, so that the three 16-byte reads of a row bring the bias along
   __device__ __forceinline__ void load_constants(int et) const {
     const int H = P.H, C = P.C;
     const float* __restrict__ b1 = P.theta + (long long)H * P.F;
     const float* __restrict__ W2 = b1 + H;
     float* w = w2t();
-    float* b = b1s();
     for (int i = et; i < H * 12; i += kFusedEpiThreads) {
       const int j = i / 12, c = i - 12 * j;
-      w[i] = (c < C) ? __ldg(W2 + (size_t)c * H + j) : 0.f;
+      w[i] = (c < C) ? __ldg(W2 + (size_t)c * H + j) : (c == 10 ? __ldg(b1 + j) : 0.f);
     }
-    for (int i = et; i < H; i += kFusedEpiThreads) b[i] = __ldg(b1 + i);
   }
 
   // One tile.  tmem_acc: the accumulator's first column; released(): called by every epilogue thread after its last
@@ -506,7 +503,6 @@ struct FusedEpi {
     const int tt = q * 32 + lane;            // 0..127: the tile row this thread owns
     const int et = set * 128 + tt;           // among the epilogue threads
     const float* w2 = w2t();
-    const float* b1v = b1s();
     float* ch = chunks();
     float* dzs = ch + kFusedSets * 2 * kFusedPlane;   // [128][12]
     float* accA = dzs + 128 * 12;            // [12][H]
@@ -524,24 +520,23 @@ struct FusedEpi {
     const uint32_t taddr = tmem_acc + ((uint32_t)(q * 32) << 16);
     constexpr int kStep = kFusedChunk * kFusedSets;
     // ---- pass 1: partial scores over this set's chunks, as packed pairs of classes z2[k] = (z[2k], z[2k+1])
-    unsigned long long z2[6];
+    unsigned long long z2[5];
 #pragma unroll
-    for (int c = 0; c < 6; ++c) z2[c] = 0ull;
+    for (int c = 0; c < 5; ++c) z2[c] = 0ull;
     for (int c0 = kFusedChunk * set; c0 < nt; c0 += kStep) {
       uint32_t v[kFusedChunk];
       umma::tmem_load_16(taddr + (uint32_t)c0, v);
-      const float* wch = w2 + c0 * 12;                 // this chunk's rows of W2^T and entries of b1
-      const float* bch = b1v + c0;
+      const float* wch = w2 + c0 * 12;                 // this chunk's rows of W2^T (with b1 in slot 10)
       const int ncol = H - c0 < kFusedChunk ? H - c0 : kFusedChunk;   // columns of the chunk that exist (<= 0: none)
       auto score = [&](int i) {
-        const float h = fmaxf(__uint_as_float(v[i]) + bch[i], 0.f);
-        const unsigned long long hh = pack2(h, h);
         const ulonglong2 wa = *reinterpret_cast<const ulonglong2*>(wch + i * 12);
         const ulonglong2 wb = *reinterpret_cast<const ulonglong2*>(wch + i * 12 + 4);
         const ulonglong2 wc = *reinterpret_cast<const ulonglong2*>(wch + i * 12 + 8);
+        const float h = fmaxf(__uint_as_float(v[i]) + __uint_as_float((uint32_t)wc.y), 0.f);
+        const unsigned long long hh = pack2(h, h);
         z2[0] = ffma2(hh, wa.x, z2[0]); z2[1] = ffma2(hh, wa.y, z2[1]);
         z2[2] = ffma2(hh, wb.x, z2[2]); z2[3] = ffma2(hh, wb.y, z2[3]);
-        z2[4] = ffma2(hh, wc.x, z2[4]); z2[5] = ffma2(hh, wc.y, z2[5]);
+        z2[4] = ffma2(hh, wc.x, z2[4]);
       };
       if (ncol == kFusedChunk) {                       // every chunk but the last: no per-column test
 #pragma unroll
@@ -556,7 +551,7 @@ struct FusedEpi {
       ulonglong2* zp = reinterpret_cast<ulonglong2*>(zpart + (set * 128 + tt) * 12);
       zp[0] = make_ulonglong2(z2[0], z2[1]);
       zp[1] = make_ulonglong2(z2[2], z2[3]);
-      zp[2] = make_ulonglong2(z2[4], z2[5]);
+      zp[2] = make_ulonglong2(z2[4], 0ull);
     }
     sync_all();
     float dz[12];
@@ -595,9 +590,9 @@ struct FusedEpi {
     }
     sync_all();   // dZ is published; nobody reads the partial scores any more (the chunk buffers take their place)
     // ---- pass 2
-    unsigned long long dz2[6];
+    unsigned long long dz2[5];
 #pragma unroll
-    for (int c = 0; c < 6; ++c) dz2[c] = pack2(dz[2 * c], dz[2 * c + 1]);
+    for (int c = 0; c < 5; ++c) dz2[c] = pack2(dz[2 * c], dz[2 * c + 1]);
     const long long col = D.rowoffT[m] + trow;
     const bool in_segment = col < D.rowoffT[m + 1];        // rows of the padded segment (zeros beyond the shard)
     // column phase: this thread sums the columns 2 cg, 2 cg + 1 of a chunk over the rows 32 q + rho + 2 k, k = 0..7;
@@ -612,20 +607,19 @@ struct FusedEpi {
         released_yet = true;
       }
       const float* wch = w2 + c0 * 12;
-      const float* bch = b1v + c0;
       const int ncol = H - c0 < kFusedChunk ? H - c0 : kFusedChunk;
       __nv_bfloat16* dcol = D.dHT + blocked_index(c0, col, D.rpk_d);   // column c0 + i of this row: dcol[64 i]
       float* ph = chunk_h + tt * kFusedPitch;
       float* pd = chunk_d + tt * kFusedPitch;
       auto back = [&](int i) {
-        const float h = fmaxf(__uint_as_float(v[i]) + bch[i], 0.f);
         const ulonglong2 wa = *reinterpret_cast<const ulonglong2*>(wch + i * 12);
         const ulonglong2 wb = *reinterpret_cast<const ulonglong2*>(wch + i * 12 + 4);
         const ulonglong2 wc = *reinterpret_cast<const ulonglong2*>(wch + i * 12 + 8);
+        const float h = fmaxf(__uint_as_float(v[i]) + __uint_as_float((uint32_t)wc.y), 0.f);
         // even and odd classes in the two halves of a packed sum, added at the end
         unsigned long long d2 = ffma2(dz2[0], wa.x, 0ull);
         d2 = ffma2(dz2[1], wa.y, d2); d2 = ffma2(dz2[2], wb.x, d2); d2 = ffma2(dz2[3], wb.y, d2);
-        d2 = ffma2(dz2[4], wc.x, d2); d2 = ffma2(dz2[5], wc.y, d2);
+        d2 = ffma2(dz2[4], wc.x, d2);
         float d_even, d_odd;
         unpack2(d2, d_even, d_odd);
         const float dh = h > 0.f ? d_even + d_odd : 0.f;
