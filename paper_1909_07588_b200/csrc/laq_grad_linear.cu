@@ -779,7 +779,9 @@ __global__ void __launch_bounds__(256) grad_finalize_kernel(const Params P, int 
 //   softmax    one thread per (row, class), a row's classes in neighbouring lanes: sum of the partials in a fixed
 //              order, maximum and sum of the row by shuffles (the same order in every lane of a row), residual, loss;
 //              the row's label is asked for before the score product;
-//   gradient   thread = four consecutive features: acc[4][C] += residual[r][c] x[r][f] over the tile's rows.
+//   gradient   thread = four consecutive features: acc[4][C] += residual[r][c] x[r][f] over the tile's rows, as packed
+//              pairs of classes: a row's residuals are read once as they lie (three broadcast reads, 40 bytes) and
+//              each of the thread's four samples is doubled in a register.
 // Every offset is an immediate and every loop has a known trip count.
 // ------------------------------------------------------------------------------------------------
 constexpr int kSwThreads = 256;
@@ -814,7 +816,7 @@ __global__ void __launch_bounds__(kSwThreads, 1) grad_softmax_wide_kernel(const 
   float* xs0 = smem;                                  // [stages][rows][FP]
   float* ths = xs0 + kSwStages * kSwRows * FP;        // [C][F]
   float* plog = ths + C * F;                          // [28][24][C]
-  float* res = plog + kSwParts * RC;                  // [rows][12][2] residuals, each stored twice (packed pairs)
+  float* res = plog + kSwParts * RC;                  // [rows][12] residuals (slots C .. 11 stay zero)
   __shared__ double shd[kSwThreads / 32];
   __shared__ __align__(8) unsigned long long bars[kSwStages];
   const int m = blockIdx.y, t = threadIdx.x, lane = t & 31, w = t >> 5;
@@ -842,15 +844,19 @@ __global__ void __launch_bounds__(kSwThreads, 1) grad_softmax_wide_kernel(const 
   }
   for (int i = t; i < C * F4; i += kSwThreads)
     reinterpret_cast<float4*>(ths)[i] = __ldg(reinterpret_cast<const float4*>(P.theta) + i);
+  for (int i = t; i < kSwRows * 12; i += kSwThreads) res[i] = 0.f;
   __syncthreads();
   if (w == kSwWarps)   // the first tiles of this block, one per stage but the last
     for (int s = 0; s < kSwStages - 1; ++s)
       if ((long long)blockIdx.x + (long long)s * gridDim.x < ntiles) request(blockIdx.x + (long long)s * gridDim.x, s);
 
   const bool owner = t < F4;                          // gradient phase: thread t owns features 4t .. 4t+3
-  unsigned long long acc01[C], acc23[C];              // packed pairs (features 4t, 4t+1) and (4t+2, 4t+3)
+  constexpr int CP = (C + 1) / 2;                     // pairs of classes (2k, 2k+1)
+  unsigned long long acc[4][CP];                      // [feature][pair of classes]
 #pragma unroll
-  for (int c = 0; c < C; ++c) acc01[c] = acc23[c] = 0ull;
+  for (int f = 0; f < 4; ++f)
+#pragma unroll
+    for (int c = 0; c < CP; ++c) acc[f][c] = 0ull;
   double loss = 0.0;
   const int rg = lane & 7, kp = lane >> 3;
   // softmax phase: warp w owns rows kSwRpl w .. kSwRpl w + kSwRpl - 1, lane = (row within the warp, class)
@@ -936,8 +942,7 @@ __global__ void __launch_bounds__(kSwThreads, 1) grad_softmax_wide_kernel(const 
       const bool live = row_rc < nr;
       const float inv = 1.0f / sum;
       const float rv = live ? (e * inv - (cls_rc == yv ? 1.f : 0.f)) : 0.f;
-      res[(row_rc * 12 + cls_rc) * 2] = rv;
-      res[(row_rc * 12 + cls_rc) * 2 + 1] = rv;
+      res[row_rc * 12 + cls_rc] = rv;
       if (live && cls_rc == 0) loss += (double)((zmax + logf(sum)) - zy);
     }
     __syncthreads();
@@ -945,18 +950,24 @@ __global__ void __launch_bounds__(kSwThreads, 1) grad_softmax_wide_kernel(const 
       const float* xc = xs + 4 * t;
 #pragma unroll 4
       for (int r = 0; r < kSwRows; ++r) {             // rows beyond the piece hold zero residuals and zero samples
-        const ulonglong2 x = *reinterpret_cast<const ulonglong2*>(xc + r * FP);
-        const ulonglong2* rp = reinterpret_cast<const ulonglong2*>(res + r * 24);
-#pragma unroll
-        for (int c = 0; c < C; c += 2) {
-          const ulonglong2 rr = rp[c >> 1];           // (r_c, r_c), (r_c+1, r_c+1)
-          acc01[c] = ffma2(rr.x, x.x, acc01[c]);
-          acc23[c] = ffma2(rr.x, x.y, acc23[c]);
-          if (c + 1 < C) {
-            acc01[c + 1] = ffma2(rr.y, x.x, acc01[c + 1]);
-            acc23[c + 1] = ffma2(rr.y, x.y, acc23[c + 1]);
+        const float4 x = *reinterpret_cast<const float4*>(xc + r * FP);
+        const unsigned long long xx[4] = {pack2(x.x, x.x), pack2(x.y, x.y), pack2(x.z, x.z), pack2(x.w, x.w)};
+        unsigned long long rr[6];                     // (r_0, r_1), (r_2, r_3), ...
+        {
+          const ulonglong2 a = *reinterpret_cast<const ulonglong2*>(res + r * 12);
+          rr[0] = a.x;
+          rr[1] = a.y;
+          if (CP > 2) {
+            const ulonglong2 b = *reinterpret_cast<const ulonglong2*>(res + r * 12 + 4);
+            rr[2] = b.x;
+            rr[3] = b.y;
           }
+          if (CP > 4) rr[4] = *reinterpret_cast<const unsigned long long*>(res + r * 12 + 8);
         }
+#pragma unroll
+        for (int c = 0; c < CP; ++c)
+#pragma unroll
+          for (int f = 0; f < 4; ++f) acc[f][c] = ffma2(rr[c], xx[f], acc[f][c]);
       }
     }
     if (++s == kSwStages) {
@@ -979,11 +990,14 @@ __global__ void __launch_bounds__(kSwThreads, 1) grad_softmax_wide_kernel(const 
   float* gp = P.gpart + ((long long)m * gbpw + blockIdx.x) * P.ps;
   if (owner) {
 #pragma unroll
-    for (int c = 0; c < C; ++c) {
-      float4 v;
-      unpack2(acc01[c], v.x, v.y);
-      unpack2(acc23[c], v.z, v.w);
-      *reinterpret_cast<float4*>(gp + c * F + 4 * t) = v;
+    for (int c = 0; c < CP; ++c) {
+      float4 lo, hi;                                  // classes 2c and 2c + 1
+      unpack2(acc[0][c], lo.x, hi.x);
+      unpack2(acc[1][c], lo.y, hi.y);
+      unpack2(acc[2][c], lo.z, hi.z);
+      unpack2(acc[3][c], lo.w, hi.w);
+      *reinterpret_cast<float4*>(gp + (2 * c) * F + 4 * t) = lo;
+      if (2 * c + 1 < C) *reinterpret_cast<float4*>(gp + (2 * c + 1) * F + 4 * t) = hi;
     }
   }
   loss = warp_sum_d(loss);
