@@ -458,7 +458,7 @@ constexpr int kFusedPitch = kFusedChunk + 1;           // row pitch of a chunk p
 constexpr int kFusedPlane = 128 * kFusedPitch;         // one plane: 128 rows of a chunk
 
 __host__ __device__ inline size_t fused_extra_floats(int H) {
-  return (size_t)H * 12 + (size_t)kFusedSets * 2 * kFusedPlane + 128 * 12 + (size_t)12 * H + (size_t)((H + 3) & ~3) + 16;
+  return (size_t)H * 12 + 16 + (size_t)kFusedSets * 2 * kFusedPlane + 128 * 12 + (size_t)12 * H + (size_t)((H + 3) & ~3) + 16;
 }
 __host__ __device__ inline size_t fused_smem_bytes(int nt, int H) {
   return kFusedStages * umma::stage_bytes(nt) + 1024 + fused_extra_floats(H) * 4;
@@ -479,7 +479,8 @@ struct FusedEpi {
     }
   }
   __device__ __forceinline__ float* w2t() const { return base; }                                   // [H][12]
-  __device__ __forceinline__ float* chunks() const { return base + (size_t)P.H * 12; }            // [sets][h, dh][128][17]
+  __device__ __forceinline__ float* b2s() const { return base + (size_t)P.H * 12; }               // [16]: b2, then zeros
+  __device__ __forceinline__ float* chunks() const { return b2s() + 16; }                         // [sets][h, dh][128][17]
 
   // once per block: W2 transposed (j-major, rows of 12: ten classes at most, then b1[j], then zero) into shared
   // memory, so that the three 16-byte reads of a row bring the bias along
@@ -492,6 +493,7 @@ struct FusedEpi {
       const int j = i / 12, c = i - 12 * j;
       w[i] = (c < C) ? __ldg(W2 + (size_t)c * H + j) : (c == 10 ? __ldg(b1 + j) : 0.f);
     }
+    if (et < 16) b2s()[et] = (et < C) ? __ldg(W2 + (size_t)C * H + et) : 0.f;
   }
 
   // One tile.  tmem_acc: the accumulator's first column; released(): called by every epilogue thread after its last
@@ -512,7 +514,7 @@ struct FusedEpi {
     float* chunk_d = chunk_h + kFusedPlane;
     float* red = chunk_h;                    // [16][11][16] partial column sums, reuses both chunk planes
     float* zpart = ch;                       // [sets][128][12] partial scores of the sets, before the chunks are used
-    const float* __restrict__ b2 = P.theta + (long long)H * F + H + (long long)C * H;
+    const float* b2 = b2s();                 // shared-memory copy
     const long long n = P.N[m];
     const long long trow = (long long)tile * umma::kTileM + tt;   // row within the worker's shard
     const bool valid = trow < n && win.contains(trow);
@@ -558,18 +560,26 @@ struct FusedEpi {
     double loss = 0.0;
     {  // every set does the softmax of the row (the same arithmetic), set 0 keeps the loss and publishes dZ
       float z[12];
+      {  // the sets' partials in order, three 16-byte reads per set
+        const float4* zp4 = reinterpret_cast<const float4*>(zpart + tt * 12);
+        const float4 a0 = zp4[0], a1 = zp4[1], a2 = zp4[2];
+        z[0] = a0.x; z[1] = a0.y; z[2] = a0.z; z[3] = a0.w;
+        z[4] = a1.x; z[5] = a1.y; z[6] = a1.z; z[7] = a1.w;
+        z[8] = a2.x; z[9] = a2.y; z[10] = a2.z; z[11] = a2.w;
 #pragma unroll
-      for (int c = 0; c < 12; ++c) {
-        float zs = zpart[tt * 12 + c];
-#pragma unroll
-        for (int s2 = 1; s2 < kFusedSets; ++s2) zs += zpart[(s2 * 128 + tt) * 12 + c];   // the sets' partials in order
-        z[c] = zs;
+        for (int s2 = 1; s2 < kFusedSets; ++s2) {
+          const float4* p4 = zp4 + s2 * (128 * 12 / 4);
+          const float4 b0 = p4[0], b1q = p4[1], b2q = p4[2];
+          z[0] += b0.x; z[1] += b0.y; z[2] += b0.z; z[3] += b0.w;
+          z[4] += b1q.x; z[5] += b1q.y; z[6] += b1q.z; z[7] += b1q.w;
+          z[8] += b2q.x; z[9] += b2q.y; z[10] += b2q.z; z[11] += b2q.w;
+        }
       }
       float zmax = -3.0e38f;
 #pragma unroll
       for (int c = 0; c < 12; ++c)
         if (c < C) {
-          z[c] += __ldg(b2 + c);
+          z[c] += b2[c];
           zmax = fmaxf(zmax, z[c]);
         }
       float e[12], sum = 0.f;
@@ -584,7 +594,12 @@ struct FusedEpi {
       for (int c = 0; c < 12; ++c) {
         if (c == yv) zy = z[c];
         dz[c] = (valid && c < C) ? (e[c] * inv - (c == yv ? 1.f : 0.f)) : 0.f;
-        if (set == 0) dzs[tt * 12 + c] = dz[c];
+      }
+      if (set == 0) {
+        float4* d4 = reinterpret_cast<float4*>(dzs + tt * 12);
+        d4[0] = make_float4(dz[0], dz[1], dz[2], dz[3]);
+        d4[1] = make_float4(dz[4], dz[5], dz[6], dz[7]);
+        d4[2] = make_float4(dz[8], dz[9], dz[10], dz[11]);
       }
       if (valid && set == 0) loss = (double)((zmax + logf(sum)) - zy);
     }
