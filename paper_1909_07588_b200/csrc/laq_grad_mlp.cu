@@ -458,7 +458,7 @@ constexpr int kFusedPitch = kFusedChunk + 1;           // row pitch of a chunk p
 constexpr int kFusedPlane = 128 * kFusedPitch;         // one plane: 128 rows of a chunk
 
 __host__ __device__ inline size_t fused_extra_floats(int H) {
-  return (size_t)H * 12 + 16 + (size_t)kFusedSets * 2 * kFusedPlane + 128 * 12 + (size_t)12 * H + (size_t)((H + 3) & ~3) + 16;
+  return (size_t)H * 12 + 16 + (size_t)kFusedSets * 2 * kFusedPlane + 128 * 12 + 16;
 }
 __host__ __device__ inline size_t fused_smem_bytes(int nt, int H) {
   return kFusedStages * umma::stage_bytes(nt) + 1024 + fused_extra_floats(H) * 4;
@@ -507,9 +507,9 @@ struct FusedEpi {
     const float* w2 = w2t();
     float* ch = chunks();
     float* dzs = ch + kFusedSets * 2 * kFusedPlane;   // [128][12]
-    float* accA = dzs + 128 * 12;            // [12][H]
-    float* accB = accA + (size_t)12 * H;     // [H]   column sums of dh: the b1 gradient
-    double* lossw = reinterpret_cast<double*>(accB + ((H + 3) & ~3));      // [4] (8-byte aligned: all sizes even)
+    double* lossw = reinterpret_cast<double*>(dzs + 128 * 12);             // [4]
+    // the tile's partials in memory: [db1 (H) | dW2 (C H) | db2 (C)]
+    float* sp = D.spart + ((long long)m * D.gb + tile) * (H + C * H + C);
     float* chunk_h = ch + set * (2 * kFusedPlane);   // this set's h chunk, the dh chunk behind it
     float* chunk_d = chunk_h + kFusedPlane;
     float* red = chunk_h;                    // [16][11][16] partial column sums, reuses both chunk planes
@@ -701,30 +701,24 @@ struct FusedEpi {
           float sum = 0.f;
 #pragma unroll
           for (int gq = 0; gq < 16; ++gq) sum += red[(gq * 11 + k) * kFusedChunk + cc];
-          if (k < 10) accA[k * H + j] = sum; else accB[j] = sum;
+          if (k < C) sp[H + k * H + j] = sum;              // dW2[k][j]
+          else if (k == 10) sp[j] = sum;                   // db1[j]
         }
       }
       sync_set(set);
     }
     if (!released_yet) released();                         // a set without chunks never read the accumulator
-    // ---- the tile's partials: [db1 (H) | dW2 (C H) | db2 (C)] and the loss
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, o);
-    if (lane == 0 && set == 0) lossw[q] = loss;
-    sync_all();
-    const int gb = D.gb;
-    float* sp = D.spart + ((long long)m * gb + tile) * (H + C * H + C);
-    for (int j = et; j < H; j += kFusedEpiThreads) {
-      sp[j] = accB[j];
-      for (int c = 0; c < C; ++c) sp[H + c * H + j] = accA[c * H + j];
-    }
+    // ---- db2 and the loss (every set has written the column sums of its own chunks above)
     if (set == 1 && tt < C) {
       float s = 0.f;
       for (int r = 0; r < 128; ++r) s += dzs[r * 12 + tt];
       sp[H + C * H + tt] = s;
     }
-    if (et == 0) D.lpart[(long long)m * gb + tile] = ((lossw[0] + lossw[1]) + lossw[2]) + lossw[3];
-    sync_all();   // the scratch is free for the next tile
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, o);
+    if (lane == 0 && set == 0) lossw[q] = loss;
+    sync_all();   // the scratch is free for the next tile (its loss terms are only written again after two more of these)
+    if (et == 0) D.lpart[(long long)m * D.gb + tile] = ((lossw[0] + lossw[1]) + lossw[2]) + lossw[3];
   }
 };
 
